@@ -1,0 +1,267 @@
+/*
+ * bcp.h - C ABI of the B200 load-time checkpoint resharding engine.
+ *
+ * The library implements the device-side hot path of load-time resharding as the
+ * ByteCheckpoint paper (arXiv 2407.20143) states the problem:
+ *
+ *   - every tensor has a fully qualified name (FQN) and a global shape
+ *     (Sec. 3.2, "Model and optimizer states");
+ *   - every saved or wanted shard is an index tuple (fqn, nD_offsets, nD_lengths)
+ *     inside that global shape: the ShardMeta (Sec. 3.2);
+ *   - a ByteMeta gives the byte start offset and length of the shard inside its
+ *     storage file (Sec. 3.2, "Checkpoint representation");
+ *   - an irregular shard (a 1-D slice of a flattened tensor, as ZeRO / FSDP produce)
+ *     is represented by several regular ShardMeta entries
+ *     (Sec. 3.2, "Decomposing irregular tensors");
+ *   - at load time each new shard is matched against the saved shards and the
+ *     matching segments are copied into it (Sec. 3.3, Step 2 and Step 5).
+ *
+ * A "storage file" is a device buffer here (a blob); all source ranks and all target
+ * ranks are separate buffers on ONE GPU.  No numeric conversion happens anywhere:
+ * the engine moves raw bytes.
+ *
+ * Conventions
+ *   - Every function returns an int: BCP_OK (0) or a negative bcp_status.  A failing
+ *     call leaves its outputs untouched and launches nothing.  bcp_last_error()
+ *     returns a thread-local, NUL-terminated description of the last failure on the
+ *     calling thread (valid until that thread's next failing call).
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are addresses in the
+ *     memory of the CUDA device that is current when the call is made.
+ *   - `stream` arguments are CUDA stream handles (cudaStream_t) passed as void*;
+ *     NULL is the legacy default stream.
+ *   - Nothing here throws, aborts or traps the device.
+ */
+#ifndef BCP_H_
+#define BCP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BCP_MAX_NDIM 8
+
+typedef enum {
+  BCP_OK = 0,
+  BCP_ERR_INVALID = -1,   /* null pointer, bad ndim/itemsize/kind, negative length, box outside the
+                             global shape, byte_length != element count * itemsize, bad option    */
+  BCP_ERR_MISMATCH = -2,  /* entries of one FQN disagree on itemsize, dtype_tag, ndim or global shape */
+  BCP_ERR_OVERLAP = -3,   /* two source entries of one FQN hold the same element                 */
+  BCP_ERR_UNCOVERED = -4, /* some element of a target entry is held by no source entry           */
+  BCP_ERR_BOUNDS = -5,    /* a byte range reaches past the size given for its buffer              */
+  BCP_ERR_DST_ALIAS = -6, /* two target entries write overlapping byte ranges of one buffer       */
+  BCP_ERR_CUDA = -7,      /* a CUDA runtime call failed (message carries the CUDA error string)   */
+  BCP_ERR_NOMEM = -8,     /* host allocation failed                                               */
+  BCP_ERR_DEVICE_TIMEOUT = -9, /* a bounded device-side wait gave up (TMA path only)              */
+  BCP_ERR_CAPACITY = -10  /* an output array supplied by the caller is too small                  */
+} bcp_status;
+
+typedef enum { BCP_BOX = 0, BCP_FLAT_SLICE = 1 } bcp_kind;
+
+/*
+ * One entry of the paper's TensorShardToBasicByteMap (Sec. 3.2): ShardMeta
+ * (fqn, offsets, lengths) + the part of BasicMeta that matters for raw bytes
+ * (itemsize, dtype_tag) + ByteMeta (buf_index, byte_offset, byte_length).
+ *
+ * Layout of the bytes (the paper gives only offset and length): the entry's elements are
+ * stored densely in C (row-major) order.
+ *   BCP_BOX        : the box offsets[0..ndim) + lengths[0..ndim) of the global tensor.
+ *   BCP_FLAT_SLICE : elements [flat_begin, flat_end) of the C-order flattening of the
+ *                    box offsets/lengths (the rank's local tensor), i.e. an irregular
+ *                    shard; the library decomposes it into regular boxes itself.
+ * ndim == 0 is a scalar (one element).  Zero-volume entries are legal and produce no work.
+ */
+typedef struct {
+  const char* fqn;      /* host, NUL-terminated, caller-owned; read only during bcp_plan       */
+  uint32_t itemsize;    /* bytes per element: 1, 2, 4 or 8                                      */
+  uint32_t dtype_tag;   /* opaque dtype identity; must agree across all entries of an FQN       */
+  uint32_t ndim;        /* 0..BCP_MAX_NDIM                                                      */
+  uint32_t kind;        /* bcp_kind                                                             */
+  int64_t global_shape[BCP_MAX_NDIM];
+  int64_t offsets[BCP_MAX_NDIM];
+  int64_t lengths[BCP_MAX_NDIM];
+  int64_t flat_begin;   /* BCP_FLAT_SLICE only; 0 <= flat_begin <= flat_end <= prod(lengths)    */
+  int64_t flat_end;
+  uint32_t buf_index;   /* source: which blob; target: which target-rank buffer                 */
+  uint32_t reserved;    /* must be 0                                                            */
+  uint64_t byte_offset; /* ByteMeta start inside that buffer                                    */
+  uint64_t byte_length; /* ByteMeta length = element count * itemsize                           */
+} bcp_shard_meta;
+
+/* Planner / launch options.  Zero in any field selects the default written beside it. */
+typedef struct {
+  uint32_t tile_bytes;     /* payload of one CTA-wide work unit; default 65536; multiple of 4096      */
+  uint32_t small_bytes;    /* work units with a payload below this go to the warp path; default 4096  */
+  uint32_t block_threads;  /* threads per CTA of the copy kernel: 128..1024, multiple of 32; default 512 */
+  uint32_t ctas_per_sm;    /* persistent CTAs per SM; default 2                                       */
+  uint32_t order;          /* 0 default (= 1); 1 order work by source address (replica reads of one
+                              source region run back to back and hit L2); 2 order by target address    */
+  uint32_t path_mask;      /* 0 default (= all); bit 0 register (LDG/STG) path, bit 1 TMA staging path */
+  uint32_t cache_hints;    /* 0 default (= 1); 1 streaming loads and stores; 2 plain accesses          */
+  uint32_t reserved[9];    /* must be 0 */
+} bcp_plan_opts;
+
+typedef struct bcp_plan bcp_plan_t;
+
+/*
+ * One unit of the flat work list the planner produces and the kernels execute:
+ * rows x row_bytes bytes from src_buf at src_off (rows src_pitch apart) to dst_buf at
+ * dst_off (rows dst_pitch apart).  Pitches are 0 when rows == 1.
+ */
+typedef struct {
+  uint64_t src_off;
+  uint64_t dst_off;
+  uint64_t src_pitch;
+  uint64_t dst_pitch;
+  uint32_t row_bytes;
+  uint32_t rows;
+  uint32_t src_buf;
+  uint32_t dst_buf;
+  uint32_t flags;       /* BCP_TILE_* */
+  uint32_t reserved[3];
+} bcp_tile;
+
+#define BCP_TILE_GRAN_MASK 0x7u /* log2 of the widest power-of-two access (<= 16 B) that divides
+                                   src_off, dst_off, row_bytes and both pitches                  */
+#define BCP_TILE_ZERO 0x8u      /* no source: write zero bytes (pack padding)                    */
+#define BCP_TILE_SMALL 0x10u    /* executed by one warp                                          */
+#define BCP_TILE_TMA 0x20u      /* eligible for the TMA staging path                             */
+
+typedef struct {
+  uint64_t n_src_entries;    /* after decomposing flat slices                        */
+  uint64_t n_dst_entries;
+  uint64_t n_fqns;
+  uint64_t n_intersections;  /* non-empty source x target box intersections          */
+  uint64_t n_items;          /* after dimension collapse and coalescing               */
+  uint64_t n_tiles;          /* CTA-wide work units                                   */
+  uint64_t n_small_tiles;    /* warp work units                                       */
+  uint64_t n_strided_tiles;  /* work units with rows > 1                              */
+  uint64_t n_tma_tiles;      /* work units eligible for the TMA path                  */
+  uint64_t bytes_copied;     /* payload bytes the list writes = sum of target bytes   */
+  uint64_t bytes_src_unique; /* distinct source bytes the list reads                  */
+  uint64_t bytes_misaligned; /* payload in units whose access granularity is < 16 B   */
+  double plan_ms;            /* host time spent in bcp_plan                           */
+} bcp_plan_stats_t;
+
+/* ByteMeta of one tensor inside a packed blob (Sec. 3.2): start offset and length. */
+typedef struct {
+  uint64_t byte_offset;
+  uint64_t byte_length;
+} bcp_pack_meta;
+
+/* Library version (major*10000 + minor*100 + patch). Never fails. */
+int bcp_version(void);
+
+/* Thread-local message of the last failing call on this thread ("" if none). */
+const char* bcp_last_error(void);
+
+/*
+ * Irregular-tensor decomposition (Sec. 3.2, "Decomposing irregular tensors").
+ * Elements [flat_begin, flat_end) of the C-order flattening of a dense local tensor of
+ * shape lengths[0..ndim) are rewritten as the fewest regular boxes, listed in flat order;
+ * each box is a contiguous sub-range of the flattening and together they tile the range.
+ * out_off / out_len (host, caller-owned, cap rows of BCP_MAX_NDIM) receive box offsets and
+ * lengths RELATIVE to the local tensor; *n receives the box count (at most 2*ndim - 1,
+ * 0 for an empty range).  BCP_ERR_CAPACITY if cap is too small (then *n is the needed count).
+ */
+int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int64_t flat_end,
+                  int64_t (*out_off)[BCP_MAX_NDIM], int64_t (*out_len)[BCP_MAX_NDIM], size_t cap,
+                  size_t* n);
+
+/*
+ * Load-time matching and plan construction (Sec. 3.3, Step 2; plan reuse: Sec. 4.1,
+ * "Plan and metadata cache").  Host only: no device is touched, so it also runs on a
+ * machine without a GPU.
+ *
+ * src[n_src] are the saved entries, dst[n_dst] the wanted ones; src_buf_bytes[n_src_bufs]
+ * and dst_buf_bytes[n_dst_bufs] give each buffer's size for bounds checks.  All arrays are
+ * host memory, caller-owned, read only during the call.  For every target entry the
+ * planner finds all source entries of the same FQN whose boxes intersect it, checks that
+ * they cover it exactly once, and lowers every intersection to work units
+ * (bcp_tile).  Source entries of one FQN must be pairwise disjoint; target entries may
+ * overlap one another as boxes (replicas) but not as byte ranges.
+ * On success *out_plan owns host (and, after the first bcp_reshard, device) copies of the
+ * work list; release it with bcp_plan_destroy.  A plan holds no buffer addresses and can
+ * be executed any number of times on any buffers of the planned sizes.
+ */
+int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes,
+             size_t n_src_bufs, const bcp_shard_meta* dst, size_t n_dst,
+             const uint64_t* dst_buf_bytes, size_t n_dst_bufs, const bcp_plan_opts* opts,
+             bcp_plan_t** out_plan);
+
+int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out);
+
+/*
+ * Host copy of the work list, in execution order (CTA-wide units first, then warp
+ * units).  Writes min(cap, count) records to out (may be NULL when cap == 0) and the
+ * full count to *n.
+ */
+int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n);
+
+/*
+ * Execute a plan (Sec. 3.3, Step 5: copy every matched segment into its target shard).
+ * src_blobs[n_src_bufs] and dst_bufs[n_dst_bufs] are HOST arrays of DEVICE pointers, at
+ * least as large as planned; counts must equal the planned ones.  The call uploads the
+ * work list on first use, enqueues the pointer tables and the copy kernel on `stream`
+ * and returns without waiting; buffers must stay valid until the stream reaches that
+ * point.  Executions of one plan must be ordered (same stream, or externally
+ * synchronised): they share the plan's device-side pointer tables and ticket counter.
+ * Target bytes not named by any target entry are left untouched.
+ */
+int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs,
+                void* const* dst_bufs, size_t n_dst_bufs, void* stream);
+
+/*
+ * Same operation with HOST buffers (host pointers to host memory, pinned for full speed):
+ * copies every source blob to plan-owned device staging memory, runs the kernels,
+ * copies every target buffer back, all on `stream`, and waits for completion.
+ * Target bytes not named by any target entry come back as zero.
+ */
+int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
+                     void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);
+
+/*
+ * Device status word of the plan's last finished execution: 0, or BCP_ERR_DEVICE_TIMEOUT
+ * if a bounded wait in the TMA path gave up (the rest of that unit was then copied
+ * through registers, so the result is still complete).  Synchronises `stream`.
+ */
+int bcp_plan_device_status(bcp_plan_t* plan, void* stream);
+
+/* Waits for the plan's last execution, frees host and device memory. NULL is accepted. */
+int bcp_plan_destroy(bcp_plan_t* plan);
+
+/*
+ * Blob layout for a rank's tensors (ByteMeta table, Sec. 3.2): tensor i of
+ * tensor_bytes[i] bytes starts at out_offsets[i], the smallest multiple of `align`
+ * (a power of two >= 16) not below the end of tensor i-1; *out_blob_bytes is the end of
+ * the last tensor rounded up to `align`.  Host arrays, caller-owned.
+ */
+int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint64_t* out_offsets,
+                    uint64_t* out_blob_bytes);
+
+/*
+ * Pack n tensors into one contiguous save blob (the device-side stand-in for the
+ * serialisation step of the save pipeline, Sec. 4.2): tensors[i] (device pointer,
+ * metas[i].byte_length bytes) is copied to blob + metas[i].byte_offset; every blob byte
+ * in [0, blob_bytes) that belongs to no tensor is written as zero.  metas must be sorted
+ * by byte_offset and non-overlapping, inside blob_bytes.  tensors and metas are host
+ * arrays.  Asynchronous on `stream`.  Work lists are cached inside the library per
+ * (metas, blob_bytes), so repeated packs of the same layout only upload pointers.
+ */
+int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,
+             uint64_t blob_bytes, void* stream);
+
+/* Inverse of bcp_pack (the deserialisation step of the load pipeline, Sec. 4.2):
+ * blob + metas[i].byte_offset -> tensors[i].  Padding is ignored. */
+int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_meta* metas, size_t n,
+               void* const* tensors, void* stream);
+
+/* Drops the cached pack / unpack work lists (waits for their last executions). */
+int bcp_pack_cache_clear(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCP_H_ */

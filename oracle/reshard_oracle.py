@@ -1,0 +1,169 @@
+"""CPU oracle for load-time checkpoint resharding and save-blob packing.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition the CUDA library is
+checked against; it shares no code with the library and must never be imported by the
+product path (only by tests/, the smoke check and the CPU-baseline leg of the benchmark).
+
+What it computes follows the paper's representation (arXiv 2407.20143):
+  * a tensor is named by its FQN and has a global shape; a shard is the box
+    (nD_offsets, nD_lengths) of that shape (Sec. 3.2, "Model and optimizer states");
+  * a ByteMeta locates the shard's bytes in a storage file (Sec. 3.2, "Checkpoint
+    representation"); bytes are the shard's elements densely in C order;
+  * an irregular shard is a contiguous range of the C-order flattening of a rank's local
+    tensor (Sec. 3.2, "Decomposing irregular tensors");
+  * loading under a new parallelism gives every new shard the elements of the saved
+    shards that fall into it (Sec. 3.3, Step 2 and Step 5).
+The method reaches exactly the result with a plain definition, so the oracle is that
+definition: per FQN, ASSEMBLE the full global tensor from the saved shards by slice
+assignment, then SLICE it once per wanted shard.  Irregular shards go through `ravel()` of
+their local box; the oracle never decomposes them into boxes.  Everything is moved as
+unsigned integers of the element size, never as floats.
+
+Entries are duck-typed objects with the attributes fqn, itemsize, dtype_tag, global_shape,
+offsets, lengths, kind (0 box, 1 flat slice), flat_begin, flat_end, buf_index, byte_offset,
+byte_length.
+
+Pins (tests/test_oracle_pins.py): the paper's worked example of an irregular shard, the
+identity / round-trip / exact-cover invariants, textbook reductions to numpy concatenate
+and split, a brute-force per-element index map on tiny inputs, and the closed-form
+index-pattern fill.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+from collections import defaultdict
+from typing import Dict, Iterable, List, Sequence, Tuple
+
+import numpy as np
+
+_UINT = {1: np.uint8, 2: np.uint16, 4: np.uint32, 8: np.uint64}
+FLAT_SLICE = 1
+
+
+class OracleError(ValueError):
+    pass
+
+
+def _box(e) -> Tuple[slice, ...]:
+    return tuple(slice(int(o), int(o) + int(l)) for o, l in zip(e.offsets, e.lengths))
+
+
+def _payload(blob: np.ndarray, e) -> np.ndarray:
+    """The entry's bytes, viewed as a 1-D array of unsigned integers of the element size."""
+    raw = blob[e.byte_offset:e.byte_offset + e.byte_length]
+    if raw.size != e.byte_length:
+        raise OracleError(f"{e.fqn}: byte range outside its buffer")
+    return np.ascontiguousarray(raw).view(_UINT[e.itemsize])
+
+
+def check_family(entries: Sequence) -> Tuple[Tuple[int, ...], int]:
+    """All entries of one FQN must agree on global shape and dtype (Sec. 3.2)."""
+    e0 = entries[0]
+    for e in entries:
+        if (tuple(e.global_shape) != tuple(e0.global_shape) or e.itemsize != e0.itemsize
+                or e.dtype_tag != e0.dtype_tag):
+            raise OracleError(f"{e.fqn}: entries disagree on global shape or dtype")
+        for o, l, g in zip(e.offsets, e.lengths, e.global_shape):
+            if o < 0 or l < 0 or o + l > g:
+                raise OracleError(f"{e.fqn}: box outside the global shape")
+    return tuple(int(g) for g in e0.global_shape), int(e0.itemsize)
+
+
+def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payloads: Sequence[np.ndarray]):
+    """Full global tensor from saved shards, plus how many shards supplied each element.
+
+    Sec. 3.2: shard i covers the box offsets_i + lengths_i of the global shape; an irregular
+    shard covers elements [flat_begin, flat_end) of the flattened local box.
+    """
+    T = np.zeros(tuple(global_shape), dtype=_UINT[itemsize])
+    cover = np.zeros(tuple(global_shape), dtype=np.uint8)
+    for e, data in zip(entries, payloads):
+        b = _box(e)
+        if e.kind == FLAT_SLICE:
+            a, z = int(e.flat_begin), int(e.flat_end)
+            # values: flatten the local box, overwrite [a, z), put the box back
+            tmp = T[b].ravel()
+            tmp[a:z] = data
+            T[b] = tmp.reshape(T[b].shape)
+            # the same for the coverage count
+            cnt = cover[b].ravel()
+            cnt[a:z] += 1
+            cover[b] = cnt.reshape(cover[b].shape)
+        else:
+            T[b] = data.reshape(tuple(int(l) for l in e.lengths))
+            cover[b] += 1
+    return T, cover
+
+
+def take(T: np.ndarray, cover: np.ndarray, e) -> np.ndarray:
+    """Bytes of the wanted shard e cut out of the assembled tensor (uint8, C order)."""
+    b = _box(e)
+    if e.kind == FLAT_SLICE:
+        a, z = int(e.flat_begin), int(e.flat_end)
+        vals, cov = T[b].ravel()[a:z], cover[b].ravel()[a:z]
+    else:
+        vals, cov = T[b].ravel(), cover[b].ravel()
+    if cov.size and cov.min() < 1:
+        raise OracleError(f"{e.fqn}: wanted element held by no saved shard")
+    if cov.size and cov.max() > 1:
+        raise OracleError(f"{e.fqn}: element held by more than one saved shard")
+    return np.ascontiguousarray(vals).view(np.uint8)
+
+
+def group_by_fqn(entries: Iterable) -> Dict[str, List]:
+    g: Dict[str, List] = defaultdict(list)
+    for e in entries:
+        g[e.fqn].append(e)
+    return g
+
+
+def reshard_fqn(src_entries: Sequence, src_payloads: Sequence[np.ndarray], dst_entries: Sequence) -> List[np.ndarray]:
+    """Bytes of every wanted shard of ONE FQN, given the payloads of its saved shards."""
+    shape, itemsize = check_family(list(src_entries) + list(dst_entries))
+    T, cover = assemble(shape, itemsize, src_entries, src_payloads)
+    return [take(T, cover, d) for d in dst_entries]
+
+
+def reshard(src_metas: Sequence, src_blobs: Sequence[np.ndarray], dst_metas: Sequence,
+            dst_buf_bytes: Sequence[int], fill_byte: int = 0) -> List[np.ndarray]:
+    """Every target rank buffer (uint8 arrays); bytes no entry names keep `fill_byte`."""
+    out = [np.full(int(n), fill_byte, dtype=np.uint8) for n in dst_buf_bytes]
+    src_by, dst_by = group_by_fqn(src_metas), group_by_fqn(dst_metas)
+    for fqn, dsts in dst_by.items():
+        srcs = src_by.get(fqn, [])
+        if not srcs:
+            if all(d.byte_length == 0 for d in dsts):
+                continue
+            raise OracleError(f"{fqn}: wanted but never saved")
+        payloads = [_payload(src_blobs[s.buf_index], s) for s in srcs]
+        for d, data in zip(dsts, reshard_fqn(srcs, payloads, dsts)):
+            buf = out[d.buf_index]
+            if d.byte_offset + d.byte_length > buf.size:
+                raise OracleError(f"{fqn}: target byte range outside its buffer")
+            buf[d.byte_offset:d.byte_offset + d.byte_length] = data
+    return out
+
+
+# --------------------------------------------------------------------------- pack / unpack
+def pack_layout(sizes: Sequence[int], align: int = 256) -> Tuple[List[int], int]:
+    """ByteMeta table of a save blob (Sec. 3.2): tensor i starts at the end of tensor i-1
+    rounded up to `align`; the blob ends at the last end rounded up."""
+    offs, pos = [], 0
+    for n in sizes:
+        pos = -(-pos // align) * align
+        offs.append(pos)
+        pos += int(n)
+    return offs, -(-pos // align) * align
+
+
+def pack(tensors: Sequence[np.ndarray], align: int = 256):
+    """One contiguous blob: tensor bytes at the table's offsets, zero bytes elsewhere."""
+    raws = [np.ascontiguousarray(t).reshape(-1).view(np.uint8) for t in tensors]
+    offs, total = pack_layout([r.size for r in raws], align)
+    blob = np.zeros(total, dtype=np.uint8)
+    for r, o in zip(raws, offs):
+        blob[o:o + r.size] = r
+    return blob, [(o, r.size) for r, o in zip(raws, offs)]
+
+
+def unpack(blob: np.ndarray, table: Sequence[Tuple[int, int]]) -> List[np.ndarray]:
+    return [blob[o:o + n].copy() for (o, n) in table]

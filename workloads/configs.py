@@ -1,0 +1,107 @@
+"""The five benchmark configurations and the small scenario cases, as metadata.
+
+cfg1..cfg5 restate the shapes and parallelism changes the benchmark definition names; the
+scenario cases restate the parallelism transitions the paper itself exercises (Sec. 6.4 /
+Appendix E: PP, TP, DP and hybrid changes from TP1.DP4.PP4; Fig. 2: 8 -> 6 -> 4 workers;
+Table 3: ZeRO-2 32 -> 64 and 128 -> 64 ranks, DP75 <-> DP150) on a tiny model.
+"""
+from __future__ import annotations
+
+from typing import Callable, Dict, List
+
+from .layouts import (ModelSpec, Parallelism, ReshardCase, StateKinds, gpt_model, llama_model,
+                      moe_model, reshard_case)
+from .meta import DTYPE_BF16, DTYPE_F32
+
+MIXED = StateKinds()  # bf16 params + fp32 master / exp_avg / exp_avg_sq
+PARAMS_ONLY = StateKinds(optim=())
+OPTIM_ONLY = StateKinds(param_dtype=None)
+MOE_KINDS = StateKinds(optim=("exp_avg",))
+
+
+def cfg1(fill: str = "uniform") -> ReshardCase:
+    m = gpt_model("gpt-tiny", L=2, H=256, F=1024, V=1024, P=128)
+    return reshard_case("cfg1-tiny-gpt", m, Parallelism(tp=2, dp=2, zero="zero1"),
+                        Parallelism(tp=1, dp=4, zero="zero1"), MIXED, fill, seed=0)
+
+
+def cfg2(layers: int = 24) -> ReshardCase:
+    """GPT-3 1.3B shape.  `layers` < 24 keeps the per-layer shapes and shrinks the depth (used
+    for profiler captures that must stay small)."""
+    m = gpt_model("gpt3-1.3b", L=layers, H=2048, F=8192, V=50304, P=2048)
+    return reshard_case("cfg2-gpt3-1.3b" + ("" if layers == 24 else f"-L{layers}"), m,
+                        Parallelism(tp=4, pp=2, dp=2, zero="zero1"),
+                        Parallelism(tp=2, pp=1, dp=4, zero="zero1"), MIXED, "normal", seed=20145)
+
+
+def cfg3(layers: int = 32) -> ReshardCase:
+    m = llama_model("llama3-8b", L=layers, H=4096, nq=32, nkv=8, F=14336, V=128256, fused=True, tied=False)
+    return reshard_case("cfg3-llama3-8b" + ("" if layers == 32 else f"-L{layers}"), m,
+                        Parallelism(tp=8), Parallelism(tp=2), PARAMS_ONLY, "normal", seed=20146)
+
+
+def cfg4(layers: int = 28) -> ReshardCase:
+    m = llama_model("llama-3b-fsdp", L=layers, H=3072, nq=24, nkv=8, F=8192, V=128256, fused=False,
+                    tied=True, fsdp_units=True)
+    return reshard_case("cfg4-llama-3b-fsdp" + ("" if layers == 28 else f"-L{layers}"), m,
+                        Parallelism(dp=64, zero="fsdp"), Parallelism(dp=48, zero="fsdp"),
+                        OPTIM_ONLY, "index", seed=20147)
+
+
+def cfg5(layers: int = 16) -> ReshardCase:
+    m = moe_model("moe-64e", L=layers, H=2048, E=64, F=1408, V=32768)
+    return reshard_case("cfg5-moe" + ("" if layers == 16 else f"-L{layers}"), m,
+                        Parallelism(ep=8), Parallelism(ep=4), MOE_KINDS, "uniform", seed=20148)
+
+
+CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
+    "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
+
+# closed-form byte totals of the full-size configurations (sum over entries)
+EXPECTED_TOTALS = {
+    "cfg1": (26_249_216, 37_498_880),
+    "cfg2": (18_421_473_280, 26_406_256_640),
+    "cfg3": (16_060_522_496, 16_061_054_976),
+    "cfg4": (38_552_997_888, 38_552_997_888),
+    "cfg5": (55_579_127_808, 62_865_850_368),
+}
+
+
+# --------------------------------------------------------------------------- small scenarios
+def small_gpt() -> ModelSpec:
+    return gpt_model("gpt-s", L=8, H=64, F=256, V=512, P=32)
+
+
+def small_llama(fused: bool = True) -> ModelSpec:
+    return llama_model("llama-s", L=4, H=128, nq=8, nkv=2, F=352, V=1000, fused=fused, tied=False)
+
+
+def scenario_cases() -> List[ReshardCase]:
+    g = small_gpt()
+    base = Parallelism(tp=1, dp=4, pp=4, zero="zero1")
+    out = [
+        reshard_case("pp4-to-pp8", g, base, Parallelism(tp=1, dp=4, pp=8, zero="zero1"), MIXED),
+        reshard_case("tp1-to-tp2", g, base, Parallelism(tp=2, dp=4, pp=4, zero="zero1"), MIXED),
+        reshard_case("dp4-to-dp8", g, base, Parallelism(tp=1, dp=8, pp=4, zero="zero1"), MIXED),
+        reshard_case("hybrid", g, base, Parallelism(tp=2, dp=8, pp=2, zero="zero1"), MIXED),
+        reshard_case("workers-8-to-6", g, Parallelism(dp=8, zero="zero1"), Parallelism(dp=6, zero="zero1"), MIXED),
+        reshard_case("workers-6-to-4", g, Parallelism(dp=6, zero="zero1"), Parallelism(dp=4, zero="zero1"), MIXED),
+        reshard_case("dp75-to-dp150", g, Parallelism(tp=4, dp=75, zero="zero1"),
+                     Parallelism(tp=4, dp=150, zero="zero1"), OPTIM_ONLY),
+        reshard_case("dp150-to-dp75", g, Parallelism(tp=4, dp=150, zero="zero1"),
+                     Parallelism(tp=4, dp=75, zero="zero1"), OPTIM_ONLY),
+    ]
+    l = small_llama()
+    out += [
+        reshard_case("llama-tp8-to-tp2", l, Parallelism(tp=8), Parallelism(tp=2), PARAMS_ONLY),
+        reshard_case("llama-tp2-to-tp8", l, Parallelism(tp=2), Parallelism(tp=8), PARAMS_ONLY),
+        reshard_case("fsdp-32-to-64", llama_model("llama-f", 3, 96, 6, 2, 200, 777, fused=False, tied=True,
+                                                  fsdp_units=True),
+                     Parallelism(dp=32, zero="fsdp"), Parallelism(dp=64, zero="fsdp"), OPTIM_ONLY),
+        reshard_case("fsdp-128-to-64", llama_model("llama-f", 3, 96, 6, 2, 200, 777, fused=False, tied=True,
+                                                   fsdp_units=True),
+                     Parallelism(dp=128, zero="fsdp"), Parallelism(dp=64, zero="fsdp"), OPTIM_ONLY),
+        reshard_case("moe-ep8-to-ep4", moe_model("moe-s", 2, 64, 16, 48, 256), Parallelism(ep=8),
+                     Parallelism(ep=4), MOE_KINDS),
+    ]
+    return out
