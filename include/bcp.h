@@ -43,6 +43,12 @@ extern "C" {
 
 #define BCP_MAX_NDIM 8
 
+#if defined(__GNUC__)
+#define BCP_API __attribute__((visibility("default")))
+#else
+#define BCP_API
+#endif
+
 typedef enum {
   BCP_OK = 0,
   BCP_ERR_INVALID = -1,   /* null pointer, bad ndim/itemsize/kind, negative length, box outside the
@@ -152,10 +158,10 @@ typedef struct {
 } bcp_pack_meta;
 
 /* Library version (major*10000 + minor*100 + patch). Never fails. */
-int bcp_version(void);
+BCP_API int bcp_version(void);
 
 /* Thread-local message of the last failing call on this thread ("" if none). */
-const char* bcp_last_error(void);
+BCP_API const char* bcp_last_error(void);
 
 /*
  * Irregular-tensor decomposition (Sec. 3.2, "Decomposing irregular tensors").
@@ -166,7 +172,7 @@ const char* bcp_last_error(void);
  * lengths RELATIVE to the local tensor; *n receives the box count (at most 2*ndim - 1,
  * 0 for an empty range).  BCP_ERR_CAPACITY if cap is too small (then *n is the needed count).
  */
-int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int64_t flat_end,
+BCP_API int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int64_t flat_end,
                   int64_t (*out_off)[BCP_MAX_NDIM], int64_t (*out_len)[BCP_MAX_NDIM], size_t cap,
                   size_t* n);
 
@@ -186,19 +192,19 @@ int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int
  * work list; release it with bcp_plan_destroy.  A plan holds no buffer addresses and can
  * be executed any number of times on any buffers of the planned sizes.
  */
-int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes,
+BCP_API int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes,
              size_t n_src_bufs, const bcp_shard_meta* dst, size_t n_dst,
              const uint64_t* dst_buf_bytes, size_t n_dst_bufs, const bcp_plan_opts* opts,
              bcp_plan_t** out_plan);
 
-int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out);
+BCP_API int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out);
 
 /*
  * Host copy of the work list, in execution order (CTA-wide units first, then warp
  * units).  Writes min(cap, count) records to out (may be NULL when cap == 0) and the
  * full count to *n.
  */
-int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n);
+BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n);
 
 /*
  * Execute a plan (Sec. 3.3, Step 5: copy every matched segment into its target shard).
@@ -210,7 +216,7 @@ int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n)
  * synchronised): they share the plan's device-side pointer tables and ticket counter.
  * Target bytes not named by any target entry are left untouched.
  */
-int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs,
+BCP_API int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs,
                 void* const* dst_bufs, size_t n_dst_bufs, void* stream);
 
 /*
@@ -219,7 +225,7 @@ int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_buf
  * copies every target buffer back, all on `stream`, and waits for completion.
  * Target bytes not named by any target entry come back as zero.
  */
-int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
+BCP_API int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
                      void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);
 
 /*
@@ -227,10 +233,10 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t
  * if a bounded wait in the TMA path gave up (the rest of that unit was then copied
  * through registers, so the result is still complete).  Synchronises `stream`.
  */
-int bcp_plan_device_status(bcp_plan_t* plan, void* stream);
+BCP_API int bcp_plan_device_status(bcp_plan_t* plan, void* stream);
 
 /* Waits for the plan's last execution, frees host and device memory. NULL is accepted. */
-int bcp_plan_destroy(bcp_plan_t* plan);
+BCP_API int bcp_plan_destroy(bcp_plan_t* plan);
 
 /*
  * Blob layout for a rank's tensors (ByteMeta table, Sec. 3.2): tensor i of
@@ -238,7 +244,7 @@ int bcp_plan_destroy(bcp_plan_t* plan);
  * (a power of two >= 16) not below the end of tensor i-1; *out_blob_bytes is the end of
  * the last tensor rounded up to `align`.  Host arrays, caller-owned.
  */
-int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint64_t* out_offsets,
+BCP_API int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint64_t* out_offsets,
                     uint64_t* out_blob_bytes);
 
 /*
@@ -250,16 +256,16 @@ int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint
  * arrays.  Asynchronous on `stream`.  Work lists are cached inside the library per
  * (metas, blob_bytes), so repeated packs of the same layout only upload pointers.
  */
-int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,
+BCP_API int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,
              uint64_t blob_bytes, void* stream);
 
 /* Inverse of bcp_pack (the deserialisation step of the load pipeline, Sec. 4.2):
  * blob + metas[i].byte_offset -> tensors[i].  Padding is ignored. */
-int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_meta* metas, size_t n,
+BCP_API int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_meta* metas, size_t n,
                void* const* tensors, void* stream);
 
 /* Drops the cached pack / unpack work lists (waits for their last executions). */
-int bcp_pack_cache_clear(void);
+BCP_API int bcp_pack_cache_clear(void);
 
 #ifdef __cplusplus
 }

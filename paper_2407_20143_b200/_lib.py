@@ -1,0 +1,113 @@
+"""ctypes view of libbcp.so: structures and prototypes of include/bcp.h, nothing else."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+from . import build as _build
+
+BCP_MAX_NDIM = 8
+
+
+class ShardMetaC(C.Structure):
+    _fields_ = [
+        ("fqn", C.c_char_p),
+        ("itemsize", C.c_uint32),
+        ("dtype_tag", C.c_uint32),
+        ("ndim", C.c_uint32),
+        ("kind", C.c_uint32),
+        ("global_shape", C.c_int64 * BCP_MAX_NDIM),
+        ("offsets", C.c_int64 * BCP_MAX_NDIM),
+        ("lengths", C.c_int64 * BCP_MAX_NDIM),
+        ("flat_begin", C.c_int64),
+        ("flat_end", C.c_int64),
+        ("buf_index", C.c_uint32),
+        ("reserved", C.c_uint32),
+        ("byte_offset", C.c_uint64),
+        ("byte_length", C.c_uint64),
+    ]
+
+
+class PlanOptsC(C.Structure):
+    _fields_ = [
+        ("tile_bytes", C.c_uint32),
+        ("small_bytes", C.c_uint32),
+        ("block_threads", C.c_uint32),
+        ("ctas_per_sm", C.c_uint32),
+        ("order", C.c_uint32),
+        ("path_mask", C.c_uint32),
+        ("cache_hints", C.c_uint32),
+        ("reserved", C.c_uint32 * 9),
+    ]
+
+
+class TileC(C.Structure):
+    _fields_ = [
+        ("src_off", C.c_uint64),
+        ("dst_off", C.c_uint64),
+        ("src_pitch", C.c_uint64),
+        ("dst_pitch", C.c_uint64),
+        ("row_bytes", C.c_uint32),
+        ("rows", C.c_uint32),
+        ("src_buf", C.c_uint32),
+        ("dst_buf", C.c_uint32),
+        ("flags", C.c_uint32),
+        ("reserved", C.c_uint32 * 3),
+    ]
+
+
+class PlanStatsC(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "n_src_entries", "n_dst_entries", "n_fqns", "n_intersections", "n_items", "n_tiles", "n_small_tiles",
+        "n_strided_tiles", "n_tma_tiles", "bytes_copied", "bytes_src_unique", "bytes_misaligned")] + [
+        ("plan_ms", C.c_double)]
+
+
+class PackMetaC(C.Structure):
+    _fields_ = [("byte_offset", C.c_uint64), ("byte_length", C.c_uint64)]
+
+
+_VP = C.c_void_p
+_PROTOS = {
+    "bcp_version": (C.c_int, []),
+    "bcp_last_error": (C.c_char_p, []),
+    "bcp_decompose": (C.c_int, [C.POINTER(C.c_int64), C.c_uint32, C.c_int64, C.c_int64, _VP, _VP, C.c_size_t,
+                                C.POINTER(C.c_size_t)]),
+    "bcp_plan": (C.c_int, [C.POINTER(ShardMetaC), C.c_size_t, C.POINTER(C.c_uint64), C.c_size_t,
+                           C.POINTER(ShardMetaC), C.c_size_t, C.POINTER(C.c_uint64), C.c_size_t,
+                           C.POINTER(PlanOptsC), C.POINTER(_VP)]),
+    "bcp_plan_stats": (C.c_int, [_VP, C.POINTER(PlanStatsC)]),
+    "bcp_plan_tiles": (C.c_int, [_VP, C.POINTER(TileC), C.c_size_t, C.POINTER(C.c_size_t)]),
+    "bcp_reshard": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),
+    "bcp_reshard_host": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),
+    "bcp_plan_device_status": (C.c_int, [_VP, _VP]),
+    "bcp_plan_destroy": (C.c_int, [_VP]),
+    "bcp_pack_layout": (C.c_int, [C.POINTER(C.c_uint64), C.c_size_t, C.c_uint64, C.POINTER(C.c_uint64),
+                                  C.POINTER(C.c_uint64)]),
+    "bcp_pack": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
+    "bcp_unpack": (C.c_int, [_VP, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
+    "bcp_pack_cache_clear": (C.c_int, []),
+}
+
+EXPORTS = tuple(_PROTOS)
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Built on first use if the in-tree .so is missing or older than
+    its sources; raises if it can be neither found nor built (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.is_stale():
+            try:
+                _build.build_library()
+            except Exception as e:  # no compiler here: an existing library is still usable
+                if not os.path.exists(path):
+                    raise ImportError(f"libbcp.so is missing and could not be built: {e}") from e
+        h = C.CDLL(path)
+        for name, (res, args) in _PROTOS.items():
+            f = getattr(h, name)
+            f.restype, f.argtypes = res, args
+        _lib = h
+    return _lib

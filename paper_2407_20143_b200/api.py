@@ -1,0 +1,184 @@
+"""Python binding of the C ABI in include/bcp.h: same names, argument marshalling only.
+
+Every step of the resharding path (decomposition, matching, lowering, the copies) runs
+inside libbcp.so; this module converts Python metadata objects to C structures and torch
+tensors to device pointers.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Optional, Sequence, Tuple
+
+from . import _lib as L
+
+
+class BcpError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"bcp error {code}: {msg}")
+        self.code = code
+
+
+ERR_INVALID, ERR_MISMATCH, ERR_OVERLAP, ERR_UNCOVERED, ERR_BOUNDS, ERR_DST_ALIAS = -1, -2, -3, -4, -5, -6
+ERR_CUDA, ERR_NOMEM, ERR_DEVICE_TIMEOUT, ERR_CAPACITY = -7, -8, -9, -10
+TILE_GRAN_MASK, TILE_ZERO, TILE_SMALL, TILE_TMA = 0x7, 0x8, 0x10, 0x20
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise BcpError(rc, L.lib().bcp_last_error().decode("utf-8", "replace"))
+
+
+def _metas_to_c(metas: Sequence) -> Tuple[C.Array, list]:
+    """Objects with the attributes of workloads.meta.ShardMeta -> array of bcp_shard_meta."""
+    arr = (L.ShardMetaC * max(1, len(metas)))()
+    keep = []
+    for c, m in zip(arr, metas):
+        name = m.fqn.encode()
+        keep.append(name)
+        c.fqn = name
+        c.itemsize, c.dtype_tag, c.ndim, c.kind = m.itemsize, m.dtype_tag, len(m.global_shape), m.kind
+        for k, (g, o, l) in enumerate(zip(m.global_shape, m.offsets, m.lengths)):
+            c.global_shape[k], c.offsets[k], c.lengths[k] = g, o, l
+        c.flat_begin, c.flat_end = m.flat_begin, m.flat_end
+        c.buf_index, c.byte_offset, c.byte_length = m.buf_index, m.byte_offset, m.byte_length
+    return arr, keep
+
+
+def _u64(xs: Sequence[int]) -> C.Array:
+    return (C.c_uint64 * max(1, len(xs)))(*xs)
+
+
+def _ptrs(tensors: Sequence) -> C.Array:
+    return (C.c_void_p * max(1, len(tensors)))(*[t if isinstance(t, int) else t.data_ptr() for t in tensors])
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class Plan:
+    """Owner of a bcp_plan_t handle."""
+
+    def __init__(self, handle: int, n_src_bufs: int, n_dst_bufs: int):
+        self._h = C.c_void_p(handle)
+        self.n_src_bufs, self.n_dst_bufs = n_src_bufs, n_dst_bufs
+
+    @property
+    def handle(self) -> C.c_void_p:
+        if not self._h:
+            raise BcpError(ERR_INVALID, "plan already destroyed")
+        return self._h
+
+    def stats(self) -> dict:
+        st = L.PlanStatsC()
+        _check(L.lib().bcp_plan_stats(self.handle, C.byref(st)))
+        return {n: getattr(st, n) for n, _ in L.PlanStatsC._fields_}
+
+    def tiles(self) -> List[L.TileC]:
+        n = C.c_size_t()
+        _check(L.lib().bcp_plan_tiles(self.handle, None, 0, C.byref(n)))
+        arr = (L.TileC * max(1, n.value))()
+        _check(L.lib().bcp_plan_tiles(self.handle, arr, n.value, C.byref(n)))
+        return list(arr[: n.value])
+
+    def destroy(self) -> None:
+        if self._h:
+            h, self._h = self._h, C.c_void_p(None)
+            _check(L.lib().bcp_plan_destroy(h))
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def bcp_version() -> int:
+    return L.lib().bcp_version()
+
+
+def bcp_decompose(lengths: Sequence[int], flat_begin: int, flat_end: int):
+    """Regular boxes (offsets, lengths), relative to the local tensor, that tile a flat range."""
+    nd = len(lengths)
+    cap = max(1, 2 * nd)
+    off = ((C.c_int64 * L.BCP_MAX_NDIM) * cap)()
+    ln = ((C.c_int64 * L.BCP_MAX_NDIM) * cap)()
+    n = C.c_size_t()
+    la = (C.c_int64 * max(1, nd))(*lengths)
+    _check(L.lib().bcp_decompose(la, nd, flat_begin, flat_end, off, ln, cap, C.byref(n)))
+    return [(tuple(off[i][:nd]), tuple(ln[i][:nd])) for i in range(n.value)]
+
+
+def bcp_plan(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas: Sequence, dst_buf_bytes: Sequence[int],
+             **opts) -> Plan:
+    """Match wanted against saved entries and build the work list (host only)."""
+    sa, keep_s = _metas_to_c(src_metas)
+    da, keep_d = _metas_to_c(dst_metas)
+    o = None
+    if opts:
+        o = L.PlanOptsC()
+        for k, v in opts.items():
+            if not hasattr(o, k) or k == "reserved":
+                raise BcpError(ERR_INVALID, f"unknown plan option {k}")
+            setattr(o, k, v)
+    h = C.c_void_p()
+    _check(L.lib().bcp_plan(sa, len(src_metas), _u64(src_buf_bytes), len(src_buf_bytes), da, len(dst_metas),
+                            _u64(dst_buf_bytes), len(dst_buf_bytes), C.byref(o) if o is not None else None,
+                            C.byref(h)))
+    del keep_s, keep_d
+    return Plan(h.value, len(src_buf_bytes), len(dst_buf_bytes))
+
+
+def bcp_reshard(plan: Plan, src_blobs: Sequence, dst_bufs: Sequence, stream=None) -> None:
+    """Enqueue the copies of `plan` on `stream` (torch stream, raw handle, or None = current).
+    src_blobs / dst_bufs: torch CUDA tensors or raw device addresses."""
+    _check(L.lib().bcp_reshard(plan.handle, _ptrs(src_blobs), len(src_blobs), _ptrs(dst_bufs), len(dst_bufs),
+                               _stream(stream)))
+
+
+def bcp_reshard_host(plan: Plan, src_blobs: Sequence, dst_bufs: Sequence, stream=None) -> None:
+    """Same with host tensors (pinned for full speed); returns when the targets are filled."""
+    _check(L.lib().bcp_reshard_host(plan.handle, _ptrs(src_blobs), len(src_blobs), _ptrs(dst_bufs), len(dst_bufs),
+                                    _stream(stream)))
+
+
+def bcp_plan_device_status(plan: Plan, stream=None) -> None:
+    _check(L.lib().bcp_plan_device_status(plan.handle, _stream(stream)))
+
+
+def bcp_pack_layout(tensor_bytes: Sequence[int], align: int = 256) -> Tuple[List[int], int]:
+    n = len(tensor_bytes)
+    offs = (C.c_uint64 * max(1, n))()
+    total = C.c_uint64()
+    _check(L.lib().bcp_pack_layout(_u64(tensor_bytes), n, align, offs, C.byref(total)))
+    return list(offs[:n]), total.value
+
+
+def _pack_metas(metas: Sequence[Tuple[int, int]]) -> C.Array:
+    arr = (L.PackMetaC * max(1, len(metas)))()
+    for c, (o, n) in zip(arr, metas):
+        c.byte_offset, c.byte_length = o, n
+    return arr
+
+
+def bcp_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_bytes: Optional[int] = None,
+             stream=None) -> None:
+    """tensors[i] -> blob[metas[i] = (byte_offset, byte_length)]; padding bytes become zero."""
+    nb = blob_bytes if blob_bytes is not None else blob.numel() * blob.element_size()
+    bp = blob if isinstance(blob, int) else blob.data_ptr()
+    _check(L.lib().bcp_pack(_ptrs(tensors), _pack_metas(metas), len(tensors), bp, nb, _stream(stream)))
+
+
+def bcp_unpack(blob, metas: Sequence[Tuple[int, int]], tensors: Sequence, blob_bytes: Optional[int] = None,
+               stream=None) -> None:
+    nb = blob_bytes if blob_bytes is not None else blob.numel() * blob.element_size()
+    bp = blob if isinstance(blob, int) else blob.data_ptr()
+    _check(L.lib().bcp_unpack(bp, nb, _pack_metas(metas), len(tensors), _ptrs(tensors), _stream(stream)))
+
+
+def bcp_pack_cache_clear() -> None:
+    _check(L.lib().bcp_pack_cache_clear())

@@ -1,0 +1,382 @@
+// C ABI of the resharding engine: plan objects, execution, pack / unpack.
+#include <chrono>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+#include "plan.hpp"
+
+using namespace bcp;
+
+struct bcp_plan {
+  Options opt;
+  bcp_plan_stats_t stats;
+  std::vector<bcp_tile> tiles;  // CTA-wide units, then warp units
+  size_t n_big = 0;
+  std::vector<uint64_t> src_bytes, dst_bytes;
+  // device side, created by the first execution
+  int device = -1;
+  bcp_tile* d_tiles = nullptr;
+  void** d_ptrs = nullptr;  // source table followed by target table
+  Control* d_ctrl = nullptr;
+  uint32_t grid = 0;
+  cudaStream_t last_stream = nullptr;
+  bool ran = false;
+  std::vector<void*> h_ptrs;
+  // staging for bcp_reshard_host
+  std::vector<void*> stage_src, stage_dst;
+};
+
+namespace {
+
+#define BCP_CUDA(call)                                                                       \
+  do {                                                                                       \
+    cudaError_t e_ = (call);                                                                 \
+    if (e_ != cudaSuccess) return fail(BCP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+int bind_device(bcp_plan_t* p) {
+  int dev = 0;
+  BCP_CUDA(cudaGetDevice(&dev));
+  if (p->device >= 0) {
+    if (p->device != dev) return fail(BCP_ERR_INVALID, "plan is bound to device %d but device %d is current", p->device, dev);
+    return BCP_OK;
+  }
+  const size_t n_ptrs = p->src_bytes.size() + p->dst_bytes.size();
+  if (!p->tiles.empty()) {
+    BCP_CUDA(cudaMalloc(&p->d_tiles, p->tiles.size() * sizeof(bcp_tile)));
+    BCP_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), p->tiles.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
+  }
+  BCP_CUDA(cudaMalloc(&p->d_ptrs, (n_ptrs ? n_ptrs : 1) * sizeof(void*)));
+  BCP_CUDA(cudaMalloc(&p->d_ctrl, sizeof(Control)));
+  BCP_CUDA(cudaMemset(p->d_ctrl, 0, sizeof(Control)));
+  BCP_CUDA(copy_kernel_max_grid(p->opt.block_threads, p->opt.ctas_per_sm, &p->grid));
+  p->h_ptrs.resize(n_ptrs);
+  p->device = dev;
+  return BCP_OK;
+}
+
+int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, size_t nd, cudaStream_t stream) {
+  if (!p) return fail(BCP_ERR_INVALID, "plan is NULL");
+  if (ns != p->src_bytes.size() || nd != p->dst_bytes.size())
+    return fail(BCP_ERR_INVALID, "buffer counts (%zu, %zu) differ from the planned (%zu, %zu)", ns, nd, p->src_bytes.size(),
+                p->dst_bytes.size());
+  if ((ns && !src) || (nd && !dst)) return fail(BCP_ERR_INVALID, "pointer array is NULL");
+  for (size_t i = 0; i < ns; ++i)
+    if (!src[i] && p->src_bytes[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
+  for (size_t i = 0; i < nd; ++i)
+    if (!dst[i] && p->dst_bytes[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
+  if (int rc = bind_device(p)) return rc;
+  if (p->tiles.empty()) return BCP_OK;
+  for (size_t i = 0; i < ns; ++i) p->h_ptrs[i] = const_cast<void*>(src[i]);
+  for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
+  // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
+  BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  LaunchArgs a;
+  a.tiles = p->d_tiles;
+  a.n_big = uint32_t(p->n_big);
+  a.n_small = uint32_t(p->tiles.size() - p->n_big);
+  a.src = reinterpret_cast<const void* const*>(p->d_ptrs);
+  a.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
+  a.ctrl = p->d_ctrl;
+  a.block_threads = p->opt.block_threads;
+  const uint32_t nwarps = a.block_threads / 32;
+  const uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;
+  a.grid = uint32_t(units < p->grid ? units : p->grid);
+  a.cache_hints = p->opt.cache_hints;
+  BCP_CUDA(launch_copy(a, stream));
+  p->last_stream = stream;
+  p->ran = true;
+  return BCP_OK;
+}
+
+bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_stats_t stats,
+                      std::vector<uint64_t> src_bytes, std::vector<uint64_t> dst_bytes) {
+  bcp_plan_t* p = new (std::nothrow) bcp_plan_t;
+  if (!p) return nullptr;
+  p->opt = opt;
+  p->stats = stats;
+  build_tiles(items, opt, &p->tiles, &p->n_big, &p->stats);
+  p->src_bytes = std::move(src_bytes);
+  p->dst_bytes = std::move(dst_bytes);
+  return p;
+}
+
+double ms_since(std::chrono::steady_clock::time_point t0) {
+  return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+}
+
+// ------------------------------------------------------------------ pack / unpack plan cache
+struct PackEntry {
+  bool unpack;
+  uint64_t blob_bytes;
+  std::vector<bcp_pack_meta> metas;
+  bcp_plan_t* plan;
+  uint64_t stamp;
+};
+std::mutex g_pack_mu;
+std::vector<PackEntry> g_pack_cache;
+uint64_t g_pack_stamp = 0;
+const size_t kPackCacheMax = 16;
+
+int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_bytes, bcp_plan_t** out) {
+  for (PackEntry& e : g_pack_cache) {
+    if (e.unpack == unpack && e.blob_bytes == blob_bytes && e.metas.size() == n &&
+        (n == 0 || memcmp(e.metas.data(), metas, n * sizeof(bcp_pack_meta)) == 0)) {
+      e.stamp = ++g_pack_stamp;
+      *out = e.plan;
+      return BCP_OK;
+    }
+  }
+  uint64_t pos = 0;
+  for (size_t i = 0; i < n; ++i) {
+    if (metas[i].byte_offset < pos)
+      return fail(BCP_ERR_INVALID, "pack meta %zu starts at %llu, before the end (%llu) of the previous tensor", i,
+                  (unsigned long long)metas[i].byte_offset, (unsigned long long)pos);
+    if (metas[i].byte_offset > blob_bytes || metas[i].byte_length > blob_bytes - metas[i].byte_offset)
+      return fail(BCP_ERR_BOUNDS, "pack meta %zu reaches past the blob (%llu bytes)", i, (unsigned long long)blob_bytes);
+    pos = metas[i].byte_offset + metas[i].byte_length;
+  }
+  const auto t0 = std::chrono::steady_clock::now();
+  std::vector<Item> items;
+  std::vector<uint64_t> tensor_bytes(n), blob(1, blob_bytes);
+  pos = 0;
+  for (size_t i = 0; i < n; ++i) {
+    tensor_bytes[i] = metas[i].byte_length;
+    Item it;
+    it.row_bytes = metas[i].byte_length;
+    if (!unpack) {
+      if (metas[i].byte_offset > pos) {  // padding before this tensor is written as zeros
+        Item z;
+        z.zero = true;
+        z.dst_off = pos;
+        z.row_bytes = metas[i].byte_offset - pos;
+        items.push_back(z);
+      }
+      it.src_buf = uint32_t(i);
+      it.dst_off = metas[i].byte_offset;
+    } else {
+      it.dst_buf = uint32_t(i);
+      it.src_off = metas[i].byte_offset;
+    }
+    items.push_back(it);
+    pos = metas[i].byte_offset + metas[i].byte_length;
+  }
+  if (!unpack && pos < blob_bytes) {
+    Item z;
+    z.zero = true;
+    z.dst_off = pos;
+    z.row_bytes = blob_bytes - pos;
+    items.push_back(z);
+  }
+  Options opt;
+  opt.order = 2;
+  bcp_plan_stats_t st;
+  memset(&st, 0, sizeof st);
+  st.n_src_entries = unpack ? 1 : n;
+  st.n_dst_entries = unpack ? n : 1;
+  st.n_intersections = n;
+  bcp_plan_t* p = unpack ? finish_plan(items, opt, st, blob, tensor_bytes) : finish_plan(items, opt, st, tensor_bytes, blob);
+  if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
+  uint64_t uniq = 0;
+  for (size_t i = 0; i < n; ++i) uniq += metas[i].byte_length;
+  p->stats.bytes_src_unique = uniq;
+  p->stats.plan_ms = ms_since(t0);
+  if (g_pack_cache.size() >= kPackCacheMax) {
+    size_t victim = 0;
+    for (size_t i = 1; i < g_pack_cache.size(); ++i)
+      if (g_pack_cache[i].stamp < g_pack_cache[victim].stamp) victim = i;
+    bcp_plan_destroy(g_pack_cache[victim].plan);
+    g_pack_cache.erase(g_pack_cache.begin() + victim);
+  }
+  g_pack_cache.push_back(PackEntry{unpack, blob_bytes, std::vector<bcp_pack_meta>(metas, metas + n), p, ++g_pack_stamp});
+  *out = p;
+  return BCP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int bcp_version(void) { return 100; }
+
+const char* bcp_last_error(void) { return last_error().c_str(); }
+
+int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int64_t flat_end,
+                  int64_t (*out_off)[BCP_MAX_NDIM], int64_t (*out_len)[BCP_MAX_NDIM], size_t cap, size_t* n) {
+  if (!n || (ndim && !lengths) || ndim > BCP_MAX_NDIM) return fail(BCP_ERR_INVALID, "bcp_decompose: bad arguments");
+  int64_t vol = 1;
+  for (uint32_t k = 0; k < ndim; ++k) {
+    if (lengths[k] < 0) return fail(BCP_ERR_INVALID, "bcp_decompose: negative length");
+    vol *= lengths[k];
+  }
+  if (flat_begin < 0 || flat_end < flat_begin || flat_end > vol)
+    return fail(BCP_ERR_INVALID, "bcp_decompose: range [%lld, %lld) outside %lld elements", (long long)flat_begin,
+                (long long)flat_end, (long long)vol);
+  std::vector<RelBox> boxes;
+  decompose(lengths, ndim, flat_begin, flat_end, &boxes);
+  *n = boxes.size();
+  if (boxes.size() > cap) return fail(BCP_ERR_CAPACITY, "bcp_decompose: %zu boxes, room for %zu", boxes.size(), cap);
+  if (!boxes.empty() && (!out_off || !out_len)) return fail(BCP_ERR_INVALID, "bcp_decompose: output arrays are NULL");
+  for (size_t i = 0; i < boxes.size(); ++i)
+    for (uint32_t k = 0; k < BCP_MAX_NDIM; ++k) {
+      out_off[i][k] = k < ndim ? boxes[i].off[k] : 0;
+      out_len[i][k] = k < ndim ? boxes[i].len[k] : 0;
+    }
+  return BCP_OK;
+}
+
+int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
+             const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
+             const bcp_plan_opts* opts, bcp_plan_t** out_plan) {
+  if (!out_plan) return fail(BCP_ERR_INVALID, "out_plan is NULL");
+  const auto t0 = std::chrono::steady_clock::now();
+  Options opt;
+  if (int rc = parse_options(opts, &opt)) return rc;
+  try {
+    std::vector<Item> items;
+    bcp_plan_stats_t st;
+    memset(&st, 0, sizeof st);
+    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, &items, &st))
+      return rc;
+    bcp_plan_t* p = finish_plan(items, opt, st, std::vector<uint64_t>(src_buf_bytes, src_buf_bytes + n_src_bufs),
+                              std::vector<uint64_t>(dst_buf_bytes, dst_buf_bytes + n_dst_bufs));
+    if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
+    if (p->tiles.size() > 0xFFFF0000ull) {
+      delete p;
+      return fail(BCP_ERR_INVALID, "work list too long for one launch");
+    }
+    p->stats.plan_ms = ms_since(t0);
+    *out_plan = p;
+  } catch (const std::bad_alloc&) {
+    return fail(BCP_ERR_NOMEM, "out of host memory");
+  }
+  return BCP_OK;
+}
+
+int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out) {
+  if (!plan || !out) return fail(BCP_ERR_INVALID, "bcp_plan_stats: NULL argument");
+  *out = plan->stats;
+  return BCP_OK;
+}
+
+int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n) {
+  if (!plan || !n || (cap && !out)) return fail(BCP_ERR_INVALID, "bcp_plan_tiles: NULL argument");
+  *n = plan->tiles.size();
+  const size_t k = cap < plan->tiles.size() ? cap : plan->tiles.size();
+  if (k) memcpy(out, plan->tiles.data(), k * sizeof(bcp_tile));
+  return BCP_OK;
+}
+
+int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs, void* const* dst_bufs,
+                size_t n_dst_bufs, void* stream) {
+  return execute(plan, src_blobs, n_src_bufs, dst_bufs, n_dst_bufs, static_cast<cudaStream_t>(stream));
+}
+
+int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src_bufs, void* const* dst_host,
+                     size_t n_dst_bufs, void* stream_) {
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
+  if (n_src_bufs != plan->src_bytes.size() || n_dst_bufs != plan->dst_bytes.size())
+    return fail(BCP_ERR_INVALID, "buffer counts differ from the planned ones");
+  if ((n_src_bufs && !src_host) || (n_dst_bufs && !dst_host)) return fail(BCP_ERR_INVALID, "pointer array is NULL");
+  if (int rc = bind_device(plan)) return rc;
+  if (plan->stage_src.empty() && plan->stage_dst.empty()) {
+    plan->stage_src.assign(n_src_bufs, nullptr);
+    plan->stage_dst.assign(n_dst_bufs, nullptr);
+    for (size_t i = 0; i < n_src_bufs; ++i) BCP_CUDA(cudaMalloc(&plan->stage_src[i], plan->src_bytes[i] ? plan->src_bytes[i] : 1));
+    for (size_t i = 0; i < n_dst_bufs; ++i) BCP_CUDA(cudaMalloc(&plan->stage_dst[i], plan->dst_bytes[i] ? plan->dst_bytes[i] : 1));
+  }
+  for (size_t i = 0; i < n_src_bufs; ++i) {
+    if (!plan->src_bytes[i]) continue;
+    if (!src_host[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
+    BCP_CUDA(cudaMemcpyAsync(plan->stage_src[i], src_host[i], plan->src_bytes[i], cudaMemcpyHostToDevice, stream));
+  }
+  for (size_t i = 0; i < n_dst_bufs; ++i)
+    if (plan->dst_bytes[i]) BCP_CUDA(cudaMemsetAsync(plan->stage_dst[i], 0, plan->dst_bytes[i], stream));
+  if (int rc = execute(plan, plan->stage_src.data(), n_src_bufs, plan->stage_dst.data(), n_dst_bufs, stream)) return rc;
+  for (size_t i = 0; i < n_dst_bufs; ++i) {
+    if (!plan->dst_bytes[i]) continue;
+    if (!dst_host[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
+    BCP_CUDA(cudaMemcpyAsync(dst_host[i], plan->stage_dst[i], plan->dst_bytes[i], cudaMemcpyDeviceToHost, stream));
+  }
+  BCP_CUDA(cudaStreamSynchronize(stream));
+  return BCP_OK;
+}
+
+int bcp_plan_device_status(bcp_plan_t* plan, void* stream) {
+  if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
+  if (plan->device < 0) return BCP_OK;
+  BCP_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  Control c;
+  BCP_CUDA(cudaMemcpy(&c, plan->d_ctrl, sizeof c, cudaMemcpyDeviceToHost));
+  if (c.status) return fail(int(c.status) < 0 ? int(c.status) : BCP_ERR_DEVICE_TIMEOUT, "device reported status %d", int(c.status));
+  return BCP_OK;
+}
+
+int bcp_plan_destroy(bcp_plan_t* plan) {
+  if (!plan) return BCP_OK;
+  int rc = BCP_OK;
+  if (plan->device >= 0) {
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != plan->device) cudaSetDevice(plan->device);
+    if (plan->ran && cudaStreamSynchronize(plan->last_stream) != cudaSuccess) {
+      cudaGetLastError();
+      cudaDeviceSynchronize();
+    }
+    for (void* q : plan->stage_src) cudaFree(q);
+    for (void* q : plan->stage_dst) cudaFree(q);
+    cudaFree(plan->d_tiles);
+    cudaFree(plan->d_ptrs);
+    cudaFree(plan->d_ctrl);
+    if (cudaGetLastError() != cudaSuccess) rc = fail(BCP_ERR_CUDA, "bcp_plan_destroy: a CUDA call failed");
+    if (cur != plan->device) cudaSetDevice(cur);
+  }
+  delete plan;
+  return rc;
+}
+
+int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint64_t* out_offsets, uint64_t* out_blob_bytes) {
+  if ((n && (!tensor_bytes || !out_offsets)) || !out_blob_bytes) return fail(BCP_ERR_INVALID, "bcp_pack_layout: NULL argument");
+  if (align < 16 || (align & (align - 1))) return fail(BCP_ERR_INVALID, "bcp_pack_layout: align must be a power of two >= 16");
+  uint64_t pos = 0;
+  for (size_t i = 0; i < n; ++i) {
+    pos = (pos + align - 1) & ~(align - 1);
+    out_offsets[i] = pos;
+    pos += tensor_bytes[i];
+  }
+  *out_blob_bytes = (pos + align - 1) & ~(align - 1);
+  return BCP_OK;
+}
+
+int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob, uint64_t blob_bytes, void* stream) {
+  if ((n && (!tensors || !metas)) || (blob_bytes && !blob)) return fail(BCP_ERR_INVALID, "bcp_pack: NULL argument");
+  std::lock_guard<std::mutex> lock(g_pack_mu);
+  bcp_plan_t* p = nullptr;
+  if (int rc = pack_plan(false, metas, n, blob_bytes, &p)) return rc;
+  void* dst[1] = {blob};
+  return execute(p, tensors, n, dst, 1, static_cast<cudaStream_t>(stream));
+}
+
+int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_meta* metas, size_t n, void* const* tensors, void* stream) {
+  if ((n && (!tensors || !metas)) || (blob_bytes && !blob)) return fail(BCP_ERR_INVALID, "bcp_unpack: NULL argument");
+  std::lock_guard<std::mutex> lock(g_pack_mu);
+  bcp_plan_t* p = nullptr;
+  if (int rc = pack_plan(true, metas, n, blob_bytes, &p)) return rc;
+  const void* src[1] = {blob};
+  return execute(p, src, 1, tensors, n, static_cast<cudaStream_t>(stream));
+}
+
+int bcp_pack_cache_clear(void) {
+  std::lock_guard<std::mutex> lock(g_pack_mu);
+  int rc = BCP_OK;
+  for (PackEntry& e : g_pack_cache)
+    if (int r = bcp_plan_destroy(e.plan)) rc = r;
+  g_pack_cache.clear();
+  return rc;
+}
+
+}  // extern "C"

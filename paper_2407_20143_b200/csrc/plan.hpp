@@ -1,0 +1,57 @@
+// Internal structures shared by the host planner, the C ABI and the kernel launcher.
+#pragma once
+
+#include <cstdarg>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "bcp.h"
+
+namespace bcp {
+
+// Thread-local error text behind bcp_last_error().
+std::string& last_error();
+int fail(int code, const char* fmt, ...);
+
+// A copy (or zero-fill) request before it is cut into work units: rows x row_bytes bytes.
+struct Item {
+  uint64_t src_off = 0, dst_off = 0;
+  uint64_t src_pitch = 0, dst_pitch = 0;
+  uint64_t row_bytes = 0;  // may exceed 4 GiB; cut into tiles later
+  uint64_t rows = 1;
+  uint32_t src_buf = 0, dst_buf = 0;
+  bool zero = false;  // no source: write zeros
+};
+
+struct Options {
+  uint32_t tile_bytes = 65536;
+  uint32_t small_bytes = 4096;
+  uint32_t block_threads = 512;
+  uint32_t ctas_per_sm = 2;
+  uint32_t order = 1;
+  uint32_t path_mask = 3;
+  uint32_t cache_hints = 1;
+};
+
+int parse_options(const bcp_plan_opts* in, Options* out);
+
+// Irregular-tensor decomposition (Sec. 3.2): boxes relative to the local tensor, flat order.
+struct RelBox {
+  int64_t off[BCP_MAX_NDIM];
+  int64_t len[BCP_MAX_NDIM];
+};
+void decompose(const int64_t* lengths, uint32_t ndim, int64_t a, int64_t b, std::vector<RelBox>* out);
+
+// Matching (Sec. 3.3 Step 2) + lowering: metas -> items.  Fills the entry / intersection
+// counters of `stats`.
+int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
+                    const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
+                    std::vector<Item>* items, bcp_plan_stats_t* stats);
+
+// Coalesce adjacent items, cut them into work units, classify and order them.
+// tiles = [CTA-wide units..., warp units...]; *n_big = number of CTA-wide units.
+void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_big,
+                 bcp_plan_stats_t* stats);
+
+}  // namespace bcp

@@ -1,0 +1,218 @@
+"""Host logic of the library on CPU: decomposition, matching, lowering, work-list properties,
+error codes, exported symbols.  The work list is executed by a numpy tile simulator written
+here (the kernels are not involved) and compared with the oracle."""
+import itertools
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2407_20143_b200 as bcp
+from paper_2407_20143_b200 import _lib, api
+from oracle import reshard_oracle as orc
+from workloads import fills
+from workloads.configs import CONFIGS, EXPECTED_TOTALS, scenario_cases
+from workloads.meta import BOX, FLAT_SLICE, ShardMeta
+from workloads.random_cases import big_random_case, random_case
+
+from helpers import np_bufs, read_irregular_example
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+# ---- C ABI surface -------------------------------------------------------------------------------
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "bcp.h")).read()
+    declared = set(re.findall(r"BCP_API\s+[\w\s\*]+?\b(bcp_\w+)\s*\(", text))
+    assert declared == set(_lib.EXPORTS) and len(declared) >= 14
+    lib = _lib.lib()
+    for name in declared:
+        assert getattr(lib, name) is not None
+    assert bcp.bcp_version() >= 100
+
+
+def test_struct_sizes_match_header():
+    import ctypes as C
+
+    assert C.sizeof(_lib.TileC) == 64
+    assert C.sizeof(_lib.ShardMetaC) == 8 + 16 + 3 * 64 + 16 + 8 + 16
+    assert C.sizeof(_lib.PlanOptsC) == 64
+
+
+# ---- decomposition (Sec. 3.2) ----------------------------------------------------------------------
+def test_decompose_paper_example():
+    shape, recs = read_irregular_example()
+    for _, a, b, boxes in recs:
+        assert bcp.bcp_decompose(shape, a, b) == boxes
+
+
+def _check_decomposition(shape, a, b):
+    boxes = bcp.bcp_decompose(shape, a, b)
+    n = len(shape)
+    assert len(boxes) <= max(1, 2 * n - 1)
+    idx = np.arange(int(np.prod(shape, dtype=np.int64))).reshape(shape)
+    pos = a
+    for off, ln in boxes:
+        sub = idx[tuple(slice(o, o + l) for o, l in zip(off, ln))].ravel()
+        # each box is a contiguous piece of the flattening and the boxes follow one another
+        assert sub.size > 0 and np.array_equal(sub, np.arange(pos, pos + sub.size))
+        pos += sub.size
+    assert pos == max(a, b) if b > a else boxes == []
+
+
+def test_decompose_brute_force_small_shapes():
+    shapes = [s for nd in (1, 2, 3) for s in itertools.product(range(1, 5), repeat=nd)] + [(2, 1, 3, 2), (1, 1, 5), (3, 2, 2, 2)]
+    for shape in shapes:
+        n = int(np.prod(shape))
+        for a in range(n + 1):
+            for b in range(a, n + 1):
+                _check_decomposition(shape, a, b)
+    assert bcp.bcp_decompose((), 0, 1) == [((), ())]
+    assert bcp.bcp_decompose((), 0, 0) == []
+
+
+def test_decompose_large_and_errors():
+    _check_decomposition((128, 97, 3), 1234, 30001)
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.bcp_decompose((3, 2), 2, 9)
+    assert e.value.code == api.ERR_INVALID
+
+
+# ---- tile simulator -----------------------------------------------------------------------------------
+def run_tiles(tiles, src, dst_sizes, poison=0xA5):
+    out = [np.full(n, poison, dtype=np.uint8) for n in dst_sizes]
+    count = [np.zeros(n, dtype=np.uint8) for n in dst_sizes]
+    for t in tiles:
+        g = 1 << (t.flags & api.TILE_GRAN_MASK)
+        assert t.dst_off % g == 0 and t.row_bytes % g == 0 and t.dst_pitch % g == 0
+        for r in range(t.rows):
+            d0 = t.dst_off + r * t.dst_pitch
+            if t.flags & api.TILE_ZERO:
+                out[t.dst_buf][d0:d0 + t.row_bytes] = 0
+            else:
+                assert t.src_off % g == 0 and t.src_pitch % g == 0
+                s0 = t.src_off + r * t.src_pitch
+                chunk = src[t.src_buf][s0:s0 + t.row_bytes]
+                assert chunk.size == t.row_bytes
+                out[t.dst_buf][d0:d0 + t.row_bytes] = chunk
+            count[t.dst_buf][d0:d0 + t.row_bytes] += 1
+    return out, count
+
+
+def check_case(case, fill="index", **opts):
+    blobs = np_bufs(fills.fill_state(case.src, case.key_ids, fill, case.seed, "cpu", poison=0x5A))
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    tiles = plan.tiles()
+    st = plan.stats()
+    got, count = run_tiles(tiles, blobs, case.dst.buf_bytes)
+    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    # every named target byte is written exactly once, every other byte never
+    named = [np.zeros(n, dtype=np.uint8) for n in case.dst.buf_bytes]
+    for m in case.dst.metas:
+        named[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length] += 1
+    for c, n in zip(count, named):
+        assert np.array_equal(c, n)
+    assert st["bytes_copied"] == case.dst.total_bytes
+    tb = opts.get("tile_bytes", 65536)
+    assert all(t.rows * t.row_bytes <= tb for t in tiles)
+    assert st["n_tiles"] + st["n_small_tiles"] == len(tiles)
+    small = [bool(t.flags & api.TILE_SMALL) for t in tiles]
+    assert small == sorted(small), "CTA-wide units come first"
+    plan.destroy()
+    return st
+
+
+@pytest.mark.parametrize("case", scenario_cases(), ids=lambda c: c.name)
+def test_scenarios_match_oracle(case):
+    check_case(case)
+
+
+@pytest.mark.parametrize("fill", ["uniform", "index"])
+def test_cfg1_matches_oracle(fill):
+    st = check_case(CONFIGS["cfg1"](fill), fill)
+    assert st["bytes_misaligned"] == 0 and st["bytes_src_unique"] == EXPECTED_TOTALS["cfg1"][0]
+    assert (st["n_src_entries"], st["n_dst_entries"], st["n_intersections"]) == (234, 211, 423)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_tiny_cases(seed):
+    check_case(random_case(seed, dst_replicas=1 + seed % 2), tile_bytes=4096, small_bytes=64 if seed % 3 else 4096)
+
+
+@pytest.mark.parametrize("itemsize,seed", [(1, 1), (2, 2), (4, 3), (8, 4), (2, 5)])
+def test_big_random_cases(itemsize, seed):
+    st = check_case(big_random_case(seed, itemsize=itemsize), tile_bytes=8192, order=1 + seed % 2)
+    assert st["bytes_misaligned"] > 0
+
+
+@pytest.mark.parametrize("opts", [dict(tile_bytes=4096), dict(order=2), dict(tile_bytes=1 << 20, small_bytes=65536)])
+def test_options_do_not_change_the_result(opts):
+    check_case(scenario_cases()[3], **opts)
+
+
+# ---- full-size configurations: planning is host-only, so their work lists are checked here ---------
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_config_plans(name):
+    case = CONFIGS[name]()
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    st = plan.stats()
+    src_total, dst_total = EXPECTED_TOTALS[name]
+    assert st["bytes_copied"] == dst_total and st["bytes_src_unique"] == src_total
+    assert st["bytes_misaligned"] == 0, "every unit of the benchmark configs moves whole 16-byte vectors"
+    tiles = plan.tiles()
+    written = sum(t.rows * t.row_bytes for t in tiles)
+    assert written == dst_total
+    # in-bounds on both sides and 16-byte aligned
+    sb, db = case.src.buf_bytes, case.dst.buf_bytes
+    for t in tiles[:: max(1, len(tiles) // 5000)]:
+        assert t.src_off + (t.rows - 1) * t.src_pitch + t.row_bytes <= sb[t.src_buf]
+        assert t.dst_off + (t.rows - 1) * t.dst_pitch + t.row_bytes <= db[t.dst_buf]
+        assert (t.src_off | t.dst_off | t.row_bytes | t.src_pitch | t.dst_pitch) % 16 == 0
+    plan.destroy()
+
+
+# ---- error behaviour (all detected on the host, before any launch) -----------------------------------
+def _m(fqn="w", isz=4, tag=2, shape=(4, 4), off=(0, 0), ln=(4, 4), buf=0, boff=0, **kw):
+    return ShardMeta(fqn, isz, tag, shape, off, ln, buf, boff, **kw)
+
+
+def _plan_err(src, sb, dst, db, **opts):
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.bcp_plan(src, sb, dst, db, **opts)
+    assert str(e.value)
+    return e.value.code
+
+
+def test_error_codes():
+    full = [_m()]
+    assert _plan_err([_m(isz=3)], [64], full, [64]) == api.ERR_INVALID
+    assert _plan_err([_m(off=(1, 0))], [64], full, [64]) == api.ERR_INVALID  # box leaves the global shape
+    assert _plan_err([_m(kind=FLAT_SLICE, flat_begin=3, flat_end=20)], [128], full, [64]) == api.ERR_INVALID
+    assert _plan_err(full, [64], [_m(tag=9)], [64]) == api.ERR_MISMATCH
+    assert _plan_err(full, [64], [_m(shape=(4, 5), ln=(4, 4))], [64]) == api.ERR_MISMATCH
+    assert _plan_err([_m(ln=(3, 4)), _m(off=(2, 0), ln=(2, 4), boff=48)], [80], full, [64]) == api.ERR_OVERLAP
+    assert _plan_err([_m(ln=(3, 4))], [64], full, [64]) == api.ERR_UNCOVERED
+    assert _plan_err([], [], full, [64]) == api.ERR_UNCOVERED
+    assert _plan_err(full, [63], full, [64]) == api.ERR_BOUNDS
+    assert _plan_err(full, [64], [_m(buf=1)], [64]) == api.ERR_BOUNDS
+    assert _plan_err(full, [64], [_m(), _m(boff=32)], [128]) == api.ERR_DST_ALIAS
+    assert _plan_err(full, [64], full, [64], tile_bytes=1000) == api.ERR_INVALID
+    assert _plan_err(full, [64], full, [64], block_threads=100) == api.ERR_INVALID
+    # partial loads are fine: the saved side may hold more than is wanted
+    p = bcp.bcp_plan(full, [64], [_m(off=(1, 1), ln=(2, 2))], [16])
+    assert p.stats()["bytes_copied"] == 16
+    # zero-volume and scalar entries
+    p = bcp.bcp_plan([_m("s", 8, 4, (), (), ()), _m("e", shape=(4, 0), ln=(4, 0))], [8],
+                     [_m("s", 8, 4, (), (), ()), _m("e", shape=(4, 0), off=(1, 0), ln=(2, 0), boff=8)], [8])
+    assert p.stats()["bytes_copied"] == 8
+
+
+def test_pack_layout_matches_closed_form():
+    sizes = [1, 255, 256, 257, 4096, 3, 0, 1000]
+    for align in (16, 256, 4096):
+        assert bcp.bcp_pack_layout(sizes, align) == orc.pack_layout(sizes, align)
+    with pytest.raises(bcp.BcpError):
+        bcp.bcp_pack_layout(sizes, 24)
