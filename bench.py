@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the load-time reshard hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+One "step" is one pass of the whole hot path over one synthetic training state: one
+bcp_reshard call that materialises every target rank's shards of the configuration from
+the source blobs resident in HBM (planning is done once, outside the timed region, as the
+paper treats it as a cached one-time cost).  Rank 0 prints ONE JSON line.
+
+  value      reshard GB/s = (unique source bytes read + target bytes written) * N / step time,
+             device-timed with CUDA events, max over ranks
+  e2e        the same metric through bcp_reshard_host: pinned host buffers in, pinned host
+             buffers out, host<->device copies inside the timed region
+  roofline   algorithmic bytes per launch / average kernel duration (CUDA events on the
+             launching stream) against the measured HBM copy bandwidth
+  cpu_baseline / --impl reference
+             the numpy oracle timed on this machine's host cores on a bounded sample of the
+             same workload
+
+With N > 1 (torchrun) every rank reshards its own replica of the state: the path has no
+exchange step on one node, so ranks are independent replicas (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "reshard GB/s (bytes read+written, device-timed)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="bcp", choices=["bcp", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--layers", type=int, default=0, help="shrink the depth (profiler captures); 0 = full size")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-verify", action="store_true")
+    ap.add_argument("--pack", action="store_true", help="also time bcp_pack of one target rank (reported as extra keys)")
+    ap.add_argument("--cpu-sample-gb", type=float, default=4.0,
+                    help="bytes read+written by one pass of the CPU oracle over its sample of the workload")
+    ap.add_argument("--cpu-passes", type=int, default=5)
+    for o in ("tile-bytes", "small-bytes", "block-threads", "ctas-per-sm", "order", "path-mask", "cache-hints"):
+        ap.add_argument("--" + o, type=int, default=0)
+    return ap.parse_args()
+
+
+def plan_opts(a) -> dict:
+    o = {}
+    for k in ("tile_bytes", "small_bytes", "block_threads", "ctas_per_sm", "order", "path_mask", "cache_hints"):
+        v = getattr(a, k)
+        if v:
+            o[k] = v
+    return o
+
+
+def make_case(a):
+    from workloads.configs import CONFIGS
+
+    if a.workload == "cfg1":
+        return CONFIGS["cfg1"]("uniform")
+    return CONFIGS[a.workload](a.layers) if a.layers else CONFIGS[a.workload]()
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+        self.t0 = self.t1 = None
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
+    def wait_first_sample(self, timeout=3.0):
+        t = time.time()
+        while not self.rows and time.time() - t < timeout:
+            time.sleep(0.02)
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.t.join(timeout=2)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        inside = [r for t, r in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t)]
+        rows = inside if inside else [r for _, r in self.rows]  # too short a region: samples since warm-up
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm), "window": "timed region" if inside else "warm-up + timed region"}
+
+
+# ----------------------------------------------------------------------------------- oracle sample
+def oracle_sample(case, target_bytes: float):
+    """FQNs (spread over the state) whose wanted bytes add up to about target_bytes."""
+    from oracle import reshard_oracle as orc
+
+    by_src, by_dst = orc.group_by_fqn(case.src.metas), orc.group_by_fqn(case.dst.metas)
+    names = sorted(by_dst)
+    picked, total = [], 0
+    stride = max(1, len(names) // 64)
+    order = [n for s in range(stride) for n in names[s::stride]]
+    for n in order:
+        b = sum(d.byte_length for d in by_dst[n])
+        if b == 0 or b > target_bytes / 2:
+            continue
+        picked.append(n)
+        total += b
+        if total >= target_bytes:
+            break
+    return picked, by_src, by_dst
+
+
+def time_oracle(case, fetch_payload, target_bytes: float, steps: int = 1, warmup: int = 0):
+    """Seconds per pass of the oracle over the sample, and the sample's byte counts.
+    fetch_payload(meta) -> numpy array of the saved entry's elements (host)."""
+    from oracle import reshard_oracle as orc
+
+    picked, by_src, by_dst = oracle_sample(case, target_bytes)
+    inputs = [(by_src[n], [fetch_payload(s) for s in by_src[n]], by_dst[n]) for n in picked]
+    src_b = sum(s.byte_length for ss, _, _ in inputs for s in ss)
+    dst_b = sum(d.byte_length for _, _, ds in inputs for d in ds)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        for ss, ps, ds in inputs:
+            orc.reshard_fqn(ss, ps, ds)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    return sum(times) / len(times), src_b, dst_b, len(picked)
+
+
+def run_reference(a):
+    """The oracle as it stands, on host cores, on a bounded sample per step (rank 0 only)."""
+    from paper_2407_20143_b200 import dist as D
+
+    rank, _, _ = D.world()
+    if rank != 0:
+        return
+    import numpy as np
+
+    from oracle import reshard_oracle as orc
+    from workloads import fills
+
+    case = make_case(a)
+    keys = case.key_ids
+
+    def fetch(m):
+        return fills.entry_bytes(m, keys[m.fqn], case.fill, case.seed, "cpu").numpy().view(orc._UINT[m.itemsize])
+
+    sec, src_b, dst_b, n = time_oracle(case, fetch, a.cpu_sample_gb * 1e9 / 2, steps=a.steps, warmup=a.warmup)
+    gbs = (src_b + dst_b) / sec / 1e9
+    sample = f"{n} FQNs of {case.name}, {src_b + dst_b} bytes read+written per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": a.gpus, "steps": a.steps,
+        "warmup": a.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic", "config": {"workload": case.name, "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ----------------------------------------------------------------------------------- main arm
+def main():
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+        return
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+    from paper_2407_20143_b200 import dist as D
+    from workloads import fills
+
+    rank, local_rank, ws = D.world()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    D.init("nccl")
+    case = make_case(a)
+    keys = case.key_ids
+    opts = plan_opts(a)
+    t0 = time.perf_counter()
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    plan_ms = (time.perf_counter() - t0) * 1e3
+    st = plan.stats()
+    b_min = st["bytes_src_unique"] + st["bytes_copied"]
+    b_moved = 2 * st["bytes_copied"]
+    free, _ = torch.cuda.mem_get_info()
+    need = sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)
+    assert free > need + (2 << 30), f"{case.name} needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free"
+    src = fills.fill_state(case.src, keys, case.fill, case.seed, dev)
+    dst = [torch.zeros(n, dtype=torch.uint8, device=dev) for n in case.dst.buf_bytes]
+    stream = torch.cuda.current_stream()
+
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(a.steps)]
+    with ClockSampler(local_rank) as clocks:
+        clocks.wait_first_sample()
+        for _ in range(max(a.warmup, 3)):
+            bcp.bcp_reshard(plan, src, dst, stream)
+        torch.cuda.synchronize()
+        D.barrier()
+        torch.cuda.synchronize()
+        t_begin = torch.cuda.Event(enable_timing=True)
+        t_end = torch.cuda.Event(enable_timing=True)
+        clocks.mark_begin()
+        t_begin.record(stream)
+        for e0, e1 in evs:
+            e0.record(stream)
+            bcp.bcp_reshard(plan, src, dst, stream)
+            e1.record(stream)
+        t_end.record(stream)
+        torch.cuda.synchronize()
+        clocks.mark_end()
+    D.barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    launch_ms = sorted(e0.elapsed_time(e1) for e0, e1 in evs)
+    ms_step = D.max_over_ranks(total_ms / a.steps, dev)
+    bcp.bcp_plan_device_status(plan)
+    value = b_min * ws / (ms_step * 1e-3) / 1e9
+
+    verified = None
+    if not a.no_verify:  # spot check: a sample of target entries against the generative fill
+        verified = True
+        for m in case.dst.metas[:: max(1, len(case.dst.metas) // 48)]:
+            hi = min(m.numel, 1 << 22)
+            want = fills.entry_bytes(m, keys[m.fqn], case.fill, case.seed, dev, 0, hi)
+            got = dst[m.buf_index][m.byte_offset:m.byte_offset + hi * m.itemsize]
+            verified = verified and bool(torch.equal(got, want))
+
+    peak, peak_kind = measured_peak()
+    avg_launch_ms = sum(launch_ms) / len(launch_ms)
+    achieved = b_min / (avg_launch_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": a.steps, "warmup": max(a.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": case.name, "src_bytes": st["bytes_src_unique"], "dst_bytes": st["bytes_copied"],
+                   "bytes_per_step": b_min, "bytes_counted": "unique source bytes read + target bytes written",
+                   "src_ranks": len(case.src.buf_bytes), "dst_ranks": len(case.dst.buf_bytes),
+                   "work_units": st["n_tiles"] + st["n_small_tiles"], "l2": "inputs_exceed_l2", "fill": case.fill,
+                   "multi_gpu": "replicas only", "plan_opts": opts, "plan_ms": plan_ms},
+        "gbps_b_moved": b_moved * ws / (ms_step * 1e-3) / 1e9,
+        "pct_of_8tbs_nominal": value / ws / 8000.0 * 100.0,
+        "launch_ms": {"median": launch_ms[len(launch_ms) // 2], "best": launch_ms[0], "mean": avg_launch_ms},
+        "gpu_launches": a.steps,
+        "verified": verified,
+        "clocks": clocks.summary(),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": f"of {peak_kind}", "traffic": None, "kernel": "bcp_copy_kernel",
+                     "algorithmic_bytes_per_launch": b_min},
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):  # DRAM bytes per payload byte, from a committed ncu capture
+        try:
+            with open(traffic_file) as f:
+                tr = json.load(f).get(a.workload)
+            if tr:
+                out["roofline"]["traffic"] = tr["dram_bytes_per_algorithmic_byte"] * b_min
+                out["roofline"]["traffic_note"] = tr.get("note")
+        except Exception:
+            pass
+
+    if a.pack and rank == 0:
+        out["pack"] = time_pack(case, dst, dev, stream, a.steps)
+
+    # free the device-timed buffers' plan before the host-path run allocates its own staging
+    if not a.no_e2e:
+        out["e2e"] = run_e2e(a, case, plan, src, dst, dev, ws, b_min)
+    else:
+        out["e2e"] = None
+
+    if rank == 0 and not a.no_cpu_baseline:
+        from oracle import reshard_oracle as orc
+
+        def fetch(m):
+            t = src[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length]
+            return t.cpu().numpy().view(orc._UINT[m.itemsize])
+
+        sec, sb, db, n = time_oracle(case, fetch, a.cpu_sample_gb * 1e9 / 2, steps=a.cpu_passes, warmup=1)
+        out["cpu_baseline"] = {"value": (sb + db) / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                               "sample": f"{n} FQNs of {case.name}, {sb + db} bytes read+written per pass, "
+                                         f"mean of {a.cpu_passes} passes, {sec:.2f} s each",
+                               "host_cores_available": os.cpu_count()}
+    plan.destroy()
+    if rank == 0:
+        print(json.dumps(out))
+    D.shutdown()
+
+
+def time_pack(case, dst, dev, stream, steps):
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+
+    r = 0
+    ms = [m for m in case.dst.metas if m.buf_index == r]
+    sizes = [m.byte_length for m in ms]
+    offs, total = bcp.bcp_pack_layout(sizes, 256)
+    blob = torch.empty(total, dtype=torch.uint8, device=dev)
+    ptrs = [dst[r].data_ptr() + m.byte_offset for m in ms]
+    metas = list(zip(offs, sizes))
+    for _ in range(3):
+        bcp.bcp_pack(ptrs, metas, blob, stream=stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        bcp.bcp_pack(ptrs, metas, blob, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_step = e0.elapsed_time(e1) / steps
+    nbytes = sum(sizes) + total
+    del blob
+    return {"tensors": len(ms), "blob_bytes": total, "ms_per_pack": ms_step, "gbps": nbytes / (ms_step * 1e-3) / 1e9}
+
+
+def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
+    """bcp_reshard_host with pinned host buffers; H2D and D2H inside the timed region."""
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+    from paper_2407_20143_b200 import dist as D
+
+    h2d, d2h = sum(case.src.buf_bytes), sum(case.dst.buf_bytes)
+    try:
+        import psutil
+
+        avail = psutil.virtual_memory().available
+    except Exception:
+        avail = None
+    free, _ = torch.cuda.mem_get_info()
+    reason = None
+    if avail is not None and avail < (h2d + d2h) * ws * 1.15 + (8 << 30):
+        reason = f"host memory: {avail / 1e9:.0f} GB available, {(h2d + d2h) * ws / 1e9:.0f} GB of pinned buffers needed"
+    if free < h2d + d2h + (2 << 30):
+        reason = f"device memory: {free / 1e9:.0f} GB free, {(h2d + d2h) / 1e9:.0f} GB of staging needed"
+    ok = D.max_over_ranks(1.0 if reason else 0.0, dev) == 0.0
+    if not ok:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "skipped": reason or "another rank could not allocate"}
+    hsrc = [torch.empty(n, dtype=torch.uint8, pin_memory=True) for n in case.src.buf_bytes]
+    for h, s in zip(hsrc, src):
+        h.copy_(s)
+    hdst = [torch.empty(n, dtype=torch.uint8, pin_memory=True) for n in case.dst.buf_bytes]
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    bcp.bcp_reshard_host(plan, hsrc, hdst, stream)  # warm-up: allocates the staging buffers
+    D.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(a.e2e_steps):
+        bcp.bcp_reshard_host(plan, hsrc, hdst, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    ms = D.max_over_ranks(e0.elapsed_time(e1) / a.e2e_steps, dev)
+    same = all(bool(torch.equal(h[: 1 << 20], d[: 1 << 20].cpu())) for h, d in zip(hdst, dst))
+    return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same}
+
+
+if __name__ == "__main__":
+    main()

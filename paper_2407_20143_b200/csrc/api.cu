@@ -68,6 +68,11 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
     if (!src[i] && p->src_bytes[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
   for (size_t i = 0; i < nd; ++i)
     if (!dst[i] && p->dst_bytes[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
+  // the access width of every work unit was derived from byte offsets, so bases must be 16-byte aligned
+  for (size_t i = 0; i < ns; ++i)
+    if (reinterpret_cast<uintptr_t>(src[i]) & 15) return fail(BCP_ERR_INVALID, "source buffer %zu is not 16-byte aligned", i);
+  for (size_t i = 0; i < nd; ++i)
+    if (reinterpret_cast<uintptr_t>(dst[i]) & 15) return fail(BCP_ERR_INVALID, "target buffer %zu is not 16-byte aligned", i);
   if (int rc = bind_device(p)) return rc;
   if (p->tiles.empty()) return BCP_OK;
   for (size_t i = 0; i < ns; ++i) p->h_ptrs[i] = const_cast<void*>(src[i]);
@@ -112,6 +117,7 @@ double ms_since(std::chrono::steady_clock::time_point t0) {
 struct PackEntry {
   bool unpack;
   uint64_t blob_bytes;
+  std::vector<uint8_t> residues;  // address mod 16 of every tensor, then of the blob
   std::vector<bcp_pack_meta> metas;
   bcp_plan_t* plan;
   uint64_t stamp;
@@ -121,9 +127,13 @@ std::vector<PackEntry> g_pack_cache;
 uint64_t g_pack_stamp = 0;
 const size_t kPackCacheMax = 16;
 
-int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_bytes, bcp_plan_t** out) {
+// Tensor and blob addresses need no alignment: each is rounded down to a 16-byte boundary
+// and the remainder (`residues`) becomes part of the planned byte offsets, so the access
+// width of every unit accounts for it.  A layout is cached per set of remainders.
+int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_bytes,
+              const std::vector<uint8_t>& residues, bcp_plan_t** out) {
   for (PackEntry& e : g_pack_cache) {
-    if (e.unpack == unpack && e.blob_bytes == blob_bytes && e.metas.size() == n &&
+    if (e.unpack == unpack && e.blob_bytes == blob_bytes && e.metas.size() == n && e.residues == residues &&
         (n == 0 || memcmp(e.metas.data(), metas, n * sizeof(bcp_pack_meta)) == 0)) {
       e.stamp = ++g_pack_stamp;
       *out = e.plan;
@@ -141,25 +151,28 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
   }
   const auto t0 = std::chrono::steady_clock::now();
   std::vector<Item> items;
-  std::vector<uint64_t> tensor_bytes(n), blob(1, blob_bytes);
+  const uint64_t blob_res = residues[n];
+  std::vector<uint64_t> tensor_bytes(n), blob(1, blob_bytes + blob_res);
   pos = 0;
   for (size_t i = 0; i < n; ++i) {
-    tensor_bytes[i] = metas[i].byte_length;
+    tensor_bytes[i] = metas[i].byte_length + residues[i];
     Item it;
     it.row_bytes = metas[i].byte_length;
     if (!unpack) {
       if (metas[i].byte_offset > pos) {  // padding before this tensor is written as zeros
         Item z;
         z.zero = true;
-        z.dst_off = pos;
+        z.dst_off = blob_res + pos;
         z.row_bytes = metas[i].byte_offset - pos;
         items.push_back(z);
       }
       it.src_buf = uint32_t(i);
-      it.dst_off = metas[i].byte_offset;
+      it.src_off = residues[i];
+      it.dst_off = blob_res + metas[i].byte_offset;
     } else {
       it.dst_buf = uint32_t(i);
-      it.src_off = metas[i].byte_offset;
+      it.dst_off = residues[i];
+      it.src_off = blob_res + metas[i].byte_offset;
     }
     items.push_back(it);
     pos = metas[i].byte_offset + metas[i].byte_length;
@@ -167,7 +180,7 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
   if (!unpack && pos < blob_bytes) {
     Item z;
     z.zero = true;
-    z.dst_off = pos;
+    z.dst_off = blob_res + pos;
     z.row_bytes = blob_bytes - pos;
     items.push_back(z);
   }
@@ -191,9 +204,24 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
     bcp_plan_destroy(g_pack_cache[victim].plan);
     g_pack_cache.erase(g_pack_cache.begin() + victim);
   }
-  g_pack_cache.push_back(PackEntry{unpack, blob_bytes, std::vector<bcp_pack_meta>(metas, metas + n), p, ++g_pack_stamp});
+  g_pack_cache.push_back(PackEntry{unpack, blob_bytes, residues, std::vector<bcp_pack_meta>(metas, metas + n), p, ++g_pack_stamp});
   *out = p;
   return BCP_OK;
+}
+
+// address -> (address rounded down to 16 bytes, remainder)
+void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vector<uint8_t>* res,
+                      std::vector<const void*>* bases) {
+  res->resize(n + 1);
+  bases->resize(n ? n : 1);
+  for (size_t i = 0; i < n; ++i) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(tensors[i]);
+    (*res)[i] = uint8_t(a & 15);
+    (*bases)[i] = reinterpret_cast<const void*>(a & ~uintptr_t(15));
+  }
+  const uintptr_t b = reinterpret_cast<uintptr_t>(blob);
+  (*res)[n] = uint8_t(b & 15);
+  return reinterpret_cast<void*>(b & ~uintptr_t(15));
 }
 
 }  // namespace
@@ -355,19 +383,25 @@ int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t align, uint
 int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob, uint64_t blob_bytes, void* stream) {
   if ((n && (!tensors || !metas)) || (blob_bytes && !blob)) return fail(BCP_ERR_INVALID, "bcp_pack: NULL argument");
   std::lock_guard<std::mutex> lock(g_pack_mu);
+  std::vector<uint8_t> res;
+  std::vector<const void*> bases;
+  void* blob_base = split_addresses(tensors, n, blob, &res, &bases);
   bcp_plan_t* p = nullptr;
-  if (int rc = pack_plan(false, metas, n, blob_bytes, &p)) return rc;
-  void* dst[1] = {blob};
-  return execute(p, tensors, n, dst, 1, static_cast<cudaStream_t>(stream));
+  if (int rc = pack_plan(false, metas, n, blob_bytes, res, &p)) return rc;
+  void* dst[1] = {blob_base};
+  return execute(p, bases.data(), n, dst, 1, static_cast<cudaStream_t>(stream));
 }
 
 int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_meta* metas, size_t n, void* const* tensors, void* stream) {
   if ((n && (!tensors || !metas)) || (blob_bytes && !blob)) return fail(BCP_ERR_INVALID, "bcp_unpack: NULL argument");
   std::lock_guard<std::mutex> lock(g_pack_mu);
+  std::vector<uint8_t> res;
+  std::vector<const void*> bases;
+  const void* blob_base = split_addresses(tensors, n, const_cast<void*>(blob), &res, &bases);
   bcp_plan_t* p = nullptr;
-  if (int rc = pack_plan(true, metas, n, blob_bytes, &p)) return rc;
-  const void* src[1] = {blob};
-  return execute(p, src, 1, tensors, n, static_cast<cudaStream_t>(stream));
+  if (int rc = pack_plan(true, metas, n, blob_bytes, res, &p)) return rc;
+  const void* src[1] = {blob_base};
+  return execute(p, src, 1, const_cast<void* const*>(bases.data()), n, static_cast<cudaStream_t>(stream));
 }
 
 int bcp_pack_cache_clear(void) {

@@ -1,0 +1,297 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI, on a real GPU.
+
+Small cases are compared byte by byte over whole buffers (with guard bands and a poison fill
+around and between the named bytes).  The five full-size configurations run in the launch
+configuration the benchmark times; every target byte is checked against the closed-form
+index-pattern fill (a property that needs no oracle) and a sample of FQNs is pushed through
+the oracle element by element.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2407_20143_b200 as bcp
+from oracle import reshard_oracle as orc
+from workloads import fills
+from workloads.configs import CONFIGS, scenario_cases
+from workloads.meta import ShardMeta
+from workloads.random_cases import big_random_case, random_case
+
+pytestmark = pytest.mark.gpu
+GUARD = 4096
+POISON = 0xA5
+
+
+def guarded(sizes, device, poison=POISON):
+    """Buffers with a poisoned guard band on both sides; returns (views, backing tensors)."""
+    backs = [torch.full((n + 2 * GUARD,), poison, dtype=torch.uint8, device=device) for n in sizes]
+    return [b[GUARD:GUARD + n] for b, n in zip(backs, sizes)], backs
+
+
+def guards_intact(backs, sizes, poison=POISON):
+    return all(bool((b[:GUARD] == poison).all()) and bool((b[GUARD + n:] == poison).all()) for b, n in zip(backs, sizes))
+
+
+def run_and_compare(case, device, fill="index", runs=1, stream=None, **opts):
+    src = fills.fill_state(case.src, case.key_ids, fill, case.seed, device, poison=0x5A)
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    for _ in range(runs):
+        dst, backs = guarded(case.dst.buf_bytes, device)
+        bcp.bcp_reshard(plan, src, dst, stream=stream)
+        (stream or torch.cuda.current_stream()).synchronize()
+        bcp.bcp_plan_device_status(plan)
+        for i, (d, w) in enumerate(zip(dst, want)):
+            got = d.cpu().numpy()
+            if not np.array_equal(got, w):
+                bad = np.flatnonzero(got != w)
+                pytest.fail(f"{case.name}: buffer {i} differs at {bad.size} bytes, first at {bad[0]} "
+                            f"(got {got[bad[0]]}, want {w[bad[0]]})")
+        assert guards_intact(backs, case.dst.buf_bytes), "write outside the target buffer"
+    st = plan.stats()
+    plan.destroy()
+    return st
+
+
+# ---- small cases, whole buffers ------------------------------------------------------------------
+@pytest.mark.parametrize("fill", ["uniform", "index"])
+def test_cfg1(cuda_device, fill):
+    st = run_and_compare(CONFIGS["cfg1"](fill), cuda_device, fill, runs=3)
+    assert st["bytes_copied"] == 37_498_880
+
+
+@pytest.mark.parametrize("case", scenario_cases(), ids=lambda c: c.name)
+def test_scenarios(cuda_device, case):
+    run_and_compare(case, cuda_device)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_tiny(cuda_device, seed):
+    run_and_compare(random_case(seed, dst_replicas=1 + seed % 2), cuda_device, tile_bytes=4096,
+                    small_bytes=64 if seed % 3 else 4096)
+
+
+@pytest.mark.parametrize("itemsize,seed", [(1, 1), (2, 2), (4, 3), (8, 4), (2, 5), (4, 6)])
+def test_big_random_misaligned(cuda_device, itemsize, seed):
+    """Odd shapes and byte offsets: every access width from 1 to 16 bytes, ragged heads and tails."""
+    st = run_and_compare(big_random_case(seed, itemsize=itemsize), cuda_device, tile_bytes=8192 if seed % 2 else 65536)
+    assert st["bytes_misaligned"] > 0
+
+
+@pytest.mark.parametrize("opts", [dict(block_threads=256, ctas_per_sm=4), dict(block_threads=1024, ctas_per_sm=1),
+                                  dict(tile_bytes=4096), dict(tile_bytes=1 << 20, small_bytes=1 << 16),
+                                  dict(cache_hints=2), dict(order=2), dict(path_mask=1)])
+def test_launch_options(cuda_device, opts):
+    run_and_compare(CONFIGS["cfg1"]("index"), cuda_device, **opts)
+    run_and_compare(big_random_case(11, itemsize=2), cuda_device, **opts)
+
+
+def test_side_stream_and_plan_reuse(cuda_device):
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        run_and_compare(scenario_cases()[3], cuda_device, runs=4, stream=s)
+
+
+def test_degenerate_entries(cuda_device):
+    src_m = [ShardMeta("s", 8, 4, (), (), (), 0, 16), ShardMeta("e", 4, 2, (4, 0), (0, 0), (4, 0), 0, 0),
+             ShardMeta("one", 1, 3, (1,), (0,), (1,), 0, 31)]
+    dst_m = [ShardMeta("s", 8, 4, (), (), (), 0, 0), ShardMeta("e", 4, 2, (4, 0), (1, 0), (2, 0), 0, 8),
+             ShardMeta("one", 1, 3, (1,), (0,), (1,), 1, 5)]
+    src = [torch.arange(32, dtype=torch.uint8, device=cuda_device)]
+    plan = bcp.bcp_plan(src_m, [32], dst_m, [16, 16])
+    dst, backs = guarded([16, 16], cuda_device)
+    bcp.bcp_reshard(plan, src, dst)
+    torch.cuda.synchronize()
+    want = orc.reshard(src_m, [src[0].cpu().numpy()], dst_m, [16, 16], fill_byte=POISON)
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, [16, 16])
+    # a plan with no work at all is legal and launches nothing
+    empty = bcp.bcp_plan([], [], [], [])
+    bcp.bcp_reshard(empty, [], [])
+
+
+def test_execution_errors(cuda_device):
+    case = scenario_cases()[0]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    src = fills.make_buffers(case.src, cuda_device)
+    dst = fills.make_buffers(case.dst, cuda_device)
+    with pytest.raises(bcp.BcpError):
+        bcp.bcp_reshard(plan, src[:-1], dst)
+    with pytest.raises(bcp.BcpError):
+        bcp.bcp_reshard(plan, src, [d.data_ptr() + 4 for d in dst])  # misaligned base
+    bcp.bcp_reshard(plan, src, dst)  # the plan is still usable
+    torch.cuda.synchronize()
+
+
+def test_reshard_host(cuda_device):
+    case = CONFIGS["cfg1"]("uniform")
+    src = [s.pin_memory() for s in fills.fill_state(case.src, case.key_ids, "uniform", 0, "cpu")]
+    dst = [torch.full((n,), POISON, dtype=torch.uint8).pin_memory() for n in case.dst.buf_bytes]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    for _ in range(2):
+        bcp.bcp_reshard_host(plan, src, dst)
+        want = orc.reshard(case.src.metas, [s.numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=0)
+        assert all(np.array_equal(d.numpy(), w) for d, w in zip(dst, want))
+
+
+# ---- pack / unpack ---------------------------------------------------------------------------------
+def _pack_check(device, sizes, align, offsets=None, misalign=0):
+    g = torch.Generator(device="cpu").manual_seed(len(sizes) * 7919 + align + misalign)
+    host = [torch.randint(1, 256, (n,), dtype=torch.uint8, generator=g) for n in sizes]
+    if misalign:  # tensors that start at odd addresses inside a larger allocation
+        backing = [torch.zeros(n + 64, dtype=torch.uint8, device=device) for n in sizes]
+        dev = [b[(misalign * (i + 1)) % 61:][:n] for i, (b, n) in enumerate(zip(backing, sizes))]
+        for d, h in zip(dev, host):
+            d.copy_(h)
+    else:
+        dev = [h.to(device) for h in host]
+    offs, total = bcp.bcp_pack_layout(sizes, align)
+    want, table = orc.pack([h.numpy() for h in host], align)
+    assert total == want.size and offs == [o for o, _ in table]
+    metas = list(zip(offs, sizes))
+    blob_back = torch.full((total + 2 * GUARD + 16,), POISON, dtype=torch.uint8, device=device)
+    blob = blob_back[GUARD + misalign % 16:][:total]
+    for _ in range(2):
+        bcp.bcp_pack(dev, metas, blob)
+        torch.cuda.synchronize()
+        assert np.array_equal(blob.cpu().numpy(), want)
+    assert bool((blob_back[:GUARD + misalign % 16] == POISON).all()) and bool((blob_back[GUARD + misalign % 16 + total:] == POISON).all())
+    out = [torch.full((n,), POISON, dtype=torch.uint8, device=device) for n in sizes]
+    bcp.bcp_unpack(blob, metas, out)
+    torch.cuda.synchronize()
+    for o, h, w in zip(out, host, orc.unpack(want, table)):
+        assert np.array_equal(o.cpu().numpy(), w) and np.array_equal(w, h.numpy())
+
+
+def test_pack_unpack_small(cuda_device):
+    _pack_check(cuda_device, [1, 255, 256, 257, 4096, 3, 0, 1000, 70_001, 16, 300_000], 256)
+    _pack_check(cuda_device, [5_000_000, 17, 1 << 20, 999_999], 4096)
+    _pack_check(cuda_device, [], 256)
+    _pack_check(cuda_device, [7, 9, 100_003, 65536], 16, misalign=3)
+    bcp.bcp_pack_cache_clear()
+
+
+def test_pack_rejects_bad_tables(cuda_device):
+    t = [torch.zeros(100, dtype=torch.uint8, device=cuda_device) for _ in range(2)]
+    blob = torch.zeros(512, dtype=torch.uint8, device=cuda_device)
+    with pytest.raises(bcp.BcpError):
+        bcp.bcp_pack(t, [(0, 100), (50, 100)], blob)  # overlap
+    with pytest.raises(bcp.BcpError):
+        bcp.bcp_pack(t, [(0, 100), (450, 100)], blob)  # past the end
+
+
+def test_reshard_then_pack_small_moe(cuda_device):
+    """EP8 -> EP4 on a small MoE, then every target rank's tensors packed into one blob."""
+    case = [c for c in scenario_cases() if c.name == "moe-ep8-to-ep4"][0]
+    src = fills.fill_state(case.src, case.key_ids, "uniform", case.seed, cuda_device)
+    dst = fills.make_buffers(case.dst, cuda_device, POISON)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    bcp.bcp_reshard(plan, src, dst)
+    want_dst = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, POISON)
+    for r in range(len(dst)):
+        ms = [m for m in case.dst.metas if m.buf_index == r]
+        sizes = [m.byte_length for m in ms]
+        offs, total = bcp.bcp_pack_layout(sizes, 256)
+        blob = torch.full((total,), POISON, dtype=torch.uint8, device=cuda_device)
+        bcp.bcp_pack([dst[r].data_ptr() + m.byte_offset for m in ms], list(zip(offs, sizes)), blob)
+        torch.cuda.synchronize()
+        want_blob, _ = orc.pack([want_dst[r][m.byte_offset:m.byte_offset + m.byte_length] for m in ms], 256)
+        assert np.array_equal(blob.cpu().numpy(), want_blob)
+
+
+# ---- the five configurations at full size -------------------------------------------------------------
+def _sample_fqns(case, k):
+    names = sorted({m.fqn for m in case.dst.metas})
+    # one name of every tensor kind first (the last two dotted components), then evenly spaced ones
+    kinds, picked = set(), []
+    for n in names:
+        kind = ".".join(n.split(".")[-2:])
+        if kind not in kinds:
+            kinds.add(kind)
+            picked.append(n)
+    step = max(1, len(names) // k)
+    picked += names[::step]
+    return list(dict.fromkeys(picked))
+
+
+def _free_gb():
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()  # memory cached by earlier tests counts as free
+    free, _ = torch.cuda.mem_get_info()
+    return free / 1e9
+
+
+@pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6)])
+def test_full_size_config(cuda_device, name, max_fqn_bytes):
+    case = CONFIGS[name]()
+    need = (sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)) / 1e9 + 8
+    assert _free_gb() > need, f"{name} needs {need:.0f} GB of device memory"
+    keys = case.key_ids
+    src = fills.fill_state(case.src, keys, "index", case.seed, cuda_device, poison=0x5A)
+    dst = fills.make_buffers(case.dst, cuda_device, POISON)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)  # bench defaults
+    bcp.bcp_reshard(plan, src, dst)
+    torch.cuda.synchronize()
+    bcp.bcp_plan_device_status(plan)
+    # (1) property at full size: every named target byte equals the closed-form fill of its
+    #     global index; every other byte kept the poison
+    named = 0
+    for m in case.dst.metas:
+        n = m.numel
+        for lo in range(0, n, 1 << 26):
+            hi = min(n, lo + (1 << 26))
+            want = fills.entry_bytes(m, keys[m.fqn], "index", case.seed, cuda_device, lo, hi)
+            b = m.byte_offset + lo * m.itemsize
+            got = dst[m.buf_index][b:b + (hi - lo) * m.itemsize]
+            if not torch.equal(got, want):
+                bad = int((got != want).nonzero()[0])
+                pytest.fail(f"{name} {m.fqn}: target rank {m.buf_index} differs at byte {b + bad}")
+        named += m.byte_length
+    assert named == case.dst.total_bytes
+    poison_left = sum(int((d == POISON).sum()) for d in dst)
+    assert poison_left >= sum(case.dst.buf_bytes) - named  # padding untouched (payload may contain 0xA5 too)
+    # (2) oracle, element by element, on a sample of FQNs
+    by_src, by_dst = orc.group_by_fqn(case.src.metas), orc.group_by_fqn(case.dst.metas)
+    checked = 0
+    for fqn in _sample_fqns(case, 10):
+        ss, ds = by_src[fqn], by_dst[fqn]
+        if sum(s.byte_length for s in ss) > max_fqn_bytes:
+            continue
+        payloads = [src[s.buf_index][s.byte_offset:s.byte_offset + s.byte_length].cpu().numpy().view(orc._UINT[s.itemsize]) for s in ss]
+        for d, w in zip(ds, orc.reshard_fqn(ss, payloads, ds)):
+            got = dst[d.buf_index][d.byte_offset:d.byte_offset + d.byte_length].cpu().numpy()
+            assert np.array_equal(got, w), f"{name} {fqn}: oracle mismatch on target rank {d.buf_index}"
+            checked += d.byte_length
+    assert checked > 0
+    plan.destroy()
+    if name == "cfg5":
+        _pack_full_rank(case, dst, cuda_device)
+
+
+def _pack_full_rank(case, dst, device):
+    """cfg5: pack one target rank's 1,766 tensors (15.7 GB) into a blob with an offset table."""
+    r = len(dst) - 1
+    ms = [m for m in case.dst.metas if m.buf_index == r]
+    sizes = [m.byte_length for m in ms]
+    offs, total = bcp.bcp_pack_layout(sizes, 256)
+    assert (offs, total) == orc.pack_layout(sizes, 256)
+    blob = torch.full((total,), POISON, dtype=torch.uint8, device=device)
+    ptrs = [dst[r].data_ptr() + m.byte_offset for m in ms]
+    bcp.bcp_pack(ptrs, list(zip(offs, sizes)), blob)
+    torch.cuda.synchronize()
+    end = 0
+    for m, o in zip(ms, offs):
+        assert not bool(blob[end:o].any()), "padding must be zero"
+        assert torch.equal(blob[o:o + m.byte_length], dst[r][m.byte_offset:m.byte_offset + m.byte_length])
+        end = o + m.byte_length
+    assert not bool(blob[end:].any())
+    # oracle on the first 64 tensors
+    k = 64
+    want, _ = orc.pack([dst[r][m.byte_offset:m.byte_offset + m.byte_length].cpu().numpy() for m in ms[:k]], 256)
+    assert np.array_equal(blob[:offs[k]].cpu().numpy()[:want.size], want)
+    out = torch.full((ms[0].byte_length + ms[1].byte_length,), POISON, dtype=torch.uint8, device=device)
+    bcp.bcp_unpack(blob, list(zip(offs[:2], sizes[:2])), [out.data_ptr(), out.data_ptr() + sizes[0]], blob_bytes=total)
+    torch.cuda.synchronize()
+    assert torch.equal(out[:sizes[0]], blob[offs[0]:offs[0] + sizes[0]]) and torch.equal(out[sizes[0]:], blob[offs[1]:offs[1] + sizes[1]])
+    bcp.bcp_pack_cache_clear()
