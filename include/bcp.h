@@ -60,7 +60,8 @@ typedef enum {
   BCP_ERR_DST_ALIAS = -6, /* two target entries write overlapping byte ranges of one buffer       */
   BCP_ERR_CUDA = -7,      /* a CUDA runtime call failed (message carries the CUDA error string)   */
   BCP_ERR_NOMEM = -8,     /* host allocation failed                                               */
-  BCP_ERR_DEVICE_TIMEOUT = -9, /* a bounded device-side wait gave up (TMA path only)              */
+  BCP_ERR_DEVICE_TIMEOUT = -9, /* a bounded device-side wait gave up (TMA path only); the targets of
+                                  that execution are incomplete                                     */
   BCP_ERR_CAPACITY = -10  /* an output array supplied by the caller is too small                  */
 } bcp_status;
 
@@ -104,9 +105,19 @@ typedef struct {
   uint32_t ctas_per_sm;    /* persistent CTAs per SM; default 2                                       */
   uint32_t order;          /* 0 default (= 1); 1 order work by source address (replica reads of one
                               source region run back to back and hit L2); 2 order by target address    */
-  uint32_t path_mask;      /* 0 default (= all); bit 0 register (LDG/STG) path, bit 1 TMA staging path */
-  uint32_t cache_hints;    /* 0 default (= 1); 1 streaming loads and stores; 2 plain accesses          */
-  uint32_t reserved[9];    /* must be 0 */
+  uint32_t path_mask;      /* 0 default: 3 when at least 128 MiB of payload qualifies for TMA staging, else 1
+                              (small jobs are launch-bound and one kernel is cheaper than two);
+                              1 every unit goes through registers (LDG/STG kernel);
+                              3 units that move whole 16-byte vectors between 16-byte aligned addresses
+                              (rows of at least 512 bytes) go through the TMA staging kernel (bulk
+                              copies via shared memory), the rest through the register kernel          */
+  uint32_t cache_hints;    /* 0 default (= 1); register path: 1 streaming loads and stores, 2 plain accesses;
+                              TMA path: 3 evict-first L2 hint on stores, 4 on loads too, else no hint    */
+  uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage; default 32768; multiple of 128 */
+  uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3                               */
+  uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2                               */
+  uint32_t unroll;          /* register path: 16-byte loads in flight per thread, 4 or 8; default 4    */
+  uint32_t reserved[5];    /* must be 0 */
 } bcp_plan_opts;
 
 typedef struct bcp_plan bcp_plan_t;
@@ -208,8 +219,9 @@ BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, si
 
 /*
  * Execute a plan (Sec. 3.3, Step 5: copy every matched segment into its target shard).
- * src_blobs[n_src_bufs] and dst_bufs[n_dst_bufs] are HOST arrays of DEVICE pointers, at
- * least as large as planned; counts must equal the planned ones.  The call uploads the
+ * src_blobs[n_src_bufs] and dst_bufs[n_dst_bufs] are HOST arrays of DEVICE pointers to
+ * buffers at least as large as planned, each 16-byte aligned (BCP_ERR_INVALID otherwise),
+ * sources and targets not overlapping; counts must equal the planned ones.  The call uploads the
  * work list on first use, enqueues the pointer tables and the copy kernel on `stream`
  * and returns without waiting; buffers must stay valid until the stream reaches that
  * point.  Executions of one plan must be ordered (same stream, or externally
@@ -229,9 +241,10 @@ BCP_API int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host
                      void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);
 
 /*
- * Device status word of the plan's last finished execution: 0, or BCP_ERR_DEVICE_TIMEOUT
- * if a bounded wait in the TMA path gave up (the rest of that unit was then copied
- * through registers, so the result is still complete).  Synchronises `stream`.
+ * Device status of the plan's executions so far: BCP_OK, or BCP_ERR_DEVICE_TIMEOUT if a
+ * bounded wait of the TMA staging kernel gave up (that CTA stopped taking work, so some
+ * target bytes of that execution were not written; the plan's counters are reset and it can
+ * be executed again).  Synchronises `stream`.
  */
 BCP_API int bcp_plan_device_status(bcp_plan_t* plan, void* stream);
 
@@ -253,7 +266,8 @@ BCP_API int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t ali
  * metas[i].byte_length bytes) is copied to blob + metas[i].byte_offset; every blob byte
  * in [0, blob_bytes) that belongs to no tensor is written as zero.  metas must be sorted
  * by byte_offset and non-overlapping, inside blob_bytes.  tensors and metas are host
- * arrays.  Asynchronous on `stream`.  Work lists are cached inside the library per
+ * arrays.  Tensor and blob addresses need no particular alignment (16-byte aligned ones
+ * copy fastest).  Asynchronous on `stream`.  Work lists are cached inside the library per
  * (metas, blob_bytes), so repeated packs of the same layout only upload pointers.
  */
 BCP_API int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,

@@ -37,7 +37,11 @@ class PlanOptsC(C.Structure):
         ("order", C.c_uint32),
         ("path_mask", C.c_uint32),
         ("cache_hints", C.c_uint32),
-        ("reserved", C.c_uint32 * 9),
+        ("tma_stage_bytes", C.c_uint32),
+        ("tma_stages", C.c_uint32),
+        ("tma_ctas_per_sm", C.c_uint32),
+        ("unroll", C.c_uint32),
+        ("reserved", C.c_uint32 * 5),
     ]
 
 

@@ -13,15 +13,15 @@ using namespace bcp;
 struct bcp_plan {
   Options opt;
   bcp_plan_stats_t stats;
-  std::vector<bcp_tile> tiles;  // CTA-wide units, then warp units
-  size_t n_big = 0;
+  std::vector<bcp_tile> tiles;  // TMA units, then other CTA-wide units, then warp units
+  size_t n_tma = 0, n_big = 0;
   std::vector<uint64_t> src_bytes, dst_bytes;
   // device side, created by the first execution
   int device = -1;
   bcp_tile* d_tiles = nullptr;
   void** d_ptrs = nullptr;  // source table followed by target table
-  Control* d_ctrl = nullptr;
-  uint32_t grid = 0;
+  Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel
+  uint32_t grid = 0, tma_grid = 0;
   cudaStream_t last_stream = nullptr;
   bool ran = false;
   std::vector<void*> h_ptrs;
@@ -50,9 +50,11 @@ int bind_device(bcp_plan_t* p) {
     BCP_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), p->tiles.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
   }
   BCP_CUDA(cudaMalloc(&p->d_ptrs, (n_ptrs ? n_ptrs : 1) * sizeof(void*)));
-  BCP_CUDA(cudaMalloc(&p->d_ctrl, sizeof(Control)));
-  BCP_CUDA(cudaMemset(p->d_ctrl, 0, sizeof(Control)));
+  BCP_CUDA(cudaMalloc(&p->d_ctrl, 2 * sizeof(Control)));
+  BCP_CUDA(cudaMemset(p->d_ctrl, 0, 2 * sizeof(Control)));
   BCP_CUDA(copy_kernel_max_grid(p->opt.block_threads, p->opt.ctas_per_sm, &p->grid));
+  if (p->n_tma)
+    BCP_CUDA(tma_kernel_max_grid(p->opt.tma_stage_bytes, p->opt.tma_stages, p->opt.tma_ctas_per_sm, &p->tma_grid));
   p->h_ptrs.resize(n_ptrs);
   p->device = dev;
   return BCP_OK;
@@ -79,10 +81,24 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
   for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
   // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
   BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  if (p->n_tma) {
+    TmaLaunchArgs t;
+    t.tiles = p->d_tiles;
+    t.n_tiles = uint32_t(p->n_tma);
+    t.src = reinterpret_cast<const void* const*>(p->d_ptrs);
+    t.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
+    t.ctrl = p->d_ctrl + 1;
+    t.stage_bytes = p->opt.tma_stage_bytes;
+    t.n_stages = p->opt.tma_stages;
+    t.grid = uint32_t(p->n_tma < p->tma_grid ? p->n_tma : p->tma_grid);
+    t.wait_limit = 1u << 22;
+    t.cache_hints = p->opt.cache_hints;
+    BCP_CUDA(launch_tma(t, stream));
+  }
   LaunchArgs a;
-  a.tiles = p->d_tiles;
+  a.tiles = p->d_tiles + p->n_tma;
   a.n_big = uint32_t(p->n_big);
-  a.n_small = uint32_t(p->tiles.size() - p->n_big);
+  a.n_small = uint32_t(p->tiles.size() - p->n_tma - p->n_big);
   a.src = reinterpret_cast<const void* const*>(p->d_ptrs);
   a.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
   a.ctrl = p->d_ctrl;
@@ -91,7 +107,8 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
   const uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;
   a.grid = uint32_t(units < p->grid ? units : p->grid);
   a.cache_hints = p->opt.cache_hints;
-  BCP_CUDA(launch_copy(a, stream));
+  a.unroll = p->opt.unroll;
+  if (units) BCP_CUDA(launch_copy(a, stream));
   p->last_stream = stream;
   p->ran = true;
   return BCP_OK;
@@ -103,7 +120,7 @@ bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_s
   if (!p) return nullptr;
   p->opt = opt;
   p->stats = stats;
-  build_tiles(items, opt, &p->tiles, &p->n_big, &p->stats);
+  build_tiles(items, opt, &p->tiles, &p->n_tma, &p->n_big, &p->stats);
   p->src_bytes = std::move(src_bytes);
   p->dst_bytes = std::move(dst_bytes);
   return p;
@@ -338,9 +355,14 @@ int bcp_plan_device_status(bcp_plan_t* plan, void* stream) {
   if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
   if (plan->device < 0) return BCP_OK;
   BCP_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-  Control c;
-  BCP_CUDA(cudaMemcpy(&c, plan->d_ctrl, sizeof c, cudaMemcpyDeviceToHost));
-  if (c.status) return fail(int(c.status) < 0 ? int(c.status) : BCP_ERR_DEVICE_TIMEOUT, "device reported status %d", int(c.status));
+  Control c[2];
+  BCP_CUDA(cudaMemcpy(c, plan->d_ctrl, sizeof c, cudaMemcpyDeviceToHost));
+  const uint32_t status = c[0].status ? c[0].status : c[1].status;
+  if (status) {
+    BCP_CUDA(cudaMemset(plan->d_ctrl, 0, sizeof c));  // counters of an aborted launch are stale: start clean
+    return fail(BCP_ERR_DEVICE_TIMEOUT, "a bounded wait of the TMA staging kernel gave up (device status %d); "
+                "the targets of that execution are incomplete", int(status));
+  }
   return BCP_OK;
 }
 

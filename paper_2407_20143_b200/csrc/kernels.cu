@@ -260,7 +260,11 @@ __global__ void __launch_bounds__(NT, 1024 / NT) bcp_copy_kernel(const bcp_tile*
 
 template <int NT, int HINT>
 cudaError_t launch_as(const LaunchArgs& a, cudaStream_t stream) {
-  bcp_copy_kernel<NT, 4, HINT><<<a.grid, NT, 0, stream>>>(a.tiles, a.n_big, a.n_small, a.src, a.dst, a.ctrl);
+  if (a.unroll == 8) {
+    bcp_copy_kernel<NT, 8, HINT><<<a.grid, NT, 0, stream>>>(a.tiles, a.n_big, a.n_small, a.src, a.dst, a.ctrl);
+  } else {
+    bcp_copy_kernel<NT, 4, HINT><<<a.grid, NT, 0, stream>>>(a.tiles, a.n_big, a.n_small, a.src, a.dst, a.ctrl);
+  }
   return cudaGetLastError();
 }
 

@@ -28,7 +28,27 @@ struct LaunchArgs {
   uint32_t block_threads;
   uint32_t grid;
   uint32_t cache_hints;       // 1 streaming, 2 plain
+  uint32_t unroll;            // 4 or 8
 };
+
+struct TmaLaunchArgs {
+  const bcp_tile* tiles;  // device: n_tiles units, all eligible for bulk copies
+  uint32_t n_tiles;
+  const void* const* src;
+  void* const* dst;
+  Control* ctrl;          // device, separate from the register kernel's
+  uint32_t stage_bytes;   // shared-memory stage, multiple of 128
+  uint32_t n_stages;      // 2..8
+  uint32_t grid;
+  uint32_t wait_limit;    // mbarrier polls before a CTA gives up
+  uint32_t cache_hints;   // 3: evict-first stores; 4: evict-first loads too; else none
+};
+
+// Persistent grid of the TMA staging kernel (one warp per CTA) for a stage geometry.
+cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_t ctas_per_sm, uint32_t* grid);
+
+// Enqueue the TMA staging kernel on `stream`.
+cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream);
 
 // Largest useful persistent grid for the copy kernel on the current device.
 cudaError_t copy_kernel_max_grid(uint32_t block_threads, uint32_t ctas_per_sm, uint32_t* grid);

@@ -30,8 +30,12 @@ struct Options {
   uint32_t block_threads = 512;
   uint32_t ctas_per_sm = 2;
   uint32_t order = 1;
-  uint32_t path_mask = 3;
+  uint32_t path_mask = 0;  // 0: decided from the work list
   uint32_t cache_hints = 1;
+  uint32_t tma_stage_bytes = 32768;
+  uint32_t tma_stages = 3;
+  uint32_t tma_ctas_per_sm = 2;
+  uint32_t unroll = 4;
 };
 
 int parse_options(const bcp_plan_opts* in, Options* out);
@@ -50,8 +54,8 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
                     std::vector<Item>* items, bcp_plan_stats_t* stats);
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
-// tiles = [CTA-wide units..., warp units...]; *n_big = number of CTA-wide units.
-void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_big,
-                 bcp_plan_stats_t* stats);
+// tiles = [TMA units..., other CTA-wide units..., warp units...].
+void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_tma,
+                 size_t* n_big, bcp_plan_stats_t* stats);
 
 }  // namespace bcp

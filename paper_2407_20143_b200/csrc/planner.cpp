@@ -44,6 +44,10 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->order) o.order = in->order;
     if (in->path_mask) o.path_mask = in->path_mask;
     if (in->cache_hints) o.cache_hints = in->cache_hints;
+    if (in->tma_stage_bytes) o.tma_stage_bytes = in->tma_stage_bytes;
+    if (in->tma_stages) o.tma_stages = in->tma_stages;
+    if (in->tma_ctas_per_sm) o.tma_ctas_per_sm = in->tma_ctas_per_sm;
+    if (in->unroll) o.unroll = in->unroll;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -52,8 +56,15 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     return fail(BCP_ERR_INVALID, "block_threads must be a multiple of 32 in [128, 1024]");
   if (o.ctas_per_sm < 1 || o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
   if (o.order < 1 || o.order > 2) return fail(BCP_ERR_INVALID, "order must be 1 or 2");
-  if (o.path_mask < 1 || o.path_mask > 3) return fail(BCP_ERR_INVALID, "path_mask must be 1, 2 or 3");
-  if (o.cache_hints < 1 || o.cache_hints > 2) return fail(BCP_ERR_INVALID, "cache_hints must be 1 or 2");
+  if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3) return fail(BCP_ERR_INVALID, "path_mask must be 0, 1 or 3");
+  if (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536)
+    return fail(BCP_ERR_INVALID, "tma_stage_bytes must be a multiple of 128 in [1024, 65536]");
+  if (o.tma_stages < 2 || o.tma_stages > 8) return fail(BCP_ERR_INVALID, "tma_stages must be in [2, 8]");
+  if (uint64_t(o.tma_stage_bytes) * o.tma_stages > 200 * 1024)
+    return fail(BCP_ERR_INVALID, "tma_stage_bytes * tma_stages must not exceed 200 KiB");
+  if (o.tma_ctas_per_sm < 1 || o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
+  if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
+  if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
   *out = o;
   return BCP_OK;
 }
@@ -452,7 +463,7 @@ inline uint32_t gran_log2(uint64_t bits) {
 
 struct Cutter {
   const Options& opt;
-  std::vector<bcp_tile> big, small;
+  std::vector<bcp_tile> tma, big, small;
   bcp_plan_stats_t* st;
 
   void emit(const Item& it, uint64_t src_off, uint64_t dst_off, uint64_t rows, uint64_t row_bytes) {
@@ -482,11 +493,13 @@ struct Cutter {
       small.push_back(t);
     } else {
       // TMA staging moves whole 16-byte units between 16-byte aligned addresses
-      if (g == 4 && !it.zero && (opt.path_mask & 2) && row_bytes >= 512) {
+      if (g == 4 && !it.zero && opt.path_mask != 1 && row_bytes >= 512) {
         t.flags |= BCP_TILE_TMA;
         ++st->n_tma_tiles;
+        tma.push_back(t);
+      } else {
+        big.push_back(t);
       }
-      big.push_back(t);
     }
   }
 
@@ -536,8 +549,8 @@ struct Cutter {
 
 }  // namespace
 
-void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_big,
-                 bcp_plan_stats_t* stats) {
+void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_tma,
+                 size_t* n_big, bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
@@ -562,8 +575,18 @@ void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_t
   stats->bytes_misaligned = 0;
   stats->n_strided_tiles = 0;
   stats->n_tma_tiles = 0;
-  Cutter c{opt, {}, {}, stats};
+  Cutter c{opt, {}, {}, {}, stats};
   for (const Item& it : merged) c.cut(it);
+  if (opt.path_mask == 0) {  // small jobs are launch-bound: keep them in one kernel
+    uint64_t eligible = 0;
+    for (const bcp_tile& t : c.tma) eligible += uint64_t(t.rows) * t.row_bytes;
+    if (eligible < (128u << 20)) {
+      for (bcp_tile& t : c.tma) t.flags &= ~BCP_TILE_TMA;
+      c.big.insert(c.big.end(), c.tma.begin(), c.tma.end());
+      c.tma.clear();
+      stats->n_tma_tiles = 0;
+    }
+  }
   auto by_src = [](const bcp_tile& a, const bcp_tile& b) {
     if (a.src_buf != b.src_buf) return a.src_buf < b.src_buf;
     if (a.src_off != b.src_off) return a.src_off < b.src_off;
@@ -572,18 +595,20 @@ void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_t
   auto by_dst = [](const bcp_tile& a, const bcp_tile& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
   };
-  if (opt.order == 1) {
-    std::sort(c.big.begin(), c.big.end(), by_src);
-    std::sort(c.small.begin(), c.small.end(), by_src);
-  } else {
-    std::sort(c.big.begin(), c.big.end(), by_dst);
-    std::sort(c.small.begin(), c.small.end(), by_dst);
+  for (std::vector<bcp_tile>* v : {&c.tma, &c.big, &c.small}) {
+    if (opt.order == 1) {
+      std::sort(v->begin(), v->end(), by_src);
+    } else {
+      std::sort(v->begin(), v->end(), by_dst);
+    }
   }
-  stats->n_tiles = c.big.size();
+  stats->n_tiles = c.tma.size() + c.big.size();
   stats->n_small_tiles = c.small.size();
+  *n_tma = c.tma.size();
   *n_big = c.big.size();
   tiles->clear();
-  tiles->reserve(c.big.size() + c.small.size());
+  tiles->reserve(c.tma.size() + c.big.size() + c.small.size());
+  tiles->insert(tiles->end(), c.tma.begin(), c.tma.end());
   tiles->insert(tiles->end(), c.big.begin(), c.big.end());
   tiles->insert(tiles->end(), c.small.begin(), c.small.end());
 }

@@ -1,0 +1,285 @@
+// TMA staging path: global -> shared -> global with bulk asynchronous copies.
+//
+// A CTA is one warp that only issues copy commands; the payload never enters registers.
+// Work units (tiles whose offsets, row length and pitches are multiples of 16 bytes) are
+// drawn from an atomic ticket counter and cut into chunks of at most one shared-memory
+// stage.  A chunk is a run (one bulk copy) or a group of rows of a strided rectangle (one
+// bulk copy per row, issued by different lanes, addresses computed here: no descriptors, so a
+// plan stays independent of buffer addresses).  Loads complete on a per-stage mbarrier;
+// stores are tracked with bulk groups.  With S stages, S-1 loads and up to 2 stores are in
+// flight per CTA.  Every wait on an mbarrier is bounded: if it gives up, the CTA records
+// BCP_ERR_DEVICE_TIMEOUT, stops taking work and leaves after its stores have drained.
+// No multicast, no clusters.
+#include "kernels.cuh"
+
+namespace bcp {
+namespace {
+
+constexpr int kMaxStages = 8;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// global -> shared::cta, completion counted in bytes on the mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+// shared::cta -> global, tracked by the issuing thread's bulk group
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+
+// the same two copies with an L2 eviction-priority hint
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                   dst_smem),
+               "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+               : "memory");
+}
+
+__device__ __forceinline__ void bulk_store_hint(void* dst, uint32_t src_smem, uint32_t bytes, uint64_t pol) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(dst), "r"(src_smem),
+               "r"(bytes), "l"(pol)
+               : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memory
+  const char* src;
+  char* dst;
+  uint64_t sp, dp;
+  uint32_t rows, row_bytes;
+};
+
+// Cuts the current tile into chunks.  All lanes hold the same state.
+struct TileCursor {
+  const char* s;
+  char* d;
+  uint64_t sp, dp;
+  uint32_t rows, row_bytes;
+  uint32_t r, c;  // next row, next byte inside the row
+  bool live;
+
+  __device__ __forceinline__ bool next(uint32_t stage_bytes, Chunk* out) {
+    if (!live) return false;
+    if (row_bytes > stage_bytes || rows == 1) {  // pieces of one row
+      const uint32_t n = min(stage_bytes, row_bytes - c);
+      out->src = s + uint64_t(r) * sp + c;
+      out->dst = d + uint64_t(r) * dp + c;
+      out->rows = 1;
+      out->row_bytes = n;
+      out->sp = out->dp = 0;
+      c += n;
+      if (c == row_bytes) {
+        c = 0;
+        ++r;
+      }
+    } else {  // whole rows
+      const uint32_t k = min(stage_bytes / row_bytes, rows - r);
+      out->src = s + uint64_t(r) * sp;
+      out->dst = d + uint64_t(r) * dp;
+      out->rows = k;
+      out->row_bytes = row_bytes;
+      out->sp = sp;
+      out->dp = dp;
+      r += k;
+    }
+    if (r == rows) live = false;
+    return true;
+  }
+};
+
+__global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles,
+                                                     const void* const* __restrict__ src, void* const* __restrict__ dst,
+                                                     Control* ctrl, uint32_t stage_bytes, uint32_t n_stages,
+                                                     uint32_t wait_limit, uint32_t hints) {
+  extern __shared__ __align__(128) unsigned char stage_mem[];
+  __shared__ __align__(8) uint64_t full[kMaxStages];
+  __shared__ Chunk held[kMaxStages];
+  const uint32_t lane = threadIdx.x;
+  const uint64_t pol = policy_evict_first();
+  const bool hint_st = hints >= 3, hint_ld = hints >= 4;  // 3: stores evict-first; 4: loads too
+  if (lane == 0) {
+    for (uint32_t i = 0; i < n_stages; ++i) mbar_init(smem_u32(&full[i]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  TileCursor cur;
+  cur.live = false;
+  uint32_t pending = 0;  // lane 0: the next ticket, drawn one tile ahead so that its latency is hidden
+  if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
+  bool drained = false;  // no more tickets
+  bool failed = false;
+
+  // returns false when the work list is exhausted
+  auto produce = [&](Chunk* ch) -> bool {
+    while (!cur.live) {
+      if (drained) return false;
+      const uint32_t ticket = __shfl_sync(0xffffffffu, pending, 0);
+      if (ticket >= n_tiles) {
+        drained = true;
+        return false;
+      }
+      const bcp_tile* t = tiles + ticket;
+      const uint4 a = __ldg(reinterpret_cast<const uint4*>(t));
+      const uint4 b = __ldg(reinterpret_cast<const uint4*>(t) + 1);
+      const uint4 c = __ldg(reinterpret_cast<const uint4*>(t) + 2);
+      cur.s = static_cast<const char*>(src[c.z]) + (uint64_t(a.x) | (uint64_t(a.y) << 32));
+      cur.d = static_cast<char*>(dst[c.w]) + (uint64_t(a.z) | (uint64_t(a.w) << 32));
+      cur.sp = uint64_t(b.x) | (uint64_t(b.y) << 32);
+      cur.dp = uint64_t(b.z) | (uint64_t(b.w) << 32);
+      cur.row_bytes = c.x;
+      cur.rows = c.y;
+      cur.r = cur.c = 0;
+      cur.live = cur.rows > 0 && cur.row_bytes > 0;
+      if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);  // consumed when this tile is used up
+    }
+    return cur.next(stage_bytes, ch);
+  };
+
+  auto issue_load = [&](uint32_t stage, const Chunk& ch) {
+    const uint32_t bar = smem_u32(&full[stage]);
+    const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
+    if (lane == 0) {
+      held[stage] = ch;
+      mbar_expect_tx(bar, ch.rows * ch.row_bytes);
+    }
+    __syncwarp();
+    for (uint32_t r = lane; r < ch.rows; r += 32) {
+      if (hint_ld) {
+        bulk_load_hint(base + r * ch.row_bytes, ch.src + uint64_t(r) * ch.sp, ch.row_bytes, bar, pol);
+      } else {
+        bulk_load(base + r * ch.row_bytes, ch.src + uint64_t(r) * ch.sp, ch.row_bytes, bar);
+      }
+    }
+  };
+
+  uint32_t issued = 0, stored = 0;  // chunks whose load / store has been issued
+  Chunk ch;
+  while (issued + 1 < n_stages && produce(&ch)) {  // prologue: S-1 loads in flight
+    issue_load(issued % n_stages, ch);
+    ++issued;
+  }
+  while (stored < issued) {
+    const uint32_t stage = stored % n_stages;
+    const uint32_t parity = (stored / n_stages) & 1;
+    const uint32_t bar = smem_u32(&full[stage]);
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+      if (++spins >= wait_limit) {
+        failed = true;
+        break;
+      }
+    }
+    if (failed) {
+      // give the loads still in flight a bounded chance to land before the CTA leaves
+      for (uint32_t k = stored + 1; k < issued; ++k) {
+        const uint32_t b2 = smem_u32(&full[k % n_stages]);
+        for (uint32_t w = 0; w < wait_limit && !mbar_try_wait(b2, (k / n_stages) & 1); ++w) {
+        }
+      }
+      break;
+    }
+    __syncwarp();
+    const Chunk h = held[stage];
+    const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
+    for (uint32_t r = lane; r < h.rows; r += 32) {
+      if (hint_st) {
+        bulk_store_hint(h.dst + uint64_t(r) * h.dp, base + r * h.row_bytes, h.row_bytes, pol);
+      } else {
+        bulk_store(h.dst + uint64_t(r) * h.dp, base + r * h.row_bytes, h.row_bytes);
+      }
+    }
+    bulk_commit();
+    ++stored;
+    // the stage of the previous store is free once that store has read its shared memory
+    bulk_wait_read<1>();
+    __syncwarp();
+    if (produce(&ch)) {
+      issue_load(issued % n_stages, ch);
+      ++issued;
+    }
+  }
+  bulk_wait_all();
+  __syncwarp();
+  if (lane == 0) {
+    if (failed) atomicExch(&ctrl->status, uint32_t(BCP_ERR_DEVICE_TIMEOUT));
+    // tickets: every CTA draws until it sees one past the end; a CTA that gave up early may
+    // hold an unprocessed ticket, which the status word reports
+    __threadfence();
+    const uint32_t left = atomicAdd(&ctrl->done, 1u);
+    if (left == gridDim.x - 1) {
+      ctrl->ticket = 0;
+      ctrl->done = 0;
+      __threadfence();
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_t ctas_per_sm, uint32_t* grid) {
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const size_t smem = size_t(stage_bytes) * n_stages;
+  e = cudaFuncSetAttribute(bcp_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+  if (e != cudaSuccess) return e;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bcp_tma_kernel, 32, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
+  const uint32_t k = ctas_per_sm < uint32_t(per_sm) ? ctas_per_sm : uint32_t(per_sm);
+  *grid = uint32_t(sms) * k;
+  return cudaSuccess;
+}
+
+cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream) {
+  if (a.n_tiles == 0) return cudaSuccess;
+  if (a.n_stages < 2 || a.n_stages > kMaxStages || a.stage_bytes % 128 || a.stage_bytes == 0) return cudaErrorInvalidValue;
+  const size_t smem = size_t(a.stage_bytes) * a.n_stages;
+  bcp_tma_kernel<<<a.grid, 32, smem, stream>>>(a.tiles, a.n_tiles, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages,
+                                               a.wait_limit, a.cache_hints);
+  return cudaGetLastError();
+}
+
+}  // namespace bcp

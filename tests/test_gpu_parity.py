@@ -80,10 +80,42 @@ def test_big_random_misaligned(cuda_device, itemsize, seed):
 
 @pytest.mark.parametrize("opts", [dict(block_threads=256, ctas_per_sm=4), dict(block_threads=1024, ctas_per_sm=1),
                                   dict(tile_bytes=4096), dict(tile_bytes=1 << 20, small_bytes=1 << 16),
-                                  dict(cache_hints=2), dict(order=2), dict(path_mask=1)])
+                                  dict(cache_hints=2), dict(order=2), dict(unroll=8),
+                                  dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=2, tile_bytes=32768),
+                                  dict(path_mask=3, tma_stage_bytes=32768, tma_stages=6, tma_ctas_per_sm=1)])
 def test_launch_options(cuda_device, opts):
     run_and_compare(CONFIGS["cfg1"]("index"), cuda_device, **opts)
     run_and_compare(big_random_case(11, itemsize=2), cuda_device, **opts)
+
+
+def _dim1_split_case(shape, isz, src_parts, dst_parts):
+    from workloads.layouts import ReshardCase
+    from workloads.meta import ShardedState
+
+    def side(parts):
+        metas, sizes = [], []
+        for r in range(parts):
+            b, e = shape[1] * r // parts, shape[1] * (r + 1) // parts
+            metas.append(ShardMeta("w", isz, isz, shape, (0, b), (shape[0], e - b), r, 256))
+            sizes.append(256 + shape[0] * (e - b) * isz + 256)
+        return ShardedState(metas, sizes)
+
+    return ReshardCase(f"dim1-{src_parts}-to-{dst_parts}", side(src_parts), side(dst_parts), "index", 1)
+
+
+@pytest.mark.parametrize("opts", [dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=3),
+                                  dict(path_mask=3, tma_stage_bytes=2048, tma_stages=8, tma_ctas_per_sm=6, tile_bytes=16384),
+                                  dict(path_mask=1, unroll=8)])
+def test_wide_strided_rows(cuda_device, opts):
+    """Strided rectangles with rows of 4-12 KiB (longer than a small TMA stage) and of 512 B."""
+    run_and_compare(_dim1_split_case((96, 6144), 4, 2, 3), cuda_device, runs=2, **opts)
+    run_and_compare(_dim1_split_case((1000, 1024), 2, 4, 1), cuda_device, **opts)
+    run_and_compare(_dim1_split_case((333, 4096), 2, 1, 8), cuda_device, **opts)
+
+
+@pytest.mark.parametrize("case", scenario_cases()[:4] + scenario_cases()[8:10], ids=lambda c: c.name)
+def test_scenarios_tma_path(cuda_device, case):
+    run_and_compare(case, cuda_device, path_mask=3, tile_bytes=16384, tma_stage_bytes=4096)
 
 
 def test_side_stream_and_plan_reuse(cuda_device):
@@ -249,8 +281,14 @@ def test_full_size_config(cuda_device, name, max_fqn_bytes):
                 pytest.fail(f"{name} {m.fqn}: target rank {m.buf_index} differs at byte {b + bad}")
         named += m.byte_length
     assert named == case.dst.total_bytes
-    poison_left = sum(int((d == POISON).sum()) for d in dst)
-    assert poison_left >= sum(case.dst.buf_bytes) - named  # padding untouched (payload may contain 0xA5 too)
+    # padding between entries kept the poison
+    for r, d in enumerate(dst):
+        end = 0
+        for m in sorted((m for m in case.dst.metas if m.buf_index == r), key=lambda m: m.byte_offset):
+            if m.byte_offset > end:
+                assert bool((d[end:m.byte_offset] == POISON).all()), f"{name}: padding of rank {r} overwritten"
+            end = max(end, m.byte_offset + m.byte_length)
+        assert bool((d[end:] == POISON).all())
     # (2) oracle, element by element, on a sample of FQNs
     by_src, by_dst = orc.group_by_fqn(case.src.metas), orc.group_by_fqn(case.dst.metas)
     checked = 0
