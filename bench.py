@@ -38,6 +38,9 @@ if ROOT not in sys.path:
 METRIC = "reshard GB/s (bytes read+written, device-timed)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes moved per algorithmic byte by the dominant kernel, from ncu captures summarised
+# under profiles/ (bcp_tma_kernel_*.md): (dram__bytes_read.sum + dram__bytes_write.sum) / B_min.
+NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.993}
 
 
 def parse_args():
@@ -289,6 +292,12 @@ def main():
             got = dst[m.buf_index][m.byte_offset:m.byte_offset + hi * m.itemsize]
             verified = verified and bool(torch.equal(got, want))
 
+    # kernels enqueued by one bcp_reshard: the TMA staging kernel (if any unit qualifies) and the
+    # register kernel (if any unit is left for it)
+    n_tma = st["n_tma_tiles"]
+    n_reg = st["n_tiles"] - n_tma + st["n_small_tiles"]
+    kernels_per_step = int(n_tma > 0) + int(n_reg > 0)
+    dominant = "bcp_tma_kernel" if n_tma > 0 else "bcp_copy_kernel"
     peak, peak_kind = measured_peak()
     avg_launch_ms = sum(launch_ms) / len(launch_ms)
     achieved = b_min / (avg_launch_ms * 1e-3) / 1e9
@@ -304,23 +313,21 @@ def main():
         "gbps_b_moved": b_moved * ws / (ms_step * 1e-3) / 1e9,
         "pct_of_8tbs_nominal": value / ws / 8000.0 * 100.0,
         "launch_ms": {"median": launch_ms[len(launch_ms) // 2], "best": launch_ms[0], "mean": avg_launch_ms},
-        "gpu_launches": a.steps,
+        "gpu_launches": a.steps * kernels_per_step,
+        "kernels_per_step": kernels_per_step,
         "verified": verified,
         "clocks": clocks.summary(),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": f"of {peak_kind}", "traffic": None, "kernel": "bcp_copy_kernel",
-                     "algorithmic_bytes_per_launch": b_min},
+                     "peak_source": f"of {peak_kind}", "traffic": None, "kernel": dominant,
+                     "algorithmic_bytes_per_launch": b_min,
+                     "duration_note": "CUDA events around one bcp_reshard (all its kernels; the dominant kernel's "
+                                      "share of device time is in profiles/)"},
     }
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):  # DRAM bytes per payload byte, from a committed ncu capture
-        try:
-            with open(traffic_file) as f:
-                tr = json.load(f).get(a.workload)
-            if tr:
-                out["roofline"]["traffic"] = tr["dram_bytes_per_algorithmic_byte"] * b_min
-                out["roofline"]["traffic_note"] = tr.get("note")
-        except Exception:
-            pass
+    ratio = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get((a.workload, dominant))
+    if ratio is not None:
+        out["roofline"]["traffic"] = ratio * b_min
+        out["roofline"]["traffic_note"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch (see profiles/), " \
+                                          "scaled by algorithmic bytes where the capture ran a shallower model"
 
     if a.pack and rank == 0:
         out["pack"] = time_pack(case, dst, dev, stream, a.steps)
