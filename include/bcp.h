@@ -281,6 +281,38 @@ BCP_API int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_met
 /* Drops the cached pack / unpack work lists (waits for their last executions). */
 BCP_API int bcp_pack_cache_clear(void);
 
+/*
+ * bcp_pack for callers that cannot allocate.  (The paper has no counterpart: this entry point
+ * exists for the way the library gets embedded, not for the method.)
+ *
+ * Who needs it: a process whose device memory is already fully handed out to its own pool
+ * (a serving engine, a training job sized to the last megabyte), or code that runs where an
+ * allocation is not allowed or would synchronise the whole device.  bcp_pack allocates
+ * its device-side work list the first time a layout is seen; this call never calls
+ * cudaMalloc, cudaFree or any other allocating routine, on the device or on the host.
+ * Instead its scratch (control words, pointer table, work list) is a fixed array of about
+ * 0.8 MiB in device memory that belongs to the library image: every GPU that loads the library
+ * holds it until the process exits, whether or not this call is ever made.
+ *
+ * Same arguments, result and asynchrony as bcp_pack.  Differences:
+ *   - limits: at most BCP_STATIC_MAX_TENSORS tensors and BCP_STATIC_MAX_UNITS work units
+ *     (the unit size grows up to 64 MiB to make a blob fit); beyond that the call returns
+ *     BCP_ERR_CAPACITY and launches nothing: use bcp_pack.
+ *   - the first call on each device looks up the device address of the fixed array, with
+ *     that device current; make that first call before any stream capture begins.
+ *   - all calls share the one array per device.  Each call rewrites what it uses and clears the
+ *     control words, so calls that run one after the other on the GPU (same stream, or
+ *     otherwise ordered) are safe; two calls whose kernels may overlap on the GPU (different
+ *     streams without ordering) race on it and must not be made.  Host-side the call is
+ *     serialised by a lock.
+ *   - the work list is rebuilt on every call (nothing is cached) and runs on the register
+ *     kernel.
+ */
+#define BCP_STATIC_MAX_TENSORS 4096u
+#define BCP_STATIC_MAX_UNITS 12288u
+BCP_API int bcp_pack_static(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,
+                            uint64_t blob_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

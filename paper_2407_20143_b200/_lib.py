@@ -91,6 +91,7 @@ _PROTOS = {
     "bcp_pack": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
     "bcp_unpack": (C.c_int, [_VP, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
     "bcp_pack_cache_clear": (C.c_int, []),
+    "bcp_pack_static": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
 }
 
 EXPORTS = tuple(_PROTOS)

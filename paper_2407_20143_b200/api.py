@@ -173,6 +173,17 @@ def bcp_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_byt
     _check(L.lib().bcp_pack(_ptrs(tensors), _pack_metas(metas), len(tensors), bp, nb, _stream(stream)))
 
 
+def bcp_pack_static(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_bytes: Optional[int] = None,
+                    stream=None) -> None:
+    """bcp_pack without any allocation: the work list lives in a fixed device array inside the
+    library (at most 4096 tensors per call).  For hosts that own all device memory themselves or
+    call from a place where allocating is not allowed.  Calls must not overlap on the GPU; make
+    the first call on a device before any stream capture."""
+    nb = blob_bytes if blob_bytes is not None else blob.numel() * blob.element_size()
+    bp = blob if isinstance(blob, int) else blob.data_ptr()
+    _check(L.lib().bcp_pack_static(_ptrs(tensors), _pack_metas(metas), len(tensors), bp, nb, _stream(stream)))
+
+
 def bcp_unpack(blob, metas: Sequence[Tuple[int, int]], tensors: Sequence, blob_bytes: Optional[int] = None,
                stream=None) -> None:
     nb = blob_bytes if blob_bytes is not None else blob.numel() * blob.element_size()
