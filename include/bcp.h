@@ -108,14 +108,16 @@ typedef struct {
   uint32_t path_mask;      /* 0 default: 3 when at least 128 MiB of payload qualifies for TMA staging, else 1
                               (small jobs are launch-bound and one kernel is cheaper than two);
                               1 every unit goes through registers (LDG/STG kernel);
-                              3 units that move whole 16-byte vectors between 16-byte aligned addresses
-                              (rows of at least 512 bytes) go through the TMA staging kernel (bulk
-                              copies via shared memory), the rest through the register kernel          */
+                              3 runs of at least 512 bytes (any alignment) and rectangles with rows of at
+                              least 512 bytes whose offsets, row length and pitches are multiples of 16
+                              go through the TMA staging kernel (bulk copies via shared memory), the
+                              rest through the register kernel                                          */
   uint32_t cache_hints;    /* 0 default (= 1); register path: 1 streaming loads and stores, 2 plain accesses;
                               TMA path: 3 evict-first L2 hint on stores, 4 on loads too, else no hint    */
-  uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage; default 32768; multiple of 128 */
+  uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage, multiple of 128; default 32768, or
+                               16384 when an eighth or more of the staged payload are shifted runs      */
   uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3                               */
-  uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2                               */
+  uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2 (4 with many shifted runs)     */
   uint32_t unroll;          /* register path: 16-byte loads in flight per thread, 4 or 8; default 4    */
   uint32_t reserved[5];    /* must be 0 */
 } bcp_plan_opts;

@@ -120,9 +120,9 @@ bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_s
   if (!p) return nullptr;
   p->opt = opt;
   p->stats = stats;
-  build_tiles(items, opt, &p->tiles, &p->n_tma, &p->n_big, &p->stats);
   p->src_bytes = std::move(src_bytes);
   p->dst_bytes = std::move(dst_bytes);
+  build_tiles(items, p->opt, &p->src_bytes, &p->tiles, &p->n_tma, &p->n_big, &p->stats);
   return p;
 }
 

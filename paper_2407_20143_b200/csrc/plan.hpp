@@ -32,9 +32,9 @@ struct Options {
   uint32_t order = 1;
   uint32_t path_mask = 0;  // 0: decided from the work list
   uint32_t cache_hints = 1;
-  uint32_t tma_stage_bytes = 32768;
+  uint32_t tma_stage_bytes = 0;  // 0: chosen from the work list (see build_tiles)
   uint32_t tma_stages = 3;
-  uint32_t tma_ctas_per_sm = 2;
+  uint32_t tma_ctas_per_sm = 0;
   uint32_t unroll = 4;
 };
 
@@ -55,7 +55,8 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
 // tiles = [TMA units..., other CTA-wide units..., warp units...].
-void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_tma,
-                 size_t* n_big, bcp_plan_stats_t* stats);
+// src_bytes: sizes of the source buffers (bounds for over-reading aligned supersets).
+void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
+                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, bcp_plan_stats_t* stats);
 
 }  // namespace bcp

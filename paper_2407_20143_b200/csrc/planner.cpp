@@ -57,12 +57,12 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.ctas_per_sm < 1 || o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
   if (o.order < 1 || o.order > 2) return fail(BCP_ERR_INVALID, "order must be 1 or 2");
   if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3) return fail(BCP_ERR_INVALID, "path_mask must be 0, 1 or 3");
-  if (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536)
+  if (o.tma_stage_bytes && (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536))
     return fail(BCP_ERR_INVALID, "tma_stage_bytes must be a multiple of 128 in [1024, 65536]");
   if (o.tma_stages < 2 || o.tma_stages > 8) return fail(BCP_ERR_INVALID, "tma_stages must be in [2, 8]");
-  if (uint64_t(o.tma_stage_bytes) * o.tma_stages > 200 * 1024)
+  if (uint64_t(o.tma_stage_bytes ? o.tma_stage_bytes : 32768) * o.tma_stages > 200 * 1024)
     return fail(BCP_ERR_INVALID, "tma_stage_bytes * tma_stages must not exceed 200 KiB");
-  if (o.tma_ctas_per_sm < 1 || o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
+  if (o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
   *out = o;
@@ -463,6 +463,7 @@ inline uint32_t gran_log2(uint64_t bits) {
 
 struct Cutter {
   const Options& opt;
+  const std::vector<uint64_t>* src_bytes;  // source buffer sizes (may be null: unknown)
   std::vector<bcp_tile> tma, big, small;
   bcp_plan_stats_t* st;
 
@@ -492,8 +493,14 @@ struct Cutter {
       t.flags |= BCP_TILE_SMALL;
       small.push_back(t);
     } else {
-      // TMA staging moves whole 16-byte units between 16-byte aligned addresses
-      if (g == 4 && !it.zero && opt.path_mask != 1 && row_bytes >= 512) {
+      // TMA staging: whole 16-byte units between 16-byte aligned addresses (runs and rectangles),
+      // or a run of any alignment whose 16-byte aligned superset stays inside the source buffer
+      bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= 512;
+      if (eligible && g < 4) {
+        const uint64_t end16 = (src_off + row_bytes + 15) & ~uint64_t(15);
+        eligible = rows == 1 && src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
+      }
+      if (eligible) {
         t.flags |= BCP_TILE_TMA;
         ++st->n_tma_tiles;
         tma.push_back(t);
@@ -549,8 +556,8 @@ struct Cutter {
 
 }  // namespace
 
-void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_tile>* tiles, size_t* n_tma,
-                 size_t* n_big, bcp_plan_stats_t* stats) {
+void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
+                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
@@ -575,7 +582,7 @@ void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_t
   stats->bytes_misaligned = 0;
   stats->n_strided_tiles = 0;
   stats->n_tma_tiles = 0;
-  Cutter c{opt, {}, {}, {}, stats};
+  Cutter c{opt, src_bytes, {}, {}, {}, stats};
   for (const Item& it : merged) c.cut(it);
   if (opt.path_mask == 0) {  // small jobs are launch-bound: keep them in one kernel
     uint64_t eligible = 0;
@@ -595,6 +602,21 @@ void build_tiles(std::vector<Item>& items, const Options& opt, std::vector<bcp_t
   auto by_dst = [](const bcp_tile& a, const bcp_tile& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
   };
+  // Stage geometry of the TMA kernel when the caller left it open.  Aligned units only issue
+  // copy commands, so few CTAs with large stages are enough (2 x 3 x 32 KiB per SM); shifted
+  // runs are copied out of shared memory by the warp itself and want more warps per SM
+  // (4 x 3 x 16 KiB).  Both fill 192 KiB of shared memory per SM.
+  {
+    uint64_t total = 0, shifted = 0;
+    for (const bcp_tile& t : c.tma) {
+      const uint64_t n = uint64_t(t.rows) * t.row_bytes;
+      total += n;
+      if ((t.flags & BCP_TILE_GRAN_MASK) < 4) shifted += n;
+    }
+    const bool many_shifted = shifted * 8 >= total && total > 0;
+    if (!opt.tma_stage_bytes) opt.tma_stage_bytes = many_shifted ? 16384 : 32768;
+    if (!opt.tma_ctas_per_sm) opt.tma_ctas_per_sm = many_shifted ? 4 : 2;
+  }
   for (std::vector<bcp_tile>* v : {&c.tma, &c.big, &c.small}) {
     if (opt.order == 1) {
       std::sort(v->begin(), v->end(), by_src);

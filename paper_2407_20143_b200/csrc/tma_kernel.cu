@@ -10,6 +10,12 @@
 // flight per CTA.  Every wait on an mbarrier is bounded: if it gives up, the CTA records
 // BCP_ERR_DEVICE_TIMEOUT, stops taking work and leaves after its stores have drained.
 // No multicast, no clusters.
+//
+// Runs whose source and target addresses are not both 16-byte aligned, or differ mod 16 (odd
+// element cuts of ZeRO / FSDP flat shards, odd shapes), are staged too: the bulk load fetches
+// the 16-byte aligned superset of the source piece, and the warp itself copies the payload out
+// of shared memory with coalesced stores of the run's natural width (1, 2, 4 or 8 bytes), so
+// global reads stay full-width and writes stay contiguous whatever the relative shift.
 #include "kernels.cuh"
 
 namespace bcp {
@@ -85,6 +91,8 @@ struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memor
   char* dst;
   uint64_t sp, dp;
   uint32_t rows, row_bytes;
+  uint32_t shift;  // shifted run only: payload starts `shift` bytes into the stage
+  uint32_t width;  // 0: aligned chunk, stored with bulk copies; else log2 of the store width + 1
 };
 
 // Cuts the current tile into chunks.  All lanes hold the same state.
@@ -94,10 +102,26 @@ struct TileCursor {
   uint64_t sp, dp;
   uint32_t rows, row_bytes;
   uint32_t r, c;  // next row, next byte inside the row
+  uint32_t width;  // 0 aligned tile; else log2(access width) + 1 of a shifted run
   bool live;
 
   __device__ __forceinline__ bool next(uint32_t stage_bytes, Chunk* out) {
     if (!live) return false;
+    out->shift = 0;
+    out->width = 0;
+    if (width) {  // shifted run (rows == 1): pieces that leave room for the aligned superset
+      const uint32_t n = min(stage_bytes - 32, row_bytes - c);
+      out->src = s + c;
+      out->dst = d + c;
+      out->rows = 1;
+      out->row_bytes = n;
+      out->sp = out->dp = 0;
+      out->shift = uint32_t(reinterpret_cast<uintptr_t>(out->src) & 15);
+      out->width = width;
+      c += n;
+      if (c == row_bytes) live = false;
+      return true;
+    }
     if (row_bytes > stage_bytes || rows == 1) {  // pieces of one row
       const uint32_t n = min(stage_bytes, row_bytes - c);
       out->src = s + uint64_t(r) * sp + c;
@@ -124,6 +148,23 @@ struct TileCursor {
     return true;
   }
 };
+
+// Copy n bytes from shared memory (generic loads) to global memory, one warp, elements of V.
+template <typename V>
+__device__ __forceinline__ void warp_store_out(const unsigned char* smem, char* dst, uint32_t n, uint32_t lane) {
+  const V* sv = reinterpret_cast<const V*>(smem);
+  V* dv = reinterpret_cast<V*>(dst);
+  const uint32_t ne = n / sizeof(V);
+  uint32_t i = lane;
+  for (; i + 7 * 32 < ne; i += 8 * 32) {
+    V v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = sv[i + k * 32];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) __stcs(dv + i + k * 32, v[k]);
+  }
+  for (; i < ne; i += 32) __stcs(dv + i, sv[i]);
+}
 
 __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles,
                                                      const void* const* __restrict__ src, void* const* __restrict__ dst,
@@ -170,6 +211,10 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
       cur.rows = c.y;
       cur.r = cur.c = 0;
       cur.live = cur.rows > 0 && cur.row_bytes > 0;
+      // a run that is not 16-byte aligned on both sides and in length is staged as a shifted run
+      const uint32_t bits = a.x | a.z | c.x;  // low bits of src_off | dst_off | row_bytes (bases are 16-byte aligned)
+      cur.width = 0;
+      if (cur.rows == 1 && (bits & 15)) cur.width = (bits & 1) ? 1 : (bits & 2) ? 2 : (bits & 4) ? 3 : 4;
       if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);  // consumed when this tile is used up
     }
     return cur.next(stage_bytes, ch);
@@ -178,6 +223,16 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
   auto issue_load = [&](uint32_t stage, const Chunk& ch) {
     const uint32_t bar = smem_u32(&full[stage]);
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
+    if (ch.width) {  // aligned superset of a shifted run, one bulk copy
+      const uint32_t bytes = (ch.shift + ch.row_bytes + 15u) & ~15u;
+      if (lane == 0) {
+        held[stage] = ch;
+        mbar_expect_tx(bar, bytes);
+        bulk_load(base, ch.src - ch.shift, bytes, bar);
+      }
+      __syncwarp();
+      return;
+    }
     if (lane == 0) {
       held[stage] = ch;
       mbar_expect_tx(bar, ch.rows * ch.row_bytes);
@@ -221,7 +276,17 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     __syncwarp();
     const Chunk h = held[stage];
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
-    for (uint32_t r = lane; r < h.rows; r += 32) {
+    if (h.width) {  // shifted run: the warp copies the payload out of the stage
+      const unsigned char* p = stage_mem + stage * stage_bytes + h.shift;
+      switch (h.width) {
+        case 4: warp_store_out<uint2>(p, h.dst, h.row_bytes, lane); break;
+        case 3: warp_store_out<unsigned int>(p, h.dst, h.row_bytes, lane); break;
+        case 2: warp_store_out<unsigned short>(p, h.dst, h.row_bytes, lane); break;
+        default: warp_store_out<unsigned char>(p, h.dst, h.row_bytes, lane); break;
+      }
+      __syncwarp();
+    }
+    for (uint32_t r = lane; r < (h.width ? 0u : h.rows); r += 32) {
       if (hint_st) {
         bulk_store_hint(h.dst + uint64_t(r) * h.dp, base + r * h.row_bytes, h.row_bytes, pol);
       } else {

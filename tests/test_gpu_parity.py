@@ -13,7 +13,7 @@ import torch
 import paper_2407_20143_b200 as bcp
 from oracle import reshard_oracle as orc
 from workloads import fills
-from workloads.configs import CONFIGS, scenario_cases
+from workloads.configs import CONFIGS, STRESS, scenario_cases
 from workloads.meta import ShardMeta
 from workloads.random_cases import big_random_case, random_case
 
@@ -71,11 +71,15 @@ def test_random_tiny(cuda_device, seed):
                     small_bytes=64 if seed % 3 else 4096)
 
 
+@pytest.mark.parametrize("path_mask", [1, 3])
 @pytest.mark.parametrize("itemsize,seed", [(1, 1), (2, 2), (4, 3), (8, 4), (2, 5), (4, 6)])
-def test_big_random_misaligned(cuda_device, itemsize, seed):
-    """Odd shapes and byte offsets: every access width from 1 to 16 bytes, ragged heads and tails."""
-    st = run_and_compare(big_random_case(seed, itemsize=itemsize), cuda_device, tile_bytes=8192 if seed % 2 else 65536)
+def test_big_random_misaligned(cuda_device, itemsize, seed, path_mask):
+    """Odd shapes and byte offsets: every access width from 1 to 16 bytes, ragged heads and tails,
+    through the register kernel and through the shifted-run staging of the TMA kernel."""
+    st = run_and_compare(big_random_case(seed, itemsize=itemsize), cuda_device, tile_bytes=8192 if seed % 2 else 65536,
+                         path_mask=path_mask, tma_stage_bytes=4096 if seed % 3 == 0 else 32768)
     assert st["bytes_misaligned"] > 0
+    assert (st["n_tma_tiles"] > 0) == (path_mask == 3)
 
 
 @pytest.mark.parametrize("opts", [dict(block_threads=256, ctas_per_sm=4), dict(block_threads=1024, ctas_per_sm=1),
@@ -254,9 +258,10 @@ def _free_gb():
     return free / 1e9
 
 
-@pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6)])
+@pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6),
+                                                ("cfg4odd", 0.5e9)])
 def test_full_size_config(cuda_device, name, max_fqn_bytes):
-    case = CONFIGS[name]()
+    case = (CONFIGS.get(name) or STRESS[name])()
     need = (sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)) / 1e9 + 8
     assert _free_gb() > need, f"{name} needs {need:.0f} GB of device memory"
     keys = case.key_ids

@@ -54,6 +54,19 @@ def cfg5(layers: int = 16) -> ReshardCase:
                         Parallelism(ep=8), Parallelism(ep=4), MOE_KINDS, "uniform", seed=20148)
 
 
+def cfg4_odd(layers: int = 28) -> ReshardCase:
+    """Unscored stress variant of cfg4: DP61 -> DP47, so flat slices are 1,650,319 and 2,141,903
+    elements long (both odd): source and target byte offsets differ by odd multiples of 4 bytes
+    and no copy can use 16-byte accesses on both sides."""
+    m = llama_model("llama-3b-fsdp", L=layers, H=3072, nq=24, nkv=8, F=8192, V=128256, fused=False,
+                    tied=True, fsdp_units=True)
+    return reshard_case("cfg4-odd-dp61-to-dp47" + ("" if layers == 28 else f"-L{layers}"), m,
+                        Parallelism(dp=61, zero="fsdp"), Parallelism(dp=47, zero="fsdp"),
+                        OPTIM_ONLY, "index", seed=20149)
+
+
+STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd}
+
 CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
     "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
 
