@@ -40,7 +40,7 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes moved per algorithmic byte by the dominant kernel, from ncu captures summarised
 # under profiles/ (bcp_tma_kernel_*.md): (dram__bytes_read.sum + dram__bytes_write.sum) / B_min.
-NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.993}
+NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.9994, ("cfg3", "bcp_tma_kernel"): 0.9990}
 
 
 def parse_args():
@@ -328,8 +328,10 @@ def main():
     ratio = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get((a.workload, dominant))
     if ratio is not None:
         out["roofline"]["traffic"] = ratio * b_min
-        out["roofline"]["traffic_note"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch (see profiles/), " \
-                                          "scaled by algorithmic bytes where the capture ran a shallower model"
+        out["roofline"]["traffic_note"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch " \
+                                          "(profiles/bcp_tma_kernel_full_size_dram_bytes.md)"
+        if a.layers:
+            out["roofline"]["traffic_note"] += ", scaled by algorithmic bytes to this shallower model"
 
     if a.pack and rank == 0:
         out["pack"] = time_pack(case, dst, dev, stream, a.steps)
