@@ -196,6 +196,39 @@ def time_oracle(case, fetch_payload, target_bytes: float, steps: int = 1, warmup
     return sum(times) / len(times), src_b, dst_b, len(picked)
 
 
+def _oracle_job(i):
+    from oracle import reshard_oracle as orc
+
+    ss, ps, ds = _ORACLE_INPUTS[i]
+    orc.reshard_fqn(ss, ps, ds)
+    return i
+
+
+_ORACLE_INPUTS = []
+
+
+def time_oracle_all_cores(case, fetch_payload, target_bytes: float, passes: int = 3):
+    """The same oracle, one FQN per task over a fork pool of all host cores (inputs are
+    inherited by the workers, results are dropped)."""
+    import multiprocessing as mp
+
+    global _ORACLE_INPUTS
+    picked, by_src, by_dst = oracle_sample(case, target_bytes)
+    _ORACLE_INPUTS = [(by_src[n], [fetch_payload(s) for s in by_src[n]], by_dst[n]) for n in picked]
+    src_b = sum(s.byte_length for ss, _, _ in _ORACLE_INPUTS for s in ss)
+    dst_b = sum(d.byte_length for _, _, ds in _ORACLE_INPUTS for d in ds)
+    cores = os.cpu_count() or 1
+    ctx = mp.get_context("fork")
+    with ctx.Pool(cores) as pool:
+        pool.map(_oracle_job, range(len(_ORACLE_INPUTS)))  # warm-up
+        t0 = time.perf_counter()
+        for _ in range(passes):
+            pool.map(_oracle_job, range(len(_ORACLE_INPUTS)), chunksize=1)
+        sec = (time.perf_counter() - t0) / passes
+    _ORACLE_INPUTS = []
+    return sec, src_b, dst_b, len(picked), cores
+
+
 def run_reference(a):
     """The oracle as it stands, on host cores, on a bounded sample per step (rank 0 only)."""
     from paper_2407_20143_b200 import dist as D
@@ -354,6 +387,12 @@ def main():
                                "sample": f"{n} FQNs of {case.name}, {sb + db} bytes read+written per pass, "
                                          f"mean of {a.cpu_passes} passes, {sec:.2f} s each",
                                "host_cores_available": os.cpu_count()}
+        try:
+            sec2, sb2, db2, n2, cores = time_oracle_all_cores(case, fetch, a.cpu_sample_gb * 1e9 / 2)
+            out["cpu_baseline_all_cores"] = {"value": (sb2 + db2) / sec2 / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                             "sample": f"same {n2} FQNs, one FQN per task over a fork pool, {sec2:.2f} s per pass"}
+        except Exception as e:  # the single-core figure above is the reported baseline
+            out["cpu_baseline_all_cores"] = {"value": None, "error": str(e)[:200]}
     plan.destroy()
     if rank == 0:
         print(json.dumps(out))
@@ -383,8 +422,28 @@ def time_pack(case, dst, dev, stream, steps):
     torch.cuda.synchronize()
     ms_step = e0.elapsed_time(e1) / steps
     nbytes = sum(sizes) + total
-    del blob
-    return {"tensors": len(ms), "blob_bytes": total, "ms_per_pack": ms_step, "gbps": nbytes / (ms_step * 1e-3) / 1e9}
+    # unpack: the blob back into a second set of tensor buffers
+    outs = torch.empty(sum(sizes) + 256 * len(sizes), dtype=torch.uint8, device=dev)
+    optrs, pos = [], 0
+    for n in sizes:
+        optrs.append(outs.data_ptr() + pos)
+        pos += (n + 255) // 256 * 256
+    for _ in range(3):
+        bcp.bcp_unpack(blob, metas, optrs, stream=stream)
+    torch.cuda.synchronize()
+    u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    u0.record(stream)
+    for _ in range(steps):
+        bcp.bcp_unpack(blob, metas, optrs, stream=stream)
+    u1.record(stream)
+    torch.cuda.synchronize()
+    ms_un = u0.elapsed_time(u1) / steps
+    ok = all(bool(torch.equal(outs[o - outs.data_ptr():o - outs.data_ptr() + n],
+                              dst[r][m.byte_offset:m.byte_offset + n])) for o, n, m in list(zip(optrs, sizes, ms))[:64])
+    del blob, outs
+    return {"tensors": len(ms), "blob_bytes": total, "ms_per_pack": ms_step, "gbps": nbytes / (ms_step * 1e-3) / 1e9,
+            "ms_per_unpack": ms_un, "unpack_gbps": 2 * sum(sizes) / (ms_un * 1e-3) / 1e9, "round_trip_ok": ok,
+            "bytes_counted": "pack: tensor bytes read + blob bytes written (padding included); unpack: 2 x tensor bytes"}
 
 
 def run_e2e(a, case, plan, src, dst, dev, ws, b_min):

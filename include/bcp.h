@@ -235,9 +235,11 @@ BCP_API int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n
 
 /*
  * Same operation with HOST buffers (host pointers to host memory, pinned for full speed):
- * copies every source blob to plan-owned device staging memory, runs the kernels,
- * copies every target buffer back, all on `stream`, and waits for completion.
- * Target bytes not named by any target entry come back as zero.
+ * copies the source blobs to plan-owned device staging memory, runs the kernels and
+ * copies the target buffers back, then waits for completion.  Work is pipelined per target
+ * buffer over three streams (`stream` for the kernels, two plan-owned streams for uploads and
+ * downloads), so that downloads of finished target buffers overlap the uploads still
+ * needed by later ones.  Target bytes not named by any target entry come back as zero.
  */
 BCP_API int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
                      void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);

@@ -25,8 +25,18 @@ struct bcp_plan {
   cudaStream_t last_stream = nullptr;
   bool ran = false;
   std::vector<void*> h_ptrs;
-  // staging for bcp_reshard_host
+  // bcp_reshard_host: device staging plus a second copy of the work list grouped by target
+  // buffer, so that uploads, kernels and downloads of different target buffers overlap
+  struct Group {  // units of one target buffer inside d_host_tiles
+    size_t first = 0, n_tma = 0, n_big = 0, n_small = 0;
+    std::vector<uint32_t> needs;  // source buffers its units read
+  };
   std::vector<void*> stage_src, stage_dst;
+  bcp_tile* d_host_tiles = nullptr;
+  std::vector<Group> groups;     // one per target buffer
+  std::vector<uint32_t> order;   // target buffers in processing order
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+  std::vector<cudaEvent_t> ev_src, ev_dst;
 };
 
 namespace {
@@ -60,6 +70,40 @@ int bind_device(bcp_plan_t* p) {
   return BCP_OK;
 }
 
+// Enqueue the kernels for a slice of a device work list laid out as [TMA | CTA-wide | warp units].
+int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_big, size_t n_small, cudaStream_t stream) {
+  const size_t ns = p->src_bytes.size();
+  if (n_tma) {
+    TmaLaunchArgs t;
+    t.tiles = tiles;
+    t.n_tiles = uint32_t(n_tma);
+    t.src = reinterpret_cast<const void* const*>(p->d_ptrs);
+    t.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
+    t.ctrl = p->d_ctrl + 1;
+    t.stage_bytes = p->opt.tma_stage_bytes;
+    t.n_stages = p->opt.tma_stages;
+    t.grid = uint32_t(n_tma < p->tma_grid ? n_tma : p->tma_grid);
+    t.wait_limit = 1u << 22;
+    t.cache_hints = p->opt.cache_hints;
+    BCP_CUDA(launch_tma(t, stream));
+  }
+  LaunchArgs a;
+  a.tiles = tiles + n_tma;
+  a.n_big = uint32_t(n_big);
+  a.n_small = uint32_t(n_small);
+  a.src = reinterpret_cast<const void* const*>(p->d_ptrs);
+  a.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
+  a.ctrl = p->d_ctrl;
+  a.block_threads = p->opt.block_threads;
+  const uint32_t nwarps = a.block_threads / 32;
+  const uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;
+  a.grid = uint32_t(units < p->grid ? units : p->grid);
+  a.cache_hints = p->opt.cache_hints;
+  a.unroll = p->opt.unroll;
+  if (units) BCP_CUDA(launch_copy(a, stream));
+  return BCP_OK;
+}
+
 int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, size_t nd, cudaStream_t stream) {
   if (!p) return fail(BCP_ERR_INVALID, "plan is NULL");
   if (ns != p->src_bytes.size() || nd != p->dst_bytes.size())
@@ -81,34 +125,7 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
   for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
   // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
   BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
-  if (p->n_tma) {
-    TmaLaunchArgs t;
-    t.tiles = p->d_tiles;
-    t.n_tiles = uint32_t(p->n_tma);
-    t.src = reinterpret_cast<const void* const*>(p->d_ptrs);
-    t.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
-    t.ctrl = p->d_ctrl + 1;
-    t.stage_bytes = p->opt.tma_stage_bytes;
-    t.n_stages = p->opt.tma_stages;
-    t.grid = uint32_t(p->n_tma < p->tma_grid ? p->n_tma : p->tma_grid);
-    t.wait_limit = 1u << 22;
-    t.cache_hints = p->opt.cache_hints;
-    BCP_CUDA(launch_tma(t, stream));
-  }
-  LaunchArgs a;
-  a.tiles = p->d_tiles + p->n_tma;
-  a.n_big = uint32_t(p->n_big);
-  a.n_small = uint32_t(p->tiles.size() - p->n_tma - p->n_big);
-  a.src = reinterpret_cast<const void* const*>(p->d_ptrs);
-  a.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
-  a.ctrl = p->d_ctrl;
-  a.block_threads = p->opt.block_threads;
-  const uint32_t nwarps = a.block_threads / 32;
-  const uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;
-  a.grid = uint32_t(units < p->grid ? units : p->grid);
-  a.cache_hints = p->opt.cache_hints;
-  a.unroll = p->opt.unroll;
-  if (units) BCP_CUDA(launch_copy(a, stream));
+  if (int rc = launch_units(p, p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
   p->last_stream = stream;
   p->ran = true;
   return BCP_OK;
@@ -226,6 +243,70 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
   return BCP_OK;
 }
 
+// One-time set-up of the host-buffer path: staging buffers, streams, events, and the work list
+// regrouped by target buffer.
+int prepare_host_path(bcp_plan_t* p) {
+  if (p->s_h2d) return BCP_OK;
+  const size_t ns = p->src_bytes.size(), nd = p->dst_bytes.size();
+  p->groups.assign(nd, bcp_plan::Group());
+  std::vector<std::vector<bcp_tile>> tma(nd), big(nd), small(nd);
+  std::vector<std::vector<char>> need(nd, std::vector<char>(ns, 0));
+  for (const bcp_tile& t : p->tiles) {
+    const uint32_t d = t.dst_buf;
+    if (!(t.flags & BCP_TILE_ZERO)) need[d][t.src_buf] = 1;
+    ((t.flags & BCP_TILE_TMA) ? tma : (t.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(t);
+  }
+  std::vector<bcp_tile> flat;
+  flat.reserve(p->tiles.size());
+  for (size_t d = 0; d < nd; ++d) {
+    bcp_plan::Group& g = p->groups[d];
+    g.first = flat.size();
+    g.n_tma = tma[d].size();
+    g.n_big = big[d].size();
+    g.n_small = small[d].size();
+    flat.insert(flat.end(), tma[d].begin(), tma[d].end());
+    flat.insert(flat.end(), big[d].begin(), big[d].end());
+    flat.insert(flat.end(), small[d].begin(), small[d].end());
+    for (uint32_t sb = 0; sb < ns; ++sb)
+      if (need[d][sb]) g.needs.push_back(sb);
+  }
+  // order: always take the target buffer that needs the fewest bytes not yet uploaded, so that
+  // the first download starts early and uploads keep running under the downloads
+  std::vector<char> have(ns, 0), done(nd, 0);
+  for (size_t k = 0; k < nd; ++k) {
+    size_t best = nd;
+    uint64_t best_cost = ~uint64_t(0);
+    for (size_t d = 0; d < nd; ++d) {
+      if (done[d]) continue;
+      uint64_t cost = 0;
+      for (uint32_t sb : p->groups[d].needs)
+        if (!have[sb]) cost += p->src_bytes[sb];
+      if (cost < best_cost) {
+        best_cost = cost;
+        best = d;
+      }
+    }
+    done[best] = 1;
+    for (uint32_t sb : p->groups[best].needs) have[sb] = 1;
+    p->order.push_back(uint32_t(best));
+  }
+  if (!flat.empty()) {
+    BCP_CUDA(cudaMalloc(&p->d_host_tiles, flat.size() * sizeof(bcp_tile)));
+    BCP_CUDA(cudaMemcpy(p->d_host_tiles, flat.data(), flat.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
+  }
+  p->stage_src.assign(ns, nullptr);
+  p->stage_dst.assign(nd, nullptr);
+  for (size_t i = 0; i < ns; ++i) BCP_CUDA(cudaMalloc(&p->stage_src[i], p->src_bytes[i] ? p->src_bytes[i] : 16));
+  for (size_t i = 0; i < nd; ++i) BCP_CUDA(cudaMalloc(&p->stage_dst[i], p->dst_bytes[i] ? p->dst_bytes[i] : 16));
+  p->ev_src.assign(ns, nullptr);
+  p->ev_dst.assign(nd ? nd : 1, nullptr);
+  for (cudaEvent_t& e : p->ev_src) BCP_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (cudaEvent_t& e : p->ev_dst) BCP_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  BCP_CUDA(cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking));
+  BCP_CUDA(cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking));  // set last: marks the path as ready
+  return BCP_OK;
+}
+
 // address -> (address rounded down to 16 bytes, remainder)
 void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vector<uint8_t>* res,
                       std::vector<const void*>* bases) {
@@ -327,27 +408,45 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
   if (n_src_bufs != plan->src_bytes.size() || n_dst_bufs != plan->dst_bytes.size())
     return fail(BCP_ERR_INVALID, "buffer counts differ from the planned ones");
   if ((n_src_bufs && !src_host) || (n_dst_bufs && !dst_host)) return fail(BCP_ERR_INVALID, "pointer array is NULL");
-  if (int rc = bind_device(plan)) return rc;
-  if (plan->stage_src.empty() && plan->stage_dst.empty()) {
-    plan->stage_src.assign(n_src_bufs, nullptr);
-    plan->stage_dst.assign(n_dst_bufs, nullptr);
-    for (size_t i = 0; i < n_src_bufs; ++i) BCP_CUDA(cudaMalloc(&plan->stage_src[i], plan->src_bytes[i] ? plan->src_bytes[i] : 1));
-    for (size_t i = 0; i < n_dst_bufs; ++i) BCP_CUDA(cudaMalloc(&plan->stage_dst[i], plan->dst_bytes[i] ? plan->dst_bytes[i] : 1));
-  }
-  for (size_t i = 0; i < n_src_bufs; ++i) {
-    if (!plan->src_bytes[i]) continue;
-    if (!src_host[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
-    BCP_CUDA(cudaMemcpyAsync(plan->stage_src[i], src_host[i], plan->src_bytes[i], cudaMemcpyHostToDevice, stream));
-  }
+  for (size_t i = 0; i < n_src_bufs; ++i)
+    if (plan->src_bytes[i] && !src_host[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
   for (size_t i = 0; i < n_dst_bufs; ++i)
-    if (plan->dst_bytes[i]) BCP_CUDA(cudaMemsetAsync(plan->stage_dst[i], 0, plan->dst_bytes[i], stream));
-  if (int rc = execute(plan, plan->stage_src.data(), n_src_bufs, plan->stage_dst.data(), n_dst_bufs, stream)) return rc;
-  for (size_t i = 0; i < n_dst_bufs; ++i) {
-    if (!plan->dst_bytes[i]) continue;
-    if (!dst_host[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
-    BCP_CUDA(cudaMemcpyAsync(dst_host[i], plan->stage_dst[i], plan->dst_bytes[i], cudaMemcpyDeviceToHost, stream));
+    if (plan->dst_bytes[i] && !dst_host[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
+  if (int rc = bind_device(plan)) return rc;
+  if (int rc = prepare_host_path(plan)) return rc;
+  bcp_plan_t* p = plan;
+  // device-side pointer table: the staging buffers
+  for (size_t i = 0; i < n_src_bufs; ++i) p->h_ptrs[i] = p->stage_src[i];
+  for (size_t i = 0; i < n_dst_bufs; ++i) p->h_ptrs[n_src_bufs + i] = p->stage_dst[i];
+  BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (n_src_bufs + n_dst_bufs) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  // The upload stream starts after whatever the caller queued on `stream` before this call.
+  BCP_CUDA(cudaEventRecord(p->ev_dst[0], stream));
+  BCP_CUDA(cudaStreamWaitEvent(p->s_h2d, p->ev_dst[0], 0));
+  std::vector<char> uploaded(n_src_bufs, 0);
+  // Target buffers one after the other: upload the sources it still misses, run its units,
+  // download it.  Uploads, kernels and downloads sit on three streams, so the download of one
+  // target buffer overlaps the uploads for the next (PCIe is full duplex).
+  for (uint32_t d : p->order) {
+    const bcp_plan::Group& g = p->groups[d];
+    for (uint32_t sb : g.needs) {
+      if (uploaded[sb]) continue;
+      uploaded[sb] = 1;
+      BCP_CUDA(cudaMemcpyAsync(p->stage_src[sb], src_host[sb], p->src_bytes[sb], cudaMemcpyHostToDevice, p->s_h2d));
+      BCP_CUDA(cudaEventRecord(p->ev_src[sb], p->s_h2d));
+    }
+    if (!p->dst_bytes[d]) continue;
+    for (uint32_t sb : g.needs) BCP_CUDA(cudaStreamWaitEvent(stream, p->ev_src[sb], 0));
+    BCP_CUDA(cudaMemsetAsync(p->stage_dst[d], 0, p->dst_bytes[d], stream));
+    if (int rc = launch_units(p, p->d_host_tiles + g.first, g.n_tma, g.n_big, g.n_small, stream)) return rc;
+    BCP_CUDA(cudaEventRecord(p->ev_dst[d], stream));
+    BCP_CUDA(cudaStreamWaitEvent(p->s_d2h, p->ev_dst[d], 0));
+    BCP_CUDA(cudaMemcpyAsync(dst_host[d], p->stage_dst[d], p->dst_bytes[d], cudaMemcpyDeviceToHost, p->s_d2h));
   }
+  p->last_stream = stream;
+  p->ran = true;
+  BCP_CUDA(cudaStreamSynchronize(p->s_h2d));
   BCP_CUDA(cudaStreamSynchronize(stream));
+  BCP_CUDA(cudaStreamSynchronize(p->s_d2h));
   return BCP_OK;
 }
 
@@ -377,8 +476,17 @@ int bcp_plan_destroy(bcp_plan_t* plan) {
       cudaGetLastError();
       cudaDeviceSynchronize();
     }
+    if (plan->s_h2d) cudaStreamSynchronize(plan->s_h2d);
+    if (plan->s_d2h) cudaStreamSynchronize(plan->s_d2h);
+    for (cudaEvent_t e : plan->ev_src)
+      if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : plan->ev_dst)
+      if (e) cudaEventDestroy(e);
+    if (plan->s_h2d) cudaStreamDestroy(plan->s_h2d);
+    if (plan->s_d2h) cudaStreamDestroy(plan->s_d2h);
     for (void* q : plan->stage_src) cudaFree(q);
     for (void* q : plan->stage_dst) cudaFree(q);
+    cudaFree(plan->d_host_tiles);
     cudaFree(plan->d_tiles);
     cudaFree(plan->d_ptrs);
     cudaFree(plan->d_ctrl);
