@@ -190,6 +190,19 @@ BCP_API int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_be
                   size_t* n);
 
 /*
+ * Save-side de-duplication with load balancing (Sec. 4.1, "Balancing saving workload").
+ * Shard i has shard_bytes[i] bytes and is held by the ranks
+ * holders[holder_offsets[i] .. holder_offsets[i+1]) (at least one; rank ids < n_ranks).
+ * Shards are taken in input order and each is assigned to the holder whose cumulative
+ * assigned bytes are smallest at that moment (worst fit; ties go to the lowest rank id).
+ * rank_load[n_ranks] is read as the load every rank starts with (bytes it has to save
+ * anyway) and receives the final loads; out_owner[n_shards] receives the owners.
+ * Host only; all arrays are host memory, caller-owned.
+ */
+BCP_API int bcp_dedup_assign(const uint64_t* shard_bytes, const uint64_t* holder_offsets, const uint32_t* holders,
+                             size_t n_shards, size_t n_ranks, uint64_t* rank_load, uint32_t* out_owner);
+
+/*
  * Load-time matching and plan construction (Sec. 3.3, Step 2; plan reuse: Sec. 4.1,
  * "Plan and metadata cache").  Host only: no device is touched, so it also runs on a
  * machine without a GPU.

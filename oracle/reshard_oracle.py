@@ -167,3 +167,21 @@ def pack(tensors: Sequence[np.ndarray], align: int = 256):
 
 def unpack(blob: np.ndarray, table: Sequence[Tuple[int, int]]) -> List[np.ndarray]:
     return [blob[o:o + n].copy() for (o, n) in table]
+
+
+# --------------------------------------------------------------------------- save-side de-duplication
+def worst_fit(shard_bytes: Sequence[int], holders: Sequence[Sequence[int]], n_ranks: int, initial_load=None):
+    """Owner of every shard (Sec. 4.1, "Balancing saving workload"): walk the shards in order
+    and give each to the holder with the smallest cumulative size so far (lowest rank on ties).
+    The paper states the procedure, so this follows its steps; pinned by a hand-worked example
+    and by the list-scheduling bound (tests/test_dedup.py)."""
+    load = list(initial_load) if initial_load is not None else [0] * n_ranks
+    owners = []
+    for size, hs in zip(shard_bytes, holders):
+        if not hs:
+            raise OracleError("a shard needs at least one holder")
+        smallest = min(load[r] for r in hs)
+        owner = min(r for r in hs if load[r] == smallest)
+        load[owner] += int(size)
+        owners.append(owner)
+    return owners, load

@@ -77,6 +77,8 @@ _PROTOS = {
     "bcp_last_error": (C.c_char_p, []),
     "bcp_decompose": (C.c_int, [C.POINTER(C.c_int64), C.c_uint32, C.c_int64, C.c_int64, _VP, _VP, C.c_size_t,
                                 C.POINTER(C.c_size_t)]),
+    "bcp_dedup_assign": (C.c_int, [C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.c_size_t,
+                                   C.c_size_t, C.POINTER(C.c_uint64), C.POINTER(C.c_uint32)]),
     "bcp_plan": (C.c_int, [C.POINTER(ShardMetaC), C.c_size_t, C.POINTER(C.c_uint64), C.c_size_t,
                            C.POINTER(ShardMetaC), C.c_size_t, C.POINTER(C.c_uint64), C.c_size_t,
                            C.POINTER(PlanOptsC), C.POINTER(_VP)]),

@@ -113,6 +113,21 @@ def bcp_decompose(lengths: Sequence[int], flat_begin: int, flat_end: int):
     return [(tuple(off[i][:nd]), tuple(ln[i][:nd])) for i in range(n.value)]
 
 
+def bcp_dedup_assign(shard_bytes: Sequence[int], holders: Sequence[Sequence[int]], n_ranks: int,
+                     initial_load: Optional[Sequence[int]] = None) -> Tuple[List[int], List[int]]:
+    """Worst-fit owner of every replicated shard; returns (owners, final per-rank loads)."""
+    n = len(shard_bytes)
+    offs, flat = [0], []
+    for h in holders:
+        flat.extend(h)
+        offs.append(len(flat))
+    load = (C.c_uint64 * max(1, n_ranks))(*(initial_load if initial_load is not None else [0] * n_ranks))
+    owner = (C.c_uint32 * max(1, n))()
+    _check(L.lib().bcp_dedup_assign(_u64(shard_bytes), _u64(offs), (C.c_uint32 * max(1, len(flat)))(*flat), n, n_ranks,
+                                    load, owner))
+    return list(owner[:n]), list(load[:n_ranks])
+
+
 def bcp_plan(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas: Sequence, dst_buf_bytes: Sequence[int],
              **opts) -> Plan:
     """Match wanted against saved entries and build the work list (host only)."""

@@ -354,6 +354,28 @@ int bcp_decompose(const int64_t* lengths, uint32_t ndim, int64_t flat_begin, int
   return BCP_OK;
 }
 
+int bcp_dedup_assign(const uint64_t* shard_bytes, const uint64_t* holder_offsets, const uint32_t* holders, size_t n_shards,
+                     size_t n_ranks, uint64_t* rank_load, uint32_t* out_owner) {
+  if (n_shards && (!shard_bytes || !holder_offsets || !holders || !out_owner)) return fail(BCP_ERR_INVALID, "bcp_dedup_assign: NULL argument");
+  if (n_ranks && !rank_load) return fail(BCP_ERR_INVALID, "bcp_dedup_assign: rank_load is NULL");
+  // validate everything first: a failing call must leave its outputs untouched
+  for (size_t i = 0; i < n_shards; ++i) {
+    if (holder_offsets[i + 1] <= holder_offsets[i]) return fail(BCP_ERR_INVALID, "bcp_dedup_assign: shard %zu has no holder", i);
+    for (uint64_t k = holder_offsets[i]; k < holder_offsets[i + 1]; ++k)
+      if (holders[k] >= n_ranks) return fail(BCP_ERR_BOUNDS, "bcp_dedup_assign: shard %zu is held by rank %u of %zu", i, holders[k], n_ranks);
+  }
+  for (size_t i = 0; i < n_shards; ++i) {
+    uint32_t best = holders[holder_offsets[i]];
+    for (uint64_t k = holder_offsets[i] + 1; k < holder_offsets[i + 1]; ++k) {
+      const uint32_t r = holders[k];
+      if (rank_load[r] < rank_load[best] || (rank_load[r] == rank_load[best] && r < best)) best = r;
+    }
+    rank_load[best] += shard_bytes[i];
+    out_owner[i] = best;
+  }
+  return BCP_OK;
+}
+
 int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
              const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
              const bcp_plan_opts* opts, bcp_plan_t** out_plan) {
