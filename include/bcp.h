@@ -101,7 +101,7 @@ typedef struct {
 typedef struct {
   uint32_t tile_bytes;     /* payload of one CTA-wide work unit; default 65536; multiple of 4096      */
   uint32_t small_bytes;    /* work units with a payload below this go to the warp path; default 4096  */
-  uint32_t block_threads;  /* threads per CTA of the copy kernel: 128..1024, multiple of 32; default 512 */
+  uint32_t block_threads;  /* threads per CTA of the register kernel: 256, 512 or 1024; default 512     */
   uint32_t ctas_per_sm;    /* persistent CTAs per SM; default 2                                       */
   uint32_t order;          /* 0 default (= 1); 1 order work by source address (replica reads of one
                               source region run back to back and hit L2); 2 order by target address    */

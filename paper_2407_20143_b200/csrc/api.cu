@@ -47,13 +47,7 @@ namespace {
     if (e_ != cudaSuccess) return fail(BCP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
 
-int bind_device(bcp_plan_t* p) {
-  int dev = 0;
-  BCP_CUDA(cudaGetDevice(&dev));
-  if (p->device >= 0) {
-    if (p->device != dev) return fail(BCP_ERR_INVALID, "plan is bound to device %d but device %d is current", p->device, dev);
-    return BCP_OK;
-  }
+int bind_device_alloc(bcp_plan_t* p) {
   const size_t n_ptrs = p->src_bytes.size() + p->dst_bytes.size();
   if (!p->tiles.empty()) {
     BCP_CUDA(cudaMalloc(&p->d_tiles, p->tiles.size() * sizeof(bcp_tile)));
@@ -66,6 +60,27 @@ int bind_device(bcp_plan_t* p) {
   if (p->n_tma)
     BCP_CUDA(tma_kernel_max_grid(p->opt.tma_stage_bytes, p->opt.tma_stages, p->opt.tma_ctas_per_sm, &p->tma_grid));
   p->h_ptrs.resize(n_ptrs);
+  return BCP_OK;
+}
+
+// First execution of a plan: upload the work list to the current device and size the grids.
+int bind_device(bcp_plan_t* p) {
+  int dev = 0;
+  BCP_CUDA(cudaGetDevice(&dev));
+  if (p->device >= 0) {
+    if (p->device != dev) return fail(BCP_ERR_INVALID, "plan is bound to device %d but device %d is current", p->device, dev);
+    return BCP_OK;
+  }
+  if (int rc = bind_device_alloc(p)) {  // leave nothing half-built behind
+    cudaFree(p->d_tiles);
+    cudaFree(p->d_ptrs);
+    cudaFree(p->d_ctrl);
+    p->d_tiles = nullptr;
+    p->d_ptrs = nullptr;
+    p->d_ctrl = nullptr;
+    cudaGetLastError();
+    return rc;
+  }
   p->device = dev;
   return BCP_OK;
 }
@@ -150,6 +165,7 @@ double ms_since(std::chrono::steady_clock::time_point t0) {
 // ------------------------------------------------------------------ pack / unpack plan cache
 struct PackEntry {
   bool unpack;
+  int device;  // plans are bound to the device they first ran on
   uint64_t blob_bytes;
   std::vector<uint8_t> residues;  // address mod 16 of every tensor, then of the blob
   std::vector<bcp_pack_meta> metas;
@@ -166,8 +182,10 @@ const size_t kPackCacheMax = 16;
 // width of every unit accounts for it.  A layout is cached per set of remainders.
 int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_bytes,
               const std::vector<uint8_t>& residues, bcp_plan_t** out) {
+  int device = 0;
+  BCP_CUDA(cudaGetDevice(&device));
   for (PackEntry& e : g_pack_cache) {
-    if (e.unpack == unpack && e.blob_bytes == blob_bytes && e.metas.size() == n && e.residues == residues &&
+    if (e.unpack == unpack && e.device == device && e.blob_bytes == blob_bytes && e.metas.size() == n && e.residues == residues &&
         (n == 0 || memcmp(e.metas.data(), metas, n * sizeof(bcp_pack_meta)) == 0)) {
       e.stamp = ++g_pack_stamp;
       *out = e.plan;
@@ -238,7 +256,7 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
     bcp_plan_destroy(g_pack_cache[victim].plan);
     g_pack_cache.erase(g_pack_cache.begin() + victim);
   }
-  g_pack_cache.push_back(PackEntry{unpack, blob_bytes, residues, std::vector<bcp_pack_meta>(metas, metas + n), p, ++g_pack_stamp});
+  g_pack_cache.push_back(PackEntry{unpack, device, blob_bytes, residues, std::vector<bcp_pack_meta>(metas, metas + n), p, ++g_pack_stamp});
   *out = p;
   return BCP_OK;
 }

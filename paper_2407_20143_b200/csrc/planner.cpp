@@ -52,8 +52,8 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
   if (o.small_bytes > o.tile_bytes) return fail(BCP_ERR_INVALID, "small_bytes must not exceed tile_bytes");
-  if (o.block_threads < 128 || o.block_threads > 1024 || o.block_threads % 32)
-    return fail(BCP_ERR_INVALID, "block_threads must be a multiple of 32 in [128, 1024]");
+  if (o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024)
+    return fail(BCP_ERR_INVALID, "block_threads must be 256, 512 or 1024");
   if (o.ctas_per_sm < 1 || o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
   if (o.order < 1 || o.order > 2) return fail(BCP_ERR_INVALID, "order must be 1 or 2");
   if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3) return fail(BCP_ERR_INVALID, "path_mask must be 0, 1 or 3");
