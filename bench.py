@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--pack", action="store_true", help="also time bcp_pack of one target rank (reported as extra keys)")
+    ap.add_argument("--stage", action="store_true",
+                    help="also time asynchronous save staging of every target rank through the pinned ping-pong pool")
     ap.add_argument("--cpu-sample-gb", type=float, default=4.0,
                     help="bytes read+written by one pass of the CPU oracle over its sample of the workload")
     ap.add_argument("--cpu-passes", type=int, default=5)
@@ -368,6 +370,8 @@ def main():
 
     if a.pack and rank == 0:
         out["pack"] = time_pack(case, dst, dev, stream, a.steps)
+    if a.stage and rank == 0:
+        out["stage"] = time_stage(case, dst, dev, stream)
 
     # free the device-timed buffers' plan before the host-path run allocates its own staging
     if not a.no_e2e:
@@ -444,6 +448,49 @@ def time_pack(case, dst, dev, stream, steps):
     return {"tensors": len(ms), "blob_bytes": total, "ms_per_pack": ms_step, "gbps": nbytes / (ms_step * 1e-3) / 1e9,
             "ms_per_unpack": ms_un, "unpack_gbps": 2 * sum(sizes) / (ms_un * 1e-3) / 1e9, "round_trip_ok": ok,
             "bytes_counted": "pack: tensor bytes read + blob bytes written (padding included); unpack: 2 x tensor bytes"}
+
+
+def time_stage(case, dst, dev, stream):
+    """Save every target rank through a 2-slot stager: blocking time per save (the pack, device
+    timed) and whole-job throughput into pinned host memory (wall clock around all saves)."""
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+
+    jobs = []
+    for r in range(len(dst)):
+        ms = [m for m in case.dst.metas if m.buf_index == r]
+        sizes = [m.byte_length for m in ms]
+        offs, total = bcp.bcp_pack_layout(sizes, 256)
+        jobs.append(([dst[r].data_ptr() + m.byte_offset for m in ms], list(zip(offs, sizes)), total))
+    st = bcp.Stager(max(t for _, _, t in jobs), 2)
+    for ptrs, metas, total in jobs[:2]:  # warm-up: work lists cached, pinned pages touched
+        k = st.save(ptrs, metas, total, stream=stream)
+        st.wait(k)
+        st.release(k)
+    torch.cuda.synchronize()
+    evs, pending, blocked = [], [], []
+    t0 = time.perf_counter()
+    for ptrs, metas, total in jobs:
+        if len(pending) == 2:
+            k = pending.pop(0)
+            st.wait(k)
+            st.release(k)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        pending.append(st.save(ptrs, metas, total, stream=stream))
+        e1.record(stream)
+        evs.append((e0, e1))
+    for k in pending:
+        st.wait(k)
+        st.release(k)
+    wall = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    blocked = [e0.elapsed_time(e1) for e0, e1 in evs]
+    nbytes = sum(t for _, _, t in jobs)
+    st.destroy()
+    return {"ranks": len(jobs), "blob_bytes_total": nbytes, "wall_s": wall, "host_gbps": nbytes / wall / 1e9,
+            "blocking_ms_per_save": sum(blocked) / len(blocked), "slots": 2}
 
 
 def run_e2e(a, case, plan, src, dst, dev, ws, b_min):

@@ -299,6 +299,38 @@ BCP_API int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_met
 BCP_API int bcp_pack_cache_clear(void);
 
 /*
+ * Asynchronous save / load staging through a pool of pinned host buffers with ping-pong
+ * use (Sec. 4.2: the save pipeline copies shards to a pinned memory pool with ping-pong
+ * buffering so that only a short step blocks training; loading mirrors it).
+ *
+ * A stager owns n_slots pairs (device slot, pinned host slot) of slot_bytes each, one side
+ * stream and its events; create / destroy allocate and free them on the current device.
+ *
+ *   save:  bcp_stager_save packs the tensors into a free device slot on `stream` (like
+ *          bcp_pack) and queues the download of that slot to its pinned twin on the side
+ *          stream; it returns without waiting and reports the slot.  Once `stream` has passed
+ *          the pack, the tensors may be modified again: the blocking part of a save is the
+ *          pack alone.  bcp_stager_wait blocks until the download is complete and returns the
+ *          pinned blob (valid until the slot is released).  With two slots the pack of the next
+ *          blob overlaps the download of the previous one.
+ *   load:  bcp_stager_acquire hands out a free slot's pinned buffer for the caller to fill
+ *          (e.g. from storage); bcp_stager_load queues the upload on the side stream and the
+ *          unpack into `tensors` on `stream`, and returns without waiting.
+ *   bcp_stager_release returns a slot to the pool (waits for its copy to finish).
+ * BCP_ERR_CAPACITY: blob larger than a slot, or no free slot.  One thread at a time per stager.
+ */
+typedef struct bcp_stager bcp_stager_t;
+BCP_API int bcp_stager_create(uint64_t slot_bytes, uint32_t n_slots, bcp_stager_t** out);
+BCP_API int bcp_stager_destroy(bcp_stager_t* stager);
+BCP_API int bcp_stager_save(bcp_stager_t* stager, const void* const* tensors, const bcp_pack_meta* metas, size_t n,
+                            uint64_t blob_bytes, void* stream, uint32_t* out_slot);
+BCP_API int bcp_stager_wait(bcp_stager_t* stager, uint32_t slot, void** host_blob);
+BCP_API int bcp_stager_acquire(bcp_stager_t* stager, uint32_t* out_slot, void** host_blob);
+BCP_API int bcp_stager_load(bcp_stager_t* stager, uint32_t slot, uint64_t blob_bytes, const bcp_pack_meta* metas,
+                            size_t n, void* const* tensors, void* stream);
+BCP_API int bcp_stager_release(bcp_stager_t* stager, uint32_t slot);
+
+/*
  * bcp_pack for callers that cannot allocate.  (The paper has no counterpart: this entry point
  * exists for the way the library gets embedded, not for the method.)
  *

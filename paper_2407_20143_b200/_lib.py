@@ -93,6 +93,14 @@ _PROTOS = {
     "bcp_pack": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
     "bcp_unpack": (C.c_int, [_VP, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
     "bcp_pack_cache_clear": (C.c_int, []),
+    "bcp_stager_create": (C.c_int, [C.c_uint64, C.c_uint32, C.POINTER(_VP)]),
+    "bcp_stager_destroy": (C.c_int, [_VP]),
+    "bcp_stager_save": (C.c_int, [_VP, C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, C.c_uint64, _VP,
+                                  C.POINTER(C.c_uint32)]),
+    "bcp_stager_wait": (C.c_int, [_VP, C.c_uint32, C.POINTER(_VP)]),
+    "bcp_stager_acquire": (C.c_int, [_VP, C.POINTER(C.c_uint32), C.POINTER(_VP)]),
+    "bcp_stager_load": (C.c_int, [_VP, C.c_uint32, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
+    "bcp_stager_release": (C.c_int, [_VP, C.c_uint32]),
     "bcp_pack_static": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
 }
 

@@ -206,5 +206,56 @@ def bcp_unpack(blob, metas: Sequence[Tuple[int, int]], tensors: Sequence, blob_b
     _check(L.lib().bcp_unpack(bp, nb, _pack_metas(metas), len(tensors), _ptrs(tensors), _stream(stream)))
 
 
+class Stager:
+    """Pinned ping-pong pool for asynchronous save / load staging (bcp_stager_* calls)."""
+
+    def __init__(self, slot_bytes: int, n_slots: int = 2):
+        h = C.c_void_p()
+        _check(L.lib().bcp_stager_create(slot_bytes, n_slots, C.byref(h)))
+        self._h, self.slot_bytes, self.n_slots = h, slot_bytes, n_slots
+
+    def save(self, tensors: Sequence, metas: Sequence[Tuple[int, int]], blob_bytes: int, stream=None) -> int:
+        slot = C.c_uint32()
+        _check(L.lib().bcp_stager_save(self._h, _ptrs(tensors), _pack_metas(metas), len(tensors), blob_bytes,
+                                       _stream(stream), C.byref(slot)))
+        return slot.value
+
+    def wait(self, slot: int) -> int:
+        """Blocks until the slot's blob is in pinned host memory; returns its host address."""
+        p = C.c_void_p()
+        _check(L.lib().bcp_stager_wait(self._h, slot, C.byref(p)))
+        return p.value
+
+    def acquire(self) -> Tuple[int, int]:
+        """(slot, host address of its pinned buffer) for the caller to fill before load()."""
+        slot, p = C.c_uint32(), C.c_void_p()
+        _check(L.lib().bcp_stager_acquire(self._h, C.byref(slot), C.byref(p)))
+        return slot.value, p.value
+
+    def load(self, slot: int, blob_bytes: int, metas: Sequence[Tuple[int, int]], tensors: Sequence, stream=None) -> None:
+        _check(L.lib().bcp_stager_load(self._h, slot, blob_bytes, _pack_metas(metas), len(tensors), _ptrs(tensors),
+                                       _stream(stream)))
+
+    def release(self, slot: int) -> None:
+        _check(L.lib().bcp_stager_release(self._h, slot))
+
+    def host_view(self, address: int, nbytes: int):
+        """numpy uint8 view of a pinned slot (no copy)."""
+        import numpy as np
+
+        return np.ctypeslib.as_array((C.c_uint8 * nbytes).from_address(address))
+
+    def destroy(self) -> None:
+        if self._h:
+            h, self._h = self._h, C.c_void_p(None)
+            _check(L.lib().bcp_stager_destroy(h))
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
 def bcp_pack_cache_clear() -> None:
     _check(L.lib().bcp_pack_cache_clear())
