@@ -226,6 +226,21 @@ BCP_API int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* sr
 BCP_API int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out);
 
 /*
+ * Plan cache across processes (Sec. 4.1, "Plan and metadata cache": plans stay constant
+ * over a training session, so planning is paid once).  bcp_plan_serialize writes a
+ * self-contained, position-independent image of the plan (options, statistics, buffer
+ * sizes, work list, checksum) into out[0..cap) and the image size into *n; with cap too
+ * small (or out NULL) it writes nothing, stores the needed size and returns
+ * BCP_ERR_CAPACITY.  bcp_plan_deserialize rebuilds a plan from an image.  Because a work
+ * list drives device copies, the image is verified before use: magic, version, record size,
+ * checksum, and every unit against the recorded buffer sizes (in bounds, access width and
+ * path flags consistent with its offsets); anything else is BCP_ERR_INVALID.  Images are
+ * only meaningful to the library version that wrote them.
+ */
+BCP_API int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n);
+BCP_API int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan);
+
+/*
  * Host copy of the work list, in execution order (CTA-wide units first, then warp
  * units).  Writes min(cap, count) records to out (may be NULL when cap == 0) and the
  * full count to *n.

@@ -83,6 +83,8 @@ _PROTOS = {
                            C.POINTER(ShardMetaC), C.c_size_t, C.POINTER(C.c_uint64), C.c_size_t,
                            C.POINTER(PlanOptsC), C.POINTER(_VP)]),
     "bcp_plan_stats": (C.c_int, [_VP, C.POINTER(PlanStatsC)]),
+    "bcp_plan_serialize": (C.c_int, [_VP, _VP, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "bcp_plan_deserialize": (C.c_int, [_VP, C.c_size_t, C.POINTER(_VP)]),
     "bcp_plan_tiles": (C.c_int, [_VP, C.POINTER(TileC), C.c_size_t, C.POINTER(C.c_size_t)]),
     "bcp_reshard": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),
     "bcp_reshard_host": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),

@@ -85,6 +85,22 @@ class Plan:
         _check(L.lib().bcp_plan_tiles(self.handle, arr, n.value, C.byref(n)))
         return list(arr[: n.value])
 
+    def serialize(self) -> bytes:
+        """Self-contained image of the plan (bcp_plan_serialize) for reuse in another process."""
+        n = C.c_size_t()
+        L.lib().bcp_plan_serialize(self.handle, None, 0, C.byref(n))
+        buf = (C.c_uint8 * max(1, n.value))()
+        _check(L.lib().bcp_plan_serialize(self.handle, buf, n.value, C.byref(n)))
+        return bytes(buf[: n.value])
+
+    @staticmethod
+    def deserialize(image: bytes) -> "Plan":
+        h = C.c_void_p()
+        buf = (C.c_uint8 * max(1, len(image))).from_buffer_copy(image) if image else (C.c_uint8 * 1)()
+        _check(L.lib().bcp_plan_deserialize(buf, len(image), C.byref(h)))
+        p = Plan(h.value, 0, 0)
+        return p
+
     def destroy(self) -> None:
         if self._h:
             h, self._h = self._h, C.c_void_p(None)

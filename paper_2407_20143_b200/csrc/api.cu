@@ -428,6 +428,139 @@ int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out) {
   return BCP_OK;
 }
 
+namespace {
+const char kMagic[8] = {'B', 'C', 'P', 'P', 'L', 'A', 'N', '1'};
+struct ImageHeader {
+  char magic[8];
+  uint32_t version, tile_size;
+  Options opt;
+  bcp_plan_stats_t stats;
+  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles;
+};
+uint64_t fnv1a(const unsigned char* p, size_t n) {
+  uint64_t h = 1469598103934665603ull;
+  for (size_t i = 0; i < n; ++i) h = (h ^ p[i]) * 1099511628211ull;
+  return h;
+}
+// A unit is safe to execute if it stays inside its buffers and its flags match its geometry.
+bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db, const Options& opt) {
+  if (t.rows == 0 || t.row_bytes == 0 || t.dst_buf >= db.size()) return false;
+  const bool zero = t.flags & BCP_TILE_ZERO;
+  const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes;
+  if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
+  if (t.rows > 1 && t.dst_pitch < t.row_bytes) return false;
+  uint64_t bits = t.dst_off | t.row_bytes | t.dst_pitch;
+  if (!zero) {
+    if (t.src_buf >= sb.size()) return false;
+    const uint64_t span_s = uint64_t(t.rows - 1) * t.src_pitch + t.row_bytes;
+    if (t.src_off > sb[t.src_buf] || span_s > sb[t.src_buf] - t.src_off) return false;
+    bits |= t.src_off | t.src_pitch;
+  }
+  uint32_t g = 0;
+  while (g < 4 && !((bits >> g) & 1)) ++g;
+  if ((t.flags & BCP_TILE_GRAN_MASK) > g) return false;  // a wider access than the offsets allow would fault
+  if (t.flags & BCP_TILE_TMA) {
+    if (zero || t.row_bytes < 16) return false;
+    if (g < 4) {  // shifted run: one row, aligned superset inside the source buffer
+      if (t.rows != 1) return false;
+      if (((t.src_off + t.row_bytes + 15) & ~uint64_t(15)) > sb[t.src_buf]) return false;
+    }
+  }
+  return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
+}
+}  // namespace
+
+int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n) {
+  if (!plan || !n) return fail(BCP_ERR_INVALID, "bcp_plan_serialize: NULL argument");
+  const size_t need = sizeof(ImageHeader) + (plan->src_bytes.size() + plan->dst_bytes.size()) * sizeof(uint64_t) +
+                      plan->tiles.size() * sizeof(bcp_tile) + sizeof(uint64_t);
+  *n = need;
+  if (!out || cap < need) return fail(BCP_ERR_CAPACITY, "bcp_plan_serialize: image needs %zu bytes, room for %zu", need, out ? cap : size_t(0));
+  ImageHeader h;
+  memset(&h, 0, sizeof h);
+  memcpy(h.magic, kMagic, 8);
+  h.version = uint32_t(bcp_version());
+  h.tile_size = sizeof(bcp_tile);
+  h.opt = plan->opt;
+  h.stats = plan->stats;
+  h.n_src_bufs = plan->src_bytes.size();
+  h.n_dst_bufs = plan->dst_bytes.size();
+  h.n_tma = plan->n_tma;
+  h.n_big = plan->n_big;
+  h.n_tiles = plan->tiles.size();
+  unsigned char* p = static_cast<unsigned char*>(out);
+  memcpy(p, &h, sizeof h);
+  p += sizeof h;
+  if (h.n_src_bufs) memcpy(p, plan->src_bytes.data(), h.n_src_bufs * sizeof(uint64_t));
+  p += h.n_src_bufs * sizeof(uint64_t);
+  if (h.n_dst_bufs) memcpy(p, plan->dst_bytes.data(), h.n_dst_bufs * sizeof(uint64_t));
+  p += h.n_dst_bufs * sizeof(uint64_t);
+  if (h.n_tiles) memcpy(p, plan->tiles.data(), h.n_tiles * sizeof(bcp_tile));
+  p += h.n_tiles * sizeof(bcp_tile);
+  const uint64_t sum = fnv1a(static_cast<unsigned char*>(out), size_t(p - static_cast<unsigned char*>(out)));
+  memcpy(p, &sum, sizeof sum);
+  return BCP_OK;
+}
+
+int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
+  if (!image || !out_plan) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: NULL argument");
+  if (n < sizeof(ImageHeader) + sizeof(uint64_t)) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image too short");
+  ImageHeader h;
+  memcpy(&h, image, sizeof h);
+  if (memcmp(h.magic, kMagic, 8) != 0) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: not a plan image");
+  if (h.version != uint32_t(bcp_version()) || h.tile_size != sizeof(bcp_tile))
+    return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image of library version %u, this is %d", h.version, bcp_version());
+  const uint64_t lim = uint64_t(1) << 32;
+  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_tma > h.n_tiles || h.n_big > h.n_tiles - h.n_tma)
+    return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: implausible counts");
+  const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) + sizeof(uint64_t);
+  if (need != n) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image is %zu bytes, its header implies %llu", n, (unsigned long long)need);
+  const unsigned char* base = static_cast<const unsigned char*>(image);
+  uint64_t sum;
+  memcpy(&sum, base + n - sizeof sum, sizeof sum);
+  if (sum != fnv1a(base, n - sizeof sum)) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: checksum mismatch");
+  {  // the options were validated when the plan was made; re-check what the launch code relies on
+    const Options& o = h.opt;
+    if ((o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024) || o.ctas_per_sm < 1 || o.ctas_per_sm > 16 ||
+        o.tile_bytes < 4096 || o.tile_bytes > (64u << 20) || (o.unroll != 4 && o.unroll != 8) || o.tma_stages < 2 || o.tma_stages > 8 ||
+        o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536 ||
+        uint64_t(o.tma_stage_bytes) * o.tma_stages > 200 * 1024 || o.tma_ctas_per_sm < 1 || o.tma_ctas_per_sm > 16 || o.cache_hints < 1 ||
+        o.cache_hints > 4)
+      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: options out of range");
+  }
+  bcp_plan_t* p = new (std::nothrow) bcp_plan_t;
+  if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
+  try {
+    const unsigned char* q = base + sizeof h;
+    p->opt = h.opt;
+    p->stats = h.stats;
+    p->src_bytes.resize(h.n_src_bufs);
+    p->dst_bytes.resize(h.n_dst_bufs);
+    p->tiles.resize(h.n_tiles);
+    if (h.n_src_bufs) memcpy(p->src_bytes.data(), q, h.n_src_bufs * sizeof(uint64_t));
+    q += h.n_src_bufs * sizeof(uint64_t);
+    if (h.n_dst_bufs) memcpy(p->dst_bytes.data(), q, h.n_dst_bufs * sizeof(uint64_t));
+    q += h.n_dst_bufs * sizeof(uint64_t);
+    if (h.n_tiles) memcpy(p->tiles.data(), q, h.n_tiles * sizeof(bcp_tile));
+    p->n_tma = h.n_tma;
+    p->n_big = h.n_big;
+  } catch (const std::bad_alloc&) {
+    delete p;
+    return fail(BCP_ERR_NOMEM, "out of host memory");
+  }
+  for (size_t i = 0; i < p->tiles.size(); ++i) {
+    const bcp_tile& t = p->tiles[i];
+    const bool in_tma = i < p->n_tma, in_small = i >= p->n_tma + p->n_big;
+    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
+        bool(t.flags & BCP_TILE_SMALL) != in_small) {
+      delete p;
+      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: work unit %zu is inconsistent with the recorded buffers", i);
+    }
+  }
+  *out_plan = p;
+  return BCP_OK;
+}
+
 int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n) {
   if (!plan || !n || (cap && !out)) return fail(BCP_ERR_INVALID, "bcp_plan_tiles: NULL argument");
   *n = plan->tiles.size();

@@ -15,7 +15,7 @@ from oracle import reshard_oracle as orc
 from workloads import fills
 from workloads.configs import CONFIGS, STRESS, scenario_cases
 from workloads.meta import ShardMeta
-from workloads.random_cases import big_random_case, random_case
+from workloads.random_cases import big_random_case, many_tiny_case, random_case
 
 pytestmark = pytest.mark.gpu
 GUARD = 4096
@@ -126,6 +126,39 @@ def test_side_stream_and_plan_reuse(cuda_device):
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
         run_and_compare(scenario_cases()[3], cuda_device, runs=4, stream=s)
+
+
+@pytest.mark.parametrize("seed", range(100, 106))
+def test_random_up_to_eight_dims(cuda_device, seed):
+    run_and_compare(random_case(seed, n_tensors=3, max_ndim=8, max_dim=3, dst_replicas=1 + seed % 2), cuda_device,
+                    tile_bytes=4096)
+
+
+def test_hundred_thousand_tiny_tensors(cuda_device):
+    case = many_tiny_case(100_000)
+    g = torch.Generator(device="cpu").manual_seed(11)
+    host = [torch.randint(0, 256, (n,), dtype=torch.uint8, generator=g) for n in case.src.buf_bytes]
+    want = orc.reshard(case.src.metas, [h.numpy() for h in host], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    st = plan.stats()
+    assert st["n_fqns"] == 100_000 and st["n_small_tiles"] > 50_000 and st["plan_ms"] < 5000
+    dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(plan, [h.to(cuda_device) for h in host], dst)
+    torch.cuda.synchronize()
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
+
+
+def test_deserialized_plan_executes(cuda_device):
+    """A plan image written by one plan object runs identically when rebuilt (plan cache)."""
+    case = CONFIGS["cfg1"]("index")
+    first = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3)
+    plan = bcp.Plan.deserialize(first.serialize())
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device)
+    dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(plan, src, dst)
+    torch.cuda.synchronize()
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
 
 
 def test_degenerate_entries(cuda_device):

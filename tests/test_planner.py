@@ -142,6 +142,12 @@ def test_random_tiny_cases(seed):
     check_case(random_case(seed, dst_replicas=1 + seed % 2), tile_bytes=4096, small_bytes=64 if seed % 3 else 4096)
 
 
+@pytest.mark.parametrize("seed", range(100, 112))
+def test_random_cases_up_to_eight_dims(seed):
+    """The maximum rank the ABI allows, with flat slices that need deep decompositions."""
+    check_case(random_case(seed, n_tensors=3, max_ndim=8, max_dim=3, dst_replicas=1 + seed % 2), tile_bytes=4096)
+
+
 @pytest.mark.parametrize("itemsize,seed", [(1, 1), (2, 2), (4, 3), (8, 4), (2, 5)])
 def test_big_random_cases(itemsize, seed):
     st = check_case(big_random_case(seed, itemsize=itemsize), tile_bytes=8192, order=1 + seed % 2)
@@ -181,6 +187,41 @@ def test_plans_partitioned_by_target_rank_cover_everything():
     assert total == case.dst.total_bytes
     for g, w in zip(got, want):
         assert np.array_equal(g, w)
+
+
+# ---- plan images (plan cache across processes, Sec. 4.1) ----------------------------------------------
+def _tile_tuple(t):
+    return (t.src_off, t.dst_off, t.src_pitch, t.dst_pitch, t.row_bytes, t.rows, t.src_buf, t.dst_buf, t.flags)
+
+
+@pytest.mark.parametrize("case", [CONFIGS["cfg1"]("index"), scenario_cases()[3], big_random_case(5, itemsize=2)],
+                         ids=lambda c: c.name)
+def test_plan_image_round_trip(case):
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3, tile_bytes=16384)
+    image = plan.serialize()
+    again = bcp.Plan.deserialize(image)
+    assert [_tile_tuple(t) for t in again.tiles()] == [_tile_tuple(t) for t in plan.tiles()]
+    assert again.stats() == plan.stats()
+    assert again.serialize() == image
+    # the rebuilt work list still computes the oracle's result
+    blobs = np_bufs(fills.fill_state(case.src, case.key_ids, "index", case.seed, "cpu"))
+    got, _ = run_tiles(again.tiles(), blobs, case.dst.buf_bytes)
+    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5)
+    assert all(np.array_equal(g, w) for g, w in zip(got, want))
+
+
+def test_plan_image_is_verified():
+    case = scenario_cases()[0]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    image = bytearray(plan.serialize())
+    for bad in (image[:-1], image[:40], b"", bytes(len(image))):
+        with pytest.raises(bcp.BcpError):
+            bcp.Plan.deserialize(bytes(bad))
+    flipped = bytearray(image)
+    flipped[len(flipped) // 2] ^= 0x40  # a corrupted unit: caught by the checksum
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.Plan.deserialize(bytes(flipped))
+    assert "checksum" in str(e.value)
 
 
 # ---- full-size configurations: planning is host-only, so their work lists are checked here ---------

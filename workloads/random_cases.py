@@ -80,3 +80,23 @@ def big_random_case(seed: int, *, itemsize: int = 2, gap_mod: int = 7) -> Reshar
     src = random_side(rng, tensors, 3, max_parts=4, gap_mod=gap_mod)
     dst = random_side(rng, tensors, 2, max_parts=3, gap_mod=gap_mod, replicas=2)
     return ReshardCase(f"big-random-{seed}-i{itemsize}", src, dst, "index", seed)
+
+
+def many_tiny_case(n_tensors: int = 100_000, seed: int = 7) -> ReshardCase:
+    """10^5 tiny tensors (4..512 bytes each, odd sizes), saved on 2 ranks and wanted on 3:
+    stresses FQN grouping in the planner and the one-warp-per-unit path of the kernel."""
+    rng = np.random.default_rng(seed)
+    sizes = rng.integers(1, 129, n_tensors)
+    isz = rng.choice([1, 2, 4], n_tensors)
+    src, dst = ShardedState([], [0, 0]), ShardedState([], [0, 0, 0])
+    for t in range(n_tensors):
+        n, w = int(sizes[t]), int(isz[t])
+        cut = int(rng.integers(0, n + 1))
+        name = f"tiny.{t}"
+        for st, parts in ((src, [(0, cut), (cut, n)]), (dst, [(0, n)])):
+            for a, b in parts:
+                if b > a:
+                    r = int(rng.integers(0, len(st.buf_bytes)))
+                    st.metas.append(ShardMeta(name, w, w, (n,), (a,), (b - a,), r, st.buf_bytes[r]))
+                    st.buf_bytes[r] += (b - a) * w
+    return ReshardCase(f"many-tiny-{n_tensors}", src, dst, "index", seed)
