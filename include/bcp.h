@@ -119,7 +119,9 @@ typedef struct {
   uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3                               */
   uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2 (4 with many shifted runs)     */
   uint32_t unroll;          /* register path: 16-byte loads in flight per thread, 4 or 8; default 4    */
-  uint32_t reserved[5];    /* must be 0 */
+  uint32_t worker;          /* register path: 0 default (= 1); 1 a CTA copies a unit together; 2 every warp
+                               is a worker of its own (256-thread CTAs, ctas_per_sm up to 8)           */
+  uint32_t reserved[4];    /* must be 0 */
 } bcp_plan_opts;
 
 typedef struct bcp_plan bcp_plan_t;

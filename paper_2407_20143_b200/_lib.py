@@ -41,7 +41,8 @@ class PlanOptsC(C.Structure):
         ("tma_stages", C.c_uint32),
         ("tma_ctas_per_sm", C.c_uint32),
         ("unroll", C.c_uint32),
-        ("reserved", C.c_uint32 * 5),
+        ("worker", C.c_uint32),
+        ("reserved", C.c_uint32 * 4),
     ]
 
 

@@ -25,6 +25,7 @@ struct bcp_plan {
   cudaStream_t last_stream = nullptr;
   bool ran = false;
   std::vector<void*> h_ptrs;
+  bool table_current = false;  // the device pointer table already holds h_ptrs
   // bcp_reshard_host: device staging plus a second copy of the work list grouped by target
   // buffer, so that uploads, kernels and downloads of different target buffers overlap
   struct Group {  // units of one target buffer inside d_host_tiles
@@ -56,7 +57,11 @@ int bind_device_alloc(bcp_plan_t* p) {
   BCP_CUDA(cudaMalloc(&p->d_ptrs, (n_ptrs ? n_ptrs : 1) * sizeof(void*)));
   BCP_CUDA(cudaMalloc(&p->d_ctrl, 2 * sizeof(Control)));
   BCP_CUDA(cudaMemset(p->d_ctrl, 0, 2 * sizeof(Control)));
-  BCP_CUDA(copy_kernel_max_grid(p->opt.block_threads, p->opt.ctas_per_sm, &p->grid));
+  if (p->opt.worker == 2) {
+    BCP_CUDA(warp_kernel_max_grid(p->opt.ctas_per_sm, &p->grid));
+  } else {
+    BCP_CUDA(copy_kernel_max_grid(p->opt.block_threads, p->opt.ctas_per_sm, &p->grid));
+  }
   if (p->n_tma)
     BCP_CUDA(tma_kernel_max_grid(p->opt.tma_stage_bytes, p->opt.tma_stages, p->opt.tma_ctas_per_sm, &p->tma_grid));
   p->h_ptrs.resize(n_ptrs);
@@ -110,9 +115,15 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
   a.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
   a.ctrl = p->d_ctrl;
   a.block_threads = p->opt.block_threads;
+  a.warp_workers = p->opt.worker == 2;
   const uint32_t nwarps = a.block_threads / 32;
-  const uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;
-  a.grid = uint32_t(units < p->grid ? units : p->grid);
+  uint64_t units = uint64_t(a.n_big) + (a.n_small + nwarps - 1) / nwarps;  // CTA-wide units + batches of warp units
+  uint64_t ctas = units;
+  if (a.warp_workers) {
+    units = uint64_t(a.n_big) + a.n_small;
+    ctas = (units + 7) / 8;  // 8 warps per CTA
+  }
+  a.grid = uint32_t(ctas < p->grid ? ctas : p->grid);
   a.cache_hints = p->opt.cache_hints;
   a.unroll = p->opt.unroll;
   if (units) BCP_CUDA(launch_copy(a, stream));
@@ -136,10 +147,19 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
     if (reinterpret_cast<uintptr_t>(dst[i]) & 15) return fail(BCP_ERR_INVALID, "target buffer %zu is not 16-byte aligned", i);
   if (int rc = bind_device(p)) return rc;
   if (p->tiles.empty()) return BCP_OK;
-  for (size_t i = 0; i < ns; ++i) p->h_ptrs[i] = const_cast<void*>(src[i]);
-  for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
-  // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
-  BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  // The device pointer table is refreshed only when a base address changed since the last
+  // execution (executions of a plan are ordered, so the previous upload has been consumed).
+  bool same = p->table_current;
+  for (size_t i = 0; same && i < ns; ++i) same = p->h_ptrs[i] == src[i];
+  for (size_t i = 0; same && i < nd; ++i) same = p->h_ptrs[ns + i] == dst[i];
+  if (!same) {
+    for (size_t i = 0; i < ns; ++i) p->h_ptrs[i] = const_cast<void*>(src[i]);
+    for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
+    // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
+    p->table_current = false;
+    BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+    p->table_current = true;
+  }
   if (int rc = launch_units(p, p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
   p->last_stream = stream;
   p->ran = true;
@@ -522,7 +542,7 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   {  // the options were validated when the plan was made; re-check what the launch code relies on
     const Options& o = h.opt;
     if ((o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024) || o.ctas_per_sm < 1 || o.ctas_per_sm > 16 ||
-        o.tile_bytes < 4096 || o.tile_bytes > (64u << 20) || (o.unroll != 4 && o.unroll != 8) || o.tma_stages < 2 || o.tma_stages > 8 ||
+        o.tile_bytes < 4096 || o.tile_bytes > (64u << 20) || (o.unroll != 4 && o.unroll != 8) || (o.worker != 1 && o.worker != 2) || o.tma_stages < 2 || o.tma_stages > 8 ||
         o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536 ||
         uint64_t(o.tma_stage_bytes) * o.tma_stages > 200 * 1024 || o.tma_ctas_per_sm < 1 || o.tma_ctas_per_sm > 16 || o.cache_hints < 1 ||
         o.cache_hints > 4)
@@ -591,6 +611,7 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
   // device-side pointer table: the staging buffers
   for (size_t i = 0; i < n_src_bufs; ++i) p->h_ptrs[i] = p->stage_src[i];
   for (size_t i = 0; i < n_dst_bufs; ++i) p->h_ptrs[n_src_bufs + i] = p->stage_dst[i];
+  p->table_current = false;  // the table now names the staging buffers
   BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (n_src_bufs + n_dst_bufs) * sizeof(void*), cudaMemcpyHostToDevice, stream));
   // The upload stream starts after whatever the caller queued on `stream` before this call.
   BCP_CUDA(cudaEventRecord(p->ev_dst[0], stream));

@@ -258,6 +258,44 @@ __global__ void __launch_bounds__(NT, 1024 / NT) bcp_copy_kernel(const bcp_tile*
   }
 }
 
+// ---------------------------------------------------------------- warp workers
+// The same work list with every warp as an independent worker: a warp draws a unit (CTA-wide
+// and small units alike), copies it alone with U x 512 bytes in flight, and moves on.  No
+// CTA-wide barrier, and the ticket and the record of the next unit are fetched while the
+// current unit is being copied, so the dependent chain ticket -> record -> base pointers ->
+// data never stalls the SM: 32 warps per SM are at different points of it.
+template <int U, int HINT>
+__global__ void __launch_bounds__(256, 4) bcp_copy_kernel_warps(const bcp_tile* __restrict__ tiles, uint32_t n_units,
+                                                                const void* const* __restrict__ src,
+                                                                void* const* __restrict__ dst, Control* ctrl) {
+  const uint32_t lane = threadIdx.x & 31;
+  uint32_t pending = 0;  // lane 0: ticket drawn but not yet used
+  if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
+  uint32_t u = __shfl_sync(0xffffffffu, pending, 0);
+  if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
+  bcp_tile t;
+  if (u < n_units) t = load_tile(tiles + u);
+  while (u < n_units) {
+    const uint32_t next = __shfl_sync(0xffffffffu, pending, 0);
+    if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);  // for the unit after the next
+    bcp_tile tn;
+    if (next < n_units) tn = load_tile(tiles + next);  // in flight while this unit is copied
+    copy_tile<U, HINT, 32>(t, src, dst, lane);
+    u = next;
+    t = tn;
+  }
+  // every warp has drawn tickets past the end; the last warp to leave rewinds the counters
+  if (lane == 0) {
+    __threadfence();
+    const uint32_t left = atomicAdd(&ctrl->done, 1u);
+    if (left == gridDim.x * (blockDim.x >> 5) - 1) {
+      ctrl->ticket = 0;
+      ctrl->done = 0;
+      __threadfence();
+    }
+  }
+}
+
 template <int NT, int HINT>
 cudaError_t launch_as(const LaunchArgs& a, cudaStream_t stream) {
   if (a.unroll == 8) {
@@ -270,6 +308,15 @@ cudaError_t launch_as(const LaunchArgs& a, cudaStream_t stream) {
 
 template <int HINT>
 cudaError_t launch_hint(const LaunchArgs& a, cudaStream_t stream) {
+  if (a.warp_workers) {
+    const uint32_t n_units = a.n_big + a.n_small;
+    if (a.unroll == 8) {
+      bcp_copy_kernel_warps<8, HINT><<<a.grid, 256, 0, stream>>>(a.tiles, n_units, a.src, a.dst, a.ctrl);
+    } else {
+      bcp_copy_kernel_warps<4, HINT><<<a.grid, 256, 0, stream>>>(a.tiles, n_units, a.src, a.dst, a.ctrl);
+    }
+    return cudaGetLastError();
+  }
   switch (a.block_threads) {
     case 256: return launch_as<256, HINT>(a, stream);
     case 512: return launch_as<512, HINT>(a, stream);
@@ -279,6 +326,20 @@ cudaError_t launch_hint(const LaunchArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+cudaError_t warp_kernel_max_grid(uint32_t ctas_per_sm, uint32_t* grid) {
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bcp_copy_kernel_warps<8, 1>, 256, 0);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) per_sm = 1;
+  const uint32_t k = ctas_per_sm < uint32_t(per_sm) ? ctas_per_sm : uint32_t(per_sm);
+  *grid = uint32_t(sms) * k;
+  return cudaSuccess;
+}
 
 cudaError_t copy_kernel_max_grid(uint32_t block_threads, uint32_t ctas_per_sm, uint32_t* grid) {
   int dev = 0, sms = 0, per_sm = 0;

@@ -29,6 +29,7 @@ struct LaunchArgs {
   uint32_t grid;
   uint32_t cache_hints;       // 1 streaming, 2 plain
   uint32_t unroll;            // 4 or 8
+  uint32_t warp_workers;      // 1: every warp is an independent worker (256-thread CTAs); 0: CTA-wide units
 };
 
 struct TmaLaunchArgs {
@@ -49,6 +50,9 @@ cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_
 
 // Enqueue the TMA staging kernel on `stream`.
 cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream);
+
+// Persistent grid of the warp-worker form of the copy kernel (256-thread CTAs).
+cudaError_t warp_kernel_max_grid(uint32_t ctas_per_sm, uint32_t* grid);
 
 // Largest useful persistent grid for the copy kernel on the current device.
 cudaError_t copy_kernel_max_grid(uint32_t block_threads, uint32_t ctas_per_sm, uint32_t* grid);

@@ -36,6 +36,7 @@ struct Options {
   uint32_t tma_stages = 3;
   uint32_t tma_ctas_per_sm = 0;
   uint32_t unroll = 4;
+  uint32_t worker = 1;
 };
 
 int parse_options(const bcp_plan_opts* in, Options* out);

@@ -48,6 +48,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->tma_stages) o.tma_stages = in->tma_stages;
     if (in->tma_ctas_per_sm) o.tma_ctas_per_sm = in->tma_ctas_per_sm;
     if (in->unroll) o.unroll = in->unroll;
+    if (in->worker) o.worker = in->worker;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -65,6 +66,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
+  if (o.worker != 1 && o.worker != 2) return fail(BCP_ERR_INVALID, "worker must be 1 or 2");
   *out = o;
   return BCP_OK;
 }

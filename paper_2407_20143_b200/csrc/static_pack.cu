@@ -187,6 +187,7 @@ extern "C" int bcp_pack_static(const void* const* tensors, const bcp_pack_meta* 
   a.block_threads = 512;
   a.cache_hints = 1;
   a.unroll = 4;
+  a.warp_workers = 0;
   uint32_t grid = 0;
   BCP_S_CUDA(copy_kernel_max_grid(a.block_threads, 2, &grid));
   const uint64_t units = uint64_t(a.n_big) + (a.n_small + 15) / 16;

@@ -84,7 +84,8 @@ def test_big_random_misaligned(cuda_device, itemsize, seed, path_mask):
 
 @pytest.mark.parametrize("opts", [dict(block_threads=256, ctas_per_sm=4), dict(block_threads=1024, ctas_per_sm=1),
                                   dict(tile_bytes=4096), dict(tile_bytes=1 << 20, small_bytes=1 << 16),
-                                  dict(cache_hints=2), dict(order=2), dict(unroll=8),
+                                  dict(cache_hints=2), dict(order=2), dict(unroll=8), dict(path_mask=1, worker=2),
+                                  dict(path_mask=1, worker=2, unroll=8, ctas_per_sm=4, tile_bytes=16384),
                                   dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=2, tile_bytes=32768),
                                   dict(path_mask=3, tma_stage_bytes=32768, tma_stages=6, tma_ctas_per_sm=1)])
 def test_launch_options(cuda_device, opts):
