@@ -102,7 +102,7 @@ typedef struct {
   uint32_t tile_bytes;     /* payload of one CTA-wide work unit; default 65536; multiple of 4096      */
   uint32_t small_bytes;    /* work units with a payload below this go to the warp path; default 4096  */
   uint32_t block_threads;  /* threads per CTA of the register kernel: 256, 512 or 1024; default 512     */
-  uint32_t ctas_per_sm;    /* persistent CTAs per SM; default 2                                       */
+  uint32_t ctas_per_sm;    /* register path: persistent CTAs per SM; default 2 (4 with worker 2)       */
   uint32_t order;          /* 0 default (= 1); 1 order work by source address (replica reads of one
                               source region run back to back and hit L2); 2 order by target address    */
   uint32_t path_mask;      /* 0 default: 3 when at least 128 MiB of payload qualifies for TMA staging, else 1
@@ -115,13 +115,16 @@ typedef struct {
   uint32_t cache_hints;    /* 0 default (= 1); register path: 1 streaming loads and stores, 2 plain accesses;
                               TMA path: 3 evict-first L2 hint on stores, 4 on loads too, else no hint    */
   uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage, multiple of 128; default 32768, or
-                               16384 when an eighth or more of the staged payload are shifted runs      */
+                               16384 when an eighth or more of the staged payload are shifted runs or
+                               rectangles with rows under 2 KiB                                        */
   uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3                               */
-  uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2 (4 with many shifted runs)     */
+  uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2 (4 in the same case)            */
   uint32_t unroll;          /* register path: 16-byte loads in flight per thread, 4 or 8; default 4    */
-  uint32_t worker;          /* register path: 0 default (= 1); 1 a CTA copies a unit together; 2 every warp
-                               is a worker of its own (256-thread CTAs, ctas_per_sm up to 8)           */
-  uint32_t reserved[4];    /* must be 0 */
+  uint32_t worker;          /* register path: 1 a CTA copies a unit together; 2 every warp is a worker of
+                               its own (256-thread CTAs); default 2 when this path has at least 128 MiB
+                               to move, else 1                                                          */
+  uint32_t tma_min_row_bytes; /* TMA path: shortest row (or run) staged through TMA; default 512; multiple of 16 */
+  uint32_t reserved[3];    /* must be 0 */
 } bcp_plan_opts;
 
 typedef struct bcp_plan bcp_plan_t;

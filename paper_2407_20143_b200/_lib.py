@@ -42,7 +42,8 @@ class PlanOptsC(C.Structure):
         ("tma_ctas_per_sm", C.c_uint32),
         ("unroll", C.c_uint32),
         ("worker", C.c_uint32),
-        ("reserved", C.c_uint32 * 4),
+        ("tma_min_row_bytes", C.c_uint32),
+        ("reserved", C.c_uint32 * 3),
     ]
 
 

@@ -28,7 +28,7 @@ struct Options {
   uint32_t tile_bytes = 65536;
   uint32_t small_bytes = 4096;
   uint32_t block_threads = 512;
-  uint32_t ctas_per_sm = 2;
+  uint32_t ctas_per_sm = 0;  // 0: chosen from the work list
   uint32_t order = 1;
   uint32_t path_mask = 0;  // 0: decided from the work list
   uint32_t cache_hints = 1;
@@ -36,7 +36,8 @@ struct Options {
   uint32_t tma_stages = 3;
   uint32_t tma_ctas_per_sm = 0;
   uint32_t unroll = 4;
-  uint32_t worker = 1;
+  uint32_t worker = 0;  // 0: chosen from the work list
+  uint32_t tma_min_row_bytes = 512;
 };
 
 int parse_options(const bcp_plan_opts* in, Options* out);

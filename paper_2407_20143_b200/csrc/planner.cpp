@@ -49,13 +49,14 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->tma_ctas_per_sm) o.tma_ctas_per_sm = in->tma_ctas_per_sm;
     if (in->unroll) o.unroll = in->unroll;
     if (in->worker) o.worker = in->worker;
+    if (in->tma_min_row_bytes) o.tma_min_row_bytes = in->tma_min_row_bytes;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
   if (o.small_bytes > o.tile_bytes) return fail(BCP_ERR_INVALID, "small_bytes must not exceed tile_bytes");
   if (o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024)
     return fail(BCP_ERR_INVALID, "block_threads must be 256, 512 or 1024");
-  if (o.ctas_per_sm < 1 || o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
+  if (o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
   if (o.order < 1 || o.order > 2) return fail(BCP_ERR_INVALID, "order must be 1 or 2");
   if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3) return fail(BCP_ERR_INVALID, "path_mask must be 0, 1 or 3");
   if (o.tma_stage_bytes && (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536))
@@ -66,7 +67,9 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
-  if (o.worker != 1 && o.worker != 2) return fail(BCP_ERR_INVALID, "worker must be 1 or 2");
+  if (o.worker > 2) return fail(BCP_ERR_INVALID, "worker must be 0, 1 or 2");
+  if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
+    return fail(BCP_ERR_INVALID, "tma_min_row_bytes must be a multiple of 16 in [16, 65536]");
   *out = o;
   return BCP_OK;
 }
@@ -497,7 +500,7 @@ struct Cutter {
     } else {
       // TMA staging: whole 16-byte units between 16-byte aligned addresses (runs and rectangles),
       // or a run of any alignment whose 16-byte aligned superset stays inside the source buffer
-      bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= 512;
+      bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= opt.tma_min_row_bytes;
       if (eligible && g < 4) {
         const uint64_t end16 = (src_off + row_bytes + 15) & ~uint64_t(15);
         eligible = rows == 1 && src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
@@ -604,21 +607,32 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   auto by_dst = [](const bcp_tile& a, const bcp_tile& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
   };
-  // Stage geometry of the TMA kernel when the caller left it open.  Aligned units only issue
-  // copy commands, so few CTAs with large stages are enough (2 x 3 x 32 KiB per SM); shifted
-  // runs are copied out of shared memory by the warp itself and want more warps per SM
-  // (4 x 3 x 16 KiB).  Both fill 192 KiB of shared memory per SM.
+  // Stage geometry of the TMA kernel when the caller left it open.  Long aligned runs only need
+  // a few copy commands per stage, so two CTAs with 32 KiB stages per SM are enough; shifted
+  // runs (copied out of shared memory by the warp itself) and rectangles with rows under 2 KiB
+  // (one copy command per row) are limited by what one warp can issue and want four CTAs with
+  // 16 KiB stages.  Both fill 192 KiB of shared memory per SM.
   {
-    uint64_t total = 0, shifted = 0;
+    uint64_t total = 0, busy = 0;
     for (const bcp_tile& t : c.tma) {
       const uint64_t n = uint64_t(t.rows) * t.row_bytes;
       total += n;
-      if ((t.flags & BCP_TILE_GRAN_MASK) < 4) shifted += n;
+      if ((t.flags & BCP_TILE_GRAN_MASK) < 4 || (t.rows > 1 && t.row_bytes < 2048)) busy += n;
     }
-    const bool many_shifted = shifted * 8 >= total && total > 0;
-    if (!opt.tma_stage_bytes) opt.tma_stage_bytes = many_shifted ? 16384 : 32768;
-    if (!opt.tma_ctas_per_sm) opt.tma_ctas_per_sm = many_shifted ? 4 : 2;
+    const bool many_busy = busy * 8 >= total && total > 0;
+    if (!opt.tma_stage_bytes) opt.tma_stage_bytes = many_busy ? 16384 : 32768;
+    if (!opt.tma_ctas_per_sm) opt.tma_ctas_per_sm = many_busy ? 4 : 2;
   }
+  // Register kernel: a CTA per unit for small jobs (fewer, fatter workers start faster); every
+  // warp its own worker once the kernel has a lot to move (no barriers, deeper overlap).
+  if (!opt.worker) {
+    uint64_t reg_bytes = 0;
+    for (const bcp_tile& t : c.big) reg_bytes += uint64_t(t.rows) * t.row_bytes;
+    for (const bcp_tile& t : c.small) reg_bytes += uint64_t(t.rows) * t.row_bytes;
+    opt.worker = reg_bytes >= (128u << 20) ? 2 : 1;
+    if (opt.worker == 2 && !opt.ctas_per_sm) opt.ctas_per_sm = 4;
+  }
+  if (!opt.ctas_per_sm) opt.ctas_per_sm = 2;
   for (std::vector<bcp_tile>* v : {&c.tma, &c.big, &c.small}) {
     if (opt.order == 1) {
       std::sort(v->begin(), v->end(), by_src);

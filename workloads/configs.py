@@ -65,7 +65,18 @@ def cfg4_odd(layers: int = 28) -> ReshardCase:
                         OPTIM_ONLY, "index", seed=20149)
 
 
-STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd}
+def narrow_rows(layers: int = 4, cols: int = 256) -> ReshardCase:
+    """Unscored stress: `layers` bf16 tensors of shape (2^28 / cols, cols) split along dim 1, two
+    ways saved and four ways wanted, so every copy is a rectangle with rows of cols / 2 bytes
+    (128 bytes by default) and 512 MB per tensor."""
+    from .layouts import ModelSpec, TensorSpec
+
+    m = ModelSpec("narrow", [TensorSpec(f"t{i}.weight", ((1 << 28) // cols, cols), "row", layer=i) for i in range(layers)], layers)
+    return reshard_case(f"narrow-rows-{cols // 2}B-x{layers}", m, Parallelism(tp=2), Parallelism(tp=4), PARAMS_ONLY, "index",
+                        seed=20150)
+
+
+STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows}
 
 CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
     "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
