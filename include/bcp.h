@@ -105,19 +105,24 @@ typedef struct {
   uint32_t ctas_per_sm;    /* register path: persistent CTAs per SM; default 2 (4 with worker 2)       */
   uint32_t order;          /* 0 default (= 1); 1 order work by source address (replica reads of one
                               source region run back to back and hit L2); 2 order by target address    */
-  uint32_t path_mask;      /* 0 default: 3 when at least 128 MiB of payload qualifies for TMA staging, else 1
-                              (small jobs are launch-bound and one kernel is cheaper than two);
+  uint32_t path_mask;      /* which kernels execute the list.
                               1 every unit goes through registers (LDG/STG kernel);
-                              3 runs of at least 512 bytes (any alignment) and rectangles with rows of at
-                              least 512 bytes whose offsets, row length and pitches are multiples of 16
-                              go through the TMA staging kernel (bulk copies via shared memory), the
-                              rest through the register kernel                                          */
+                              3 runs of at least tma_min_row_bytes (any alignment) and rectangles with rows of
+                                at least that size whose offsets, row length and pitches are multiples of 16
+                                go through the TMA staging kernel (bulk copies via shared memory), the rest
+                                through the register kernel;
+                              7 as 3, and 16-byte aligned rectangles with rows of 16..2048 bytes are staged
+                                with 2-D tensor-map copies (cp.async.bulk.tensor.2d, one command per box of
+                                up to 256 rows) instead of one bulk copy per row; their descriptors are
+                                re-encoded on the host whenever a buffer address changes;
+                              0 default: 7 when at least 128 MiB of payload qualifies for TMA staging, else 1
+                                (small jobs are launch-bound and one kernel is cheaper than two)            */
   uint32_t cache_hints;    /* 0 default (= 1); register path: 1 streaming loads and stores, 2 plain accesses;
                               TMA path: 3 evict-first L2 hint on stores, 4 on loads too, else no hint    */
   uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage, multiple of 128; default 32768, or
                                16384 when an eighth or more of the staged payload are shifted runs or
                                rectangles with rows under 2 KiB                                        */
-  uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3                               */
+  uint32_t tma_stages;      /* TMA path: stages per CTA, 2..8; default 3 (4 when tensor-map boxes dominate) */
   uint32_t tma_ctas_per_sm; /* TMA path: one-warp CTAs per SM; default 2 (4 in the same case)            */
   uint32_t unroll;          /* register path: 16-byte loads in flight per thread, 4 or 8; default 4    */
   uint32_t worker;          /* register path: 1 a CTA copies a unit together; 2 every warp is a worker of
@@ -152,6 +157,9 @@ typedef struct {
 #define BCP_TILE_ZERO 0x8u      /* no source: write zero bytes (pack padding)                    */
 #define BCP_TILE_SMALL 0x10u    /* executed by one warp                                          */
 #define BCP_TILE_TMA 0x20u      /* eligible for the TMA staging path                             */
+#define BCP_TILE_TMA2D 0x40u    /* rows of a rectangle staged with 2-D tensor-map copies: reserved[0] =
+                                   rectangle index + 1, reserved[1] = first row inside the rectangle,
+                                   reserved[2] = rows per box                                    */
 
 typedef struct {
   uint64_t n_src_entries;    /* after decomposing flat slices                        */

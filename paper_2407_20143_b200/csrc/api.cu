@@ -5,6 +5,8 @@
 #include <new>
 #include <vector>
 
+#include <cuda.h>
+
 #include "kernels.cuh"
 #include "plan.hpp"
 
@@ -16,6 +18,9 @@ struct bcp_plan {
   std::vector<bcp_tile> tiles;  // TMA units, then other CTA-wide units, then warp units
   size_t n_tma = 0, n_big = 0;
   std::vector<uint64_t> src_bytes, dst_bytes;
+  std::vector<Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
+  std::vector<CUtensorMap> h_maps;
+  CUtensorMap* d_maps = nullptr;
   // device side, created by the first execution
   int device = -1;
   bcp_tile* d_tiles = nullptr;
@@ -55,6 +60,10 @@ int bind_device_alloc(bcp_plan_t* p) {
     BCP_CUDA(cudaMemcpy(p->d_tiles, p->tiles.data(), p->tiles.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
   }
   BCP_CUDA(cudaMalloc(&p->d_ptrs, (n_ptrs ? n_ptrs : 1) * sizeof(void*)));
+  if (!p->rects.empty()) {
+    BCP_CUDA(cudaMalloc(&p->d_maps, p->rects.size() * 2 * sizeof(CUtensorMap)));
+    p->h_maps.resize(p->rects.size() * 2);
+  }
   BCP_CUDA(cudaMalloc(&p->d_ctrl, 2 * sizeof(Control)));
   BCP_CUDA(cudaMemset(p->d_ctrl, 0, 2 * sizeof(Control)));
   if (p->opt.worker == 2) {
@@ -80,6 +89,8 @@ int bind_device(bcp_plan_t* p) {
     cudaFree(p->d_tiles);
     cudaFree(p->d_ptrs);
     cudaFree(p->d_ctrl);
+    cudaFree(p->d_maps);
+    p->d_maps = nullptr;
     p->d_tiles = nullptr;
     p->d_ptrs = nullptr;
     p->d_ctrl = nullptr;
@@ -87,6 +98,59 @@ int bind_device(bcp_plan_t* p) {
     return rc;
   }
   p->device = dev;
+  return BCP_OK;
+}
+
+// Tensor maps are encoded by the driver; the entry point is looked up once (no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+int encode_fn(EncodeTiledFn* out) {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    BCP_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q));
+    if (q != cudaDriverEntryPointSuccess || !sym) return fail(BCP_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  *out = fn;
+  return BCP_OK;
+}
+
+// One view of a rectangle: `rows` rows of row_bytes bytes, `pitch` apart, as a 2-D tensor of
+// 8-byte elements; a box is the whole row width times box_rows rows.
+int encode_view(EncodeTiledFn fn, CUtensorMap* map, void* base, const Rect& r, uint64_t pitch) {
+  if (reinterpret_cast<uintptr_t>(base) & 15) return fail(BCP_ERR_INVALID, "rectangle base address is not 16-byte aligned");
+  const cuuint64_t dims[2] = {r.row_bytes / 8, r.rows};
+  const cuuint64_t strides[1] = {pitch};
+  const cuuint32_t box[2] = {r.row_bytes / 8, r.box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return fail(BCP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", int(rc));
+  return BCP_OK;
+}
+
+// Upload the pointer table in h_ptrs and, for tensor-map rectangles, descriptors for those addresses.
+int upload_tables(bcp_plan_t* p, cudaStream_t stream) {
+  const size_t ns = p->src_bytes.size(), nd = p->dst_bytes.size();
+  p->table_current = false;
+  if (!p->rects.empty()) {
+    EncodeTiledFn fn;
+    if (int rc = encode_fn(&fn)) return rc;
+    for (size_t i = 0; i < p->rects.size(); ++i) {
+      const Rect& r = p->rects[i];
+      char* sb = static_cast<char*>(p->h_ptrs[r.src_buf]) + r.src_off;
+      char* db = static_cast<char*>(p->h_ptrs[ns + r.dst_buf]) + r.dst_off;
+      if (int rc = encode_view(fn, &p->h_maps[2 * i], sb, r, r.src_pitch)) return rc;
+      if (int rc = encode_view(fn, &p->h_maps[2 * i + 1], db, r, r.dst_pitch)) return rc;
+    }
+    BCP_CUDA(cudaMemcpyAsync(p->d_maps, p->h_maps.data(), p->h_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, stream));
+  }
+  // pageable sources: the runtime stages them before returning, so the host copies may be reused
+  BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  p->table_current = true;
   return BCP_OK;
 }
 
@@ -103,8 +167,9 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
     t.stage_bytes = p->opt.tma_stage_bytes;
     t.n_stages = p->opt.tma_stages;
     t.grid = uint32_t(n_tma < p->tma_grid ? n_tma : p->tma_grid);
-    t.wait_limit = 1u << 22;
+    t.wait_limit = 1u << 20;
     t.cache_hints = p->opt.cache_hints;
+    t.maps = p->d_maps;
     BCP_CUDA(launch_tma(t, stream));
   }
   LaunchArgs a;
@@ -155,10 +220,7 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
   if (!same) {
     for (size_t i = 0; i < ns; ++i) p->h_ptrs[i] = const_cast<void*>(src[i]);
     for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
-    // pageable source: the runtime stages the table before returning, so h_ptrs may be reused
-    p->table_current = false;
-    BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (ns + nd) * sizeof(void*), cudaMemcpyHostToDevice, stream));
-    p->table_current = true;
+    if (int rc = upload_tables(p, stream)) return rc;
   }
   if (int rc = launch_units(p, p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
   p->last_stream = stream;
@@ -174,7 +236,7 @@ bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_s
   p->stats = stats;
   p->src_bytes = std::move(src_bytes);
   p->dst_bytes = std::move(dst_bytes);
-  build_tiles(items, p->opt, &p->src_bytes, &p->tiles, &p->n_tma, &p->n_big, &p->stats);
+  build_tiles(items, p->opt, &p->src_bytes, &p->tiles, &p->n_tma, &p->n_big, &p->rects, &p->stats);
   return p;
 }
 
@@ -455,7 +517,7 @@ struct ImageHeader {
   uint32_t version, tile_size;
   Options opt;
   bcp_plan_stats_t stats;
-  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles;
+  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects;
 };
 uint64_t fnv1a(const unsigned char* p, size_t n) {
   uint64_t h = 1469598103934665603ull;
@@ -463,7 +525,8 @@ uint64_t fnv1a(const unsigned char* p, size_t n) {
   return h;
 }
 // A unit is safe to execute if it stays inside its buffers and its flags match its geometry.
-bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db, const Options& opt) {
+bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db, const std::vector<Rect>& rects,
+             const Options& opt) {
   if (t.rows == 0 || t.row_bytes == 0 || t.dst_buf >= db.size()) return false;
   const bool zero = t.flags & BCP_TILE_ZERO;
   const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes;
@@ -479,6 +542,18 @@ bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vect
   uint32_t g = 0;
   while (g < 4 && !((bits >> g) & 1)) ++g;
   if ((t.flags & BCP_TILE_GRAN_MASK) > g) return false;  // a wider access than the offsets allow would fault
+  if (t.flags & BCP_TILE_TMA2D) {  // must be a whole number of boxes of the rectangle it names
+    if (!(t.flags & BCP_TILE_TMA) || zero || g < 4 || t.reserved[0] == 0 || t.reserved[0] > rects.size()) return false;
+    const Rect& r = rects[t.reserved[0] - 1];
+    const uint64_t row0 = t.reserved[1];
+    if (t.reserved[2] != r.box_rows || r.box_rows == 0 || row0 % r.box_rows || row0 + t.rows > r.rows) return false;
+    if (t.rows % r.box_rows && row0 + t.rows != r.rows) return false;
+    if (t.src_buf != r.src_buf || t.dst_buf != r.dst_buf || t.row_bytes != r.row_bytes || t.src_pitch != r.src_pitch ||
+        t.dst_pitch != r.dst_pitch || t.src_off != r.src_off + row0 * r.src_pitch || t.dst_off != r.dst_off + row0 * r.dst_pitch)
+      return false;
+    if (uint64_t(r.box_rows) * r.row_bytes > opt.tma_stage_bytes) return false;
+    return uint64_t(t.rows) * t.row_bytes <= std::max<uint64_t>(opt.tile_bytes, uint64_t(r.box_rows) * r.row_bytes);
+  }
   if (t.flags & BCP_TILE_TMA) {
     if (zero || t.row_bytes < 16) return false;
     if (g < 4) {  // shifted run: one row, aligned superset inside the source buffer
@@ -488,12 +563,22 @@ bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vect
   }
   return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
 }
+// A rectangle's two views must stay inside their buffers and satisfy the tensor-map rules.
+bool rect_ok(const Rect& r, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db) {
+  if (r.src_buf >= sb.size() || r.dst_buf >= db.size() || r.rows == 0 || r.rows >= (uint64_t(1) << 31)) return false;
+  if (r.row_bytes < 16 || r.row_bytes > 2048 || r.box_rows == 0 || r.box_rows > 256) return false;
+  if ((r.src_off | r.dst_off | r.row_bytes | r.src_pitch | r.dst_pitch) & 15) return false;
+  if (r.src_pitch < r.row_bytes || r.dst_pitch < r.row_bytes || r.src_pitch >= (uint64_t(1) << 40) || r.dst_pitch >= (uint64_t(1) << 40))
+    return false;
+  const uint64_t ss = (r.rows - 1) * r.src_pitch + r.row_bytes, ds = (r.rows - 1) * r.dst_pitch + r.row_bytes;
+  return r.src_off <= sb[r.src_buf] && ss <= sb[r.src_buf] - r.src_off && r.dst_off <= db[r.dst_buf] && ds <= db[r.dst_buf] - r.dst_off;
+}
 }  // namespace
 
 int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n) {
   if (!plan || !n) return fail(BCP_ERR_INVALID, "bcp_plan_serialize: NULL argument");
   const size_t need = sizeof(ImageHeader) + (plan->src_bytes.size() + plan->dst_bytes.size()) * sizeof(uint64_t) +
-                      plan->tiles.size() * sizeof(bcp_tile) + sizeof(uint64_t);
+                      plan->tiles.size() * sizeof(bcp_tile) + plan->rects.size() * sizeof(Rect) + sizeof(uint64_t);
   *n = need;
   if (!out || cap < need) return fail(BCP_ERR_CAPACITY, "bcp_plan_serialize: image needs %zu bytes, room for %zu", need, out ? cap : size_t(0));
   ImageHeader h;
@@ -508,6 +593,7 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   h.n_tma = plan->n_tma;
   h.n_big = plan->n_big;
   h.n_tiles = plan->tiles.size();
+  h.n_rects = plan->rects.size();
   unsigned char* p = static_cast<unsigned char*>(out);
   memcpy(p, &h, sizeof h);
   p += sizeof h;
@@ -517,6 +603,8 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   p += h.n_dst_bufs * sizeof(uint64_t);
   if (h.n_tiles) memcpy(p, plan->tiles.data(), h.n_tiles * sizeof(bcp_tile));
   p += h.n_tiles * sizeof(bcp_tile);
+  if (h.n_rects) memcpy(p, plan->rects.data(), h.n_rects * sizeof(Rect));
+  p += h.n_rects * sizeof(Rect);
   const uint64_t sum = fnv1a(static_cast<unsigned char*>(out), size_t(p - static_cast<unsigned char*>(out)));
   memcpy(p, &sum, sizeof sum);
   return BCP_OK;
@@ -531,9 +619,11 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   if (h.version != uint32_t(bcp_version()) || h.tile_size != sizeof(bcp_tile))
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image of library version %u, this is %d", h.version, bcp_version());
   const uint64_t lim = uint64_t(1) << 32;
-  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_tma > h.n_tiles || h.n_big > h.n_tiles - h.n_tma)
+  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_rects >= lim || h.n_tma > h.n_tiles ||
+      h.n_big > h.n_tiles - h.n_tma)
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: implausible counts");
-  const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) + sizeof(uint64_t);
+  const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) +
+                        h.n_rects * sizeof(Rect) + sizeof(uint64_t);
   if (need != n) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image is %zu bytes, its header implies %llu", n, (unsigned long long)need);
   const unsigned char* base = static_cast<const unsigned char*>(image);
   uint64_t sum;
@@ -562,16 +652,25 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
     if (h.n_dst_bufs) memcpy(p->dst_bytes.data(), q, h.n_dst_bufs * sizeof(uint64_t));
     q += h.n_dst_bufs * sizeof(uint64_t);
     if (h.n_tiles) memcpy(p->tiles.data(), q, h.n_tiles * sizeof(bcp_tile));
+    q += h.n_tiles * sizeof(bcp_tile);
+    p->rects.resize(h.n_rects);
+    if (h.n_rects) memcpy(p->rects.data(), q, h.n_rects * sizeof(Rect));
     p->n_tma = h.n_tma;
     p->n_big = h.n_big;
   } catch (const std::bad_alloc&) {
     delete p;
     return fail(BCP_ERR_NOMEM, "out of host memory");
   }
+  for (size_t i = 0; i < p->rects.size(); ++i) {
+    if (!rect_ok(p->rects[i], p->src_bytes, p->dst_bytes)) {
+      delete p;
+      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: rectangle %zu is inconsistent with the recorded buffers", i);
+    }
+  }
   for (size_t i = 0; i < p->tiles.size(); ++i) {
     const bcp_tile& t = p->tiles[i];
     const bool in_tma = i < p->n_tma, in_small = i >= p->n_tma + p->n_big;
-    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
+    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->rects, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
         bool(t.flags & BCP_TILE_SMALL) != in_small) {
       delete p;
       return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: work unit %zu is inconsistent with the recorded buffers", i);
@@ -611,8 +710,8 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
   // device-side pointer table: the staging buffers
   for (size_t i = 0; i < n_src_bufs; ++i) p->h_ptrs[i] = p->stage_src[i];
   for (size_t i = 0; i < n_dst_bufs; ++i) p->h_ptrs[n_src_bufs + i] = p->stage_dst[i];
-  p->table_current = false;  // the table now names the staging buffers
-  BCP_CUDA(cudaMemcpyAsync(p->d_ptrs, p->h_ptrs.data(), (n_src_bufs + n_dst_bufs) * sizeof(void*), cudaMemcpyHostToDevice, stream));
+  if (int rc = upload_tables(p, stream)) return rc;
+  p->table_current = false;  // the tables now name the staging buffers, not a caller's
   // The upload stream starts after whatever the caller queued on `stream` before this call.
   BCP_CUDA(cudaEventRecord(p->ev_dst[0], stream));
   BCP_CUDA(cudaStreamWaitEvent(p->s_h2d, p->ev_dst[0], 0));
@@ -684,6 +783,7 @@ int bcp_plan_destroy(bcp_plan_t* plan) {
     cudaFree(plan->d_tiles);
     cudaFree(plan->d_ptrs);
     cudaFree(plan->d_ctrl);
+    cudaFree(plan->d_maps);
     if (cudaGetLastError() != cudaSuccess) rc = fail(BCP_ERR_CUDA, "bcp_plan_destroy: a CUDA call failed");
     if (cur != plan->device) cudaSetDevice(cur);
   }

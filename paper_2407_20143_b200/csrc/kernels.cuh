@@ -43,6 +43,7 @@ struct TmaLaunchArgs {
   uint32_t grid;
   uint32_t wait_limit;    // mbarrier polls before a CTA gives up
   uint32_t cache_hints;   // 3: evict-first stores; 4: evict-first loads too; else none
+  const void* maps;       // device: two 128-byte tensor maps (source view, target view) per tensor-map rectangle
 };
 
 // Persistent grid of the TMA staging kernel (one warp per CTA) for a stage geometry.

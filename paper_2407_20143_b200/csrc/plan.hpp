@@ -33,11 +33,18 @@ struct Options {
   uint32_t path_mask = 0;  // 0: decided from the work list
   uint32_t cache_hints = 1;
   uint32_t tma_stage_bytes = 0;  // 0: chosen from the work list (see build_tiles)
-  uint32_t tma_stages = 3;
+  uint32_t tma_stages = 0;
   uint32_t tma_ctas_per_sm = 0;
   uint32_t unroll = 4;
   uint32_t worker = 0;  // 0: chosen from the work list
   uint32_t tma_min_row_bytes = 512;
+};
+
+// A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source
+// view, target view) depend on buffer addresses and are encoded when the plan is executed.
+struct Rect {
+  uint64_t src_off, dst_off, src_pitch, dst_pitch, rows;
+  uint32_t row_bytes, src_buf, dst_buf, box_rows;
 };
 
 int parse_options(const bcp_plan_opts* in, Options* out);
@@ -59,6 +66,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
 // tiles = [TMA units..., other CTA-wide units..., warp units...].
 // src_bytes: sizes of the source buffers (bounds for over-reading aligned supersets).
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
-                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, bcp_plan_stats_t* stats);
+                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,
+                 bcp_plan_stats_t* stats);
 
 }  // namespace bcp

@@ -58,11 +58,12 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     return fail(BCP_ERR_INVALID, "block_threads must be 256, 512 or 1024");
   if (o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
   if (o.order < 1 || o.order > 2) return fail(BCP_ERR_INVALID, "order must be 1 or 2");
-  if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3) return fail(BCP_ERR_INVALID, "path_mask must be 0, 1 or 3");
+  if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3 && o.path_mask != 7)
+    return fail(BCP_ERR_INVALID, "path_mask must be 0, 1, 3 or 7");
   if (o.tma_stage_bytes && (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536))
     return fail(BCP_ERR_INVALID, "tma_stage_bytes must be a multiple of 128 in [1024, 65536]");
-  if (o.tma_stages < 2 || o.tma_stages > 8) return fail(BCP_ERR_INVALID, "tma_stages must be in [2, 8]");
-  if (uint64_t(o.tma_stage_bytes ? o.tma_stage_bytes : 32768) * o.tma_stages > 200 * 1024)
+  if (o.tma_stages && (o.tma_stages < 2 || o.tma_stages > 8)) return fail(BCP_ERR_INVALID, "tma_stages must be in [2, 8]");
+  if (uint64_t(o.tma_stage_bytes ? o.tma_stage_bytes : 32768) * (o.tma_stages ? o.tma_stages : 4) > 200 * 1024)
     return fail(BCP_ERR_INVALID, "tma_stage_bytes * tma_stages must not exceed 200 KiB");
   if (o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
@@ -470,6 +471,7 @@ struct Cutter {
   const Options& opt;
   const std::vector<uint64_t>* src_bytes;  // source buffer sizes (may be null: unknown)
   std::vector<bcp_tile> tma, big, small;
+  std::vector<Rect> rects;
   bcp_plan_stats_t* st;
 
   void emit(const Item& it, uint64_t src_off, uint64_t dst_off, uint64_t rows, uint64_t row_bytes) {
@@ -542,11 +544,50 @@ struct Cutter {
     }
   }
 
+  // Rectangle with short rows -> units made of whole boxes of a 2-D tensor map (8-byte elements,
+  // one box = all of a row x box_rows rows, at most 16 KiB).  Returns false if it does not qualify.
+  bool cut_rect(const Item& it) {
+    if ((opt.path_mask != 7 && opt.path_mask != 0) || it.zero || it.row_bytes < 16 || it.row_bytes > 2048 || it.rows >= (uint64_t(1) << 31)) return false;
+    if ((it.src_off | it.dst_off | it.row_bytes | it.src_pitch | it.dst_pitch) & 15) return false;
+    if (it.src_pitch >= (uint64_t(1) << 40) || it.dst_pitch >= (uint64_t(1) << 40)) return false;
+    if (it.rows * it.row_bytes < 32768) return false;  // not worth two descriptors
+    uint64_t cap = std::min<uint64_t>(16384, opt.tile_bytes);
+    if (opt.tma_stage_bytes) cap = std::min<uint64_t>(cap, opt.tma_stage_bytes);
+    const uint64_t box_rows = std::min<uint64_t>(256, cap / it.row_bytes);
+    if (box_rows == 0) return false;
+    const uint64_t rpt = std::max<uint64_t>(box_rows, opt.tile_bytes / it.row_bytes / box_rows * box_rows);
+    Rect rc;
+    rc.src_off = it.src_off, rc.dst_off = it.dst_off, rc.src_pitch = it.src_pitch, rc.dst_pitch = it.dst_pitch;
+    rc.rows = it.rows, rc.row_bytes = uint32_t(it.row_bytes), rc.src_buf = it.src_buf, rc.dst_buf = it.dst_buf;
+    rc.box_rows = uint32_t(box_rows);
+    rects.push_back(rc);
+    for (uint64_t r = 0; r < it.rows; r += rpt) {
+      const uint64_t nr = std::min(rpt, it.rows - r);
+      bcp_tile t;
+      memset(&t, 0, sizeof t);
+      t.src_off = it.src_off + r * it.src_pitch;
+      t.dst_off = it.dst_off + r * it.dst_pitch;
+      t.src_pitch = it.src_pitch, t.dst_pitch = it.dst_pitch;
+      t.rows = uint32_t(nr), t.row_bytes = uint32_t(it.row_bytes);
+      t.src_buf = it.src_buf, t.dst_buf = it.dst_buf;
+      t.flags = 4u | BCP_TILE_TMA | BCP_TILE_TMA2D;
+      t.reserved[0] = uint32_t(rects.size());  // index + 1
+      t.reserved[1] = uint32_t(r);
+      t.reserved[2] = uint32_t(box_rows);
+      ++st->n_strided_tiles;
+      ++st->n_tma_tiles;
+      st->bytes_copied += nr * it.row_bytes;
+      tma.push_back(t);
+    }
+    return true;
+  }
+
   void cut(const Item& it) {
     if (it.rows <= 1 || it.row_bytes == 0) {
       cut_run(it, it.src_off, it.dst_off, it.rows ? it.row_bytes : 0);
       return;
     }
+    if (cut_rect(it)) return;
     if (it.row_bytes >= opt.tile_bytes) {  // long rows: each row is a run of its own
       for (uint64_t r = 0; r < it.rows; ++r) cut_run(it, it.src_off + r * it.src_pitch, it.dst_off + r * it.dst_pitch, it.row_bytes);
       return;
@@ -562,7 +603,8 @@ struct Cutter {
 }  // namespace
 
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
-                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, bcp_plan_stats_t* stats) {
+                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,
+                 bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
@@ -587,13 +629,17 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   stats->bytes_misaligned = 0;
   stats->n_strided_tiles = 0;
   stats->n_tma_tiles = 0;
-  Cutter c{opt, src_bytes, {}, {}, {}, stats};
+  Cutter c{opt, src_bytes, {}, {}, {}, {}, stats};
   for (const Item& it : merged) c.cut(it);
   if (opt.path_mask == 0) {  // small jobs are launch-bound: keep them in one kernel
     uint64_t eligible = 0;
     for (const bcp_tile& t : c.tma) eligible += uint64_t(t.rows) * t.row_bytes;
     if (eligible < (128u << 20)) {
-      for (bcp_tile& t : c.tma) t.flags &= ~BCP_TILE_TMA;
+      for (bcp_tile& t : c.tma) {
+        t.flags &= ~(BCP_TILE_TMA | BCP_TILE_TMA2D);
+        t.reserved[0] = t.reserved[1] = t.reserved[2] = 0;
+      }
+      c.rects.clear();
       c.big.insert(c.big.end(), c.tma.begin(), c.tma.end());
       c.tma.clear();
       stats->n_tma_tiles = 0;
@@ -613,15 +659,21 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   // (one copy command per row) are limited by what one warp can issue and want four CTAs with
   // 16 KiB stages.  Both fill 192 KiB of shared memory per SM.
   {
-    uint64_t total = 0, busy = 0;
+    uint64_t total = 0, busy = 0, boxed = 0;
     for (const bcp_tile& t : c.tma) {
       const uint64_t n = uint64_t(t.rows) * t.row_bytes;
       total += n;
-      if ((t.flags & BCP_TILE_GRAN_MASK) < 4 || (t.rows > 1 && t.row_bytes < 2048)) busy += n;
+      if (t.flags & BCP_TILE_TMA2D) {
+        boxed += n;
+      } else if ((t.flags & BCP_TILE_GRAN_MASK) < 4 || (t.rows > 1 && t.row_bytes < 2048)) {
+        busy += n;
+      }
     }
     const bool many_busy = busy * 8 >= total && total > 0;
-    if (!opt.tma_stage_bytes) opt.tma_stage_bytes = many_busy ? 16384 : 32768;
+    const bool many_boxed = !many_busy && boxed * 8 >= total && total > 0;  // boxes are at most 16 KiB: deeper ring
+    if (!opt.tma_stage_bytes) opt.tma_stage_bytes = (many_busy || many_boxed) ? 16384 : 32768;
     if (!opt.tma_ctas_per_sm) opt.tma_ctas_per_sm = many_busy ? 4 : 2;
+    if (!opt.tma_stages) opt.tma_stages = many_boxed ? 4 : 3;
   }
   // Register kernel: a CTA per unit for small jobs (fewer, fatter workers start faster); every
   // warp its own worker once the kernel has a lot to move (no barriers, deeper overlap).
@@ -644,6 +696,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   stats->n_small_tiles = c.small.size();
   *n_tma = c.tma.size();
   *n_big = c.big.size();
+  if (rects) *rects = std::move(c.rects);
   tiles->clear();
   tiles->reserve(c.tma.size() + c.big.size() + c.small.size());
   tiles->insert(tiles->end(), c.tma.begin(), c.tma.end());

@@ -16,6 +16,13 @@
 // the 16-byte aligned superset of the source piece, and the warp itself copies the payload out
 // of shared memory with coalesced stores of the run's natural width (1, 2, 4 or 8 bytes), so
 // global reads stay full-width and writes stay contiguous whatever the relative shift.
+//
+// Rectangles with short rows can instead be staged with 2-D tensor-map copies
+// (cp.async.bulk.tensor.2d): one command moves a box of up to 256 rows, where the per-row form
+// would need one command per row and becomes issue-bound.  The two descriptors of a rectangle
+// (source view, target view; 8-byte elements, no swizzle) live in global memory, are encoded
+// by the host for the buffer addresses of the call, and are read through the tensormap proxy
+// after an acquire fence.
 #include "kernels.cuh"
 
 namespace bcp {
@@ -77,6 +84,24 @@ __device__ __forceinline__ void bulk_store_hint(void* dst, uint32_t src_smem, ui
                : "memory");
 }
 
+// 2-D tiled copies through a tensor map in global memory; x counts 8-byte elements, y rows
+__device__ __forceinline__ void tensormap_acquire(const void* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tensor_load_2d(uint32_t dst_smem, const void* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                   dst_smem),
+               "l"(map), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tensor_store_2d(const void* map, int x, int y, uint32_t src_smem) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y),
+               "r"(src_smem)
+               : "memory");
+}
+
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 
 template <int N>
@@ -92,8 +117,10 @@ struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memor
   uint64_t sp, dp;
   uint32_t rows, row_bytes;
   uint32_t shift;  // shifted run only: payload starts `shift` bytes into the stage
-  uint32_t width;  // 0: aligned chunk, stored with bulk copies; else log2 of the store width + 1
+  uint32_t width;  // 0: aligned chunk, stored with bulk copies; 1..4: shifted run, log2 of the store width + 1;
+                   // kTensor: one box of a tensor map (src / dst hold the descriptors, rows = box rows, shift = first row)
 };
+constexpr uint32_t kTensor = 9;
 
 // Cuts the current tile into chunks.  All lanes hold the same state.
 struct TileCursor {
@@ -102,13 +129,26 @@ struct TileCursor {
   uint64_t sp, dp;
   uint32_t rows, row_bytes;
   uint32_t r, c;  // next row, next byte inside the row
-  uint32_t width;  // 0 aligned tile; else log2(access width) + 1 of a shifted run
+  uint32_t width;  // 0 aligned tile; 1..4 log2(access width) + 1 of a shifted run; kTensor: tensor-map rectangle
+  uint32_t box_rows, row0;  // tensor-map rectangle: rows per box, first row of this unit inside the rectangle
   bool live;
 
   __device__ __forceinline__ bool next(uint32_t stage_bytes, Chunk* out) {
     if (!live) return false;
     out->shift = 0;
     out->width = 0;
+    if (width == kTensor) {  // boxes of box_rows rows; the last box of a rectangle is clipped by the descriptor
+      out->src = s;
+      out->dst = d;
+      out->rows = box_rows;
+      out->row_bytes = row_bytes;
+      out->sp = out->dp = 0;
+      out->shift = row0 + r;
+      out->width = kTensor;
+      r += min(box_rows, rows - r);
+      if (r == rows) live = false;
+      return true;
+    }
     if (width) {  // shifted run (rows == 1): pieces that leave room for the aligned superset
       const uint32_t n = min(stage_bytes - 32, row_bytes - c);
       out->src = s + c;
@@ -169,7 +209,7 @@ __device__ __forceinline__ void warp_store_out(const unsigned char* smem, char* 
 __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles,
                                                      const void* const* __restrict__ src, void* const* __restrict__ dst,
                                                      Control* ctrl, uint32_t stage_bytes, uint32_t n_stages,
-                                                     uint32_t wait_limit, uint32_t hints) {
+                                                     uint32_t wait_limit, uint32_t hints, const unsigned char* maps) {
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full[kMaxStages];
   __shared__ Chunk held[kMaxStages];
@@ -215,6 +255,18 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
       const uint32_t bits = a.x | a.z | c.x;  // low bits of src_off | dst_off | row_bytes (bases are 16-byte aligned)
       cur.width = 0;
       if (cur.rows == 1 && (bits & 15)) cur.width = (bits & 1) ? 1 : (bits & 2) ? 2 : (bits & 4) ? 3 : 4;
+      const uint4 e = __ldg(reinterpret_cast<const uint4*>(t) + 3);  // flags, reserved[0..2]
+      if (e.x & BCP_TILE_TMA2D) {  // s / d name the rectangle's descriptors instead of addresses
+        cur.width = kTensor;
+        cur.s = reinterpret_cast<const char*>(maps + uint64_t(e.y - 1) * 256);
+        cur.d = const_cast<char*>(cur.s) + 128;
+        cur.row0 = e.z;
+        cur.box_rows = e.w;
+        if (lane == 0) {
+          tensormap_acquire(cur.s);
+          tensormap_acquire(cur.d);
+        }
+      }
       if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);  // consumed when this tile is used up
     }
     return cur.next(stage_bytes, ch);
@@ -223,6 +275,15 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
   auto issue_load = [&](uint32_t stage, const Chunk& ch) {
     const uint32_t bar = smem_u32(&full[stage]);
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
+    if (ch.width == kTensor) {  // one box; the transaction count is the full box even when it is clipped
+      if (lane == 0) {
+        held[stage] = ch;
+        mbar_expect_tx(bar, ch.rows * ch.row_bytes);
+        tensor_load_2d(base, ch.src, 0, int(ch.shift), bar);
+      }
+      __syncwarp();
+      return;
+    }
     if (ch.width) {  // aligned superset of a shifted run, one bulk copy
       const uint32_t bytes = (ch.shift + ch.row_bytes + 15u) & ~15u;
       if (lane == 0) {
@@ -276,7 +337,9 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     __syncwarp();
     const Chunk h = held[stage];
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
-    if (h.width) {  // shifted run: the warp copies the payload out of the stage
+    if (h.width == kTensor) {
+      if (lane == 0) tensor_store_2d(h.dst, 0, int(h.shift), base);
+    } else if (h.width) {  // shifted run: the warp copies the payload out of the stage
       const unsigned char* p = stage_mem + stage * stage_bytes + h.shift;
       switch (h.width) {
         case 4: warp_store_out<uint2>(p, h.dst, h.row_bytes, lane); break;
@@ -343,7 +406,7 @@ cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream) {
   if (a.n_stages < 2 || a.n_stages > kMaxStages || a.stage_bytes % 128 || a.stage_bytes == 0) return cudaErrorInvalidValue;
   const size_t smem = size_t(a.stage_bytes) * a.n_stages;
   bcp_tma_kernel<<<a.grid, 32, smem, stream>>>(a.tiles, a.n_tiles, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages,
-                                               a.wait_limit, a.cache_hints);
+                                               a.wait_limit, a.cache_hints, static_cast<const unsigned char*>(a.maps));
   return cudaGetLastError();
 }
 

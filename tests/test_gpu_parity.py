@@ -87,7 +87,8 @@ def test_big_random_misaligned(cuda_device, itemsize, seed, path_mask):
                                   dict(cache_hints=2), dict(order=2), dict(unroll=8), dict(path_mask=1, worker=2),
                                   dict(path_mask=1, worker=2, unroll=8, ctas_per_sm=4, tile_bytes=16384),
                                   dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=2, tile_bytes=32768),
-                                  dict(path_mask=3, tma_stage_bytes=32768, tma_stages=6, tma_ctas_per_sm=1)])
+                                  dict(path_mask=3, tma_stage_bytes=32768, tma_stages=6, tma_ctas_per_sm=1),
+                                  dict(path_mask=7), dict(path_mask=7, tile_bytes=8192, tma_stage_bytes=4096)])
 def test_launch_options(cuda_device, opts):
     run_and_compare(CONFIGS["cfg1"]("index"), cuda_device, **opts)
     run_and_compare(big_random_case(11, itemsize=2), cuda_device, **opts)
@@ -110,12 +111,14 @@ def _dim1_split_case(shape, isz, src_parts, dst_parts):
 
 @pytest.mark.parametrize("opts", [dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=3),
                                   dict(path_mask=3, tma_stage_bytes=2048, tma_stages=8, tma_ctas_per_sm=6, tile_bytes=16384),
-                                  dict(path_mask=1, unroll=8)])
+                                  dict(path_mask=1, unroll=8), dict(path_mask=7), dict(path_mask=7, tma_stage_bytes=16384, tile_bytes=32768)])
 def test_wide_strided_rows(cuda_device, opts):
     """Strided rectangles with rows of 4-12 KiB (longer than a small TMA stage) and of 512 B."""
     run_and_compare(_dim1_split_case((96, 6144), 4, 2, 3), cuda_device, runs=2, **opts)
     run_and_compare(_dim1_split_case((1000, 1024), 2, 4, 1), cuda_device, **opts)
     run_and_compare(_dim1_split_case((333, 4096), 2, 1, 8), cuda_device, **opts)
+    run_and_compare(_dim1_split_case((5003, 256), 2, 2, 4), cuda_device, runs=2, **opts)   # 128-byte rows, ragged last box
+    run_and_compare(_dim1_split_case((777, 1032), 4, 3, 1), cuda_device, **opts)           # rows of 1376 bytes
 
 
 @pytest.mark.parametrize("case", scenario_cases()[:4] + scenario_cases()[8:10], ids=lambda c: c.name)
@@ -293,7 +296,7 @@ def _free_gb():
 
 
 @pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6),
-                                                ("cfg4odd", 0.5e9)])
+                                                ("cfg4odd", 0.5e9), ("narrow", 0.6e9)])
 def test_full_size_config(cuda_device, name, max_fqn_bytes):
     case = (CONFIGS.get(name) or STRESS[name])()
     need = (sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)) / 1e9 + 8

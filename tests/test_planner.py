@@ -154,9 +154,26 @@ def test_big_random_cases(itemsize, seed):
     assert st["bytes_misaligned"] > 0
 
 
-@pytest.mark.parametrize("opts", [dict(tile_bytes=4096), dict(order=2), dict(tile_bytes=1 << 20, small_bytes=65536)])
+@pytest.mark.parametrize("opts", [dict(tile_bytes=4096), dict(order=2), dict(tile_bytes=1 << 20, small_bytes=65536),
+                                  dict(path_mask=7), dict(path_mask=7, tile_bytes=8192)])
 def test_options_do_not_change_the_result(opts):
     check_case(scenario_cases()[3], **opts)
+    check_case(CONFIGS["cfg1"]("index"), **opts)
+
+
+def test_tensor_map_rectangles_are_whole_boxes():
+    """Units flagged for 2-D tensor-map staging cover whole boxes of their rectangle."""
+    case = CONFIGS["cfg1"]("index")
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=7)
+    tiles = [t for t in plan.tiles() if t.flags & api.TILE_TMA2D]
+    assert tiles, "cfg1 has row-parallel weights with rows of 256..1024 bytes"
+    for t in tiles:
+        box_rows = t.reserved[2]
+        assert t.reserved[0] >= 1 and box_rows >= 1 and t.reserved[1] % box_rows == 0
+        assert 16 <= t.row_bytes <= 2048 and box_rows * t.row_bytes <= 16384
+        assert (t.src_off | t.dst_off | t.src_pitch | t.dst_pitch | t.row_bytes) % 16 == 0
+    again = bcp.Plan.deserialize(plan.serialize())
+    assert [_tile_tuple(t) for t in again.tiles()] == [_tile_tuple(t) for t in plan.tiles()]
 
 
 def test_plans_partitioned_by_target_rank_cover_everything():
