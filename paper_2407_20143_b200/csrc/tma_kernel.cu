@@ -391,7 +391,13 @@ cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   const size_t smem = size_t(stage_bytes) * n_stages;
-  e = cudaFuncSetAttribute(bcp_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+  // The opt-in limit is a property of the kernel, not of a plan: raise it to the device maximum
+  // once, so that plans with different ring sizes can be executed in any order.
+  int optin = 0;
+  e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  if (smem + 1024 > size_t(optin)) return cudaErrorInvalidValue;  // 1 KiB of static shared memory and slack
+  e = cudaFuncSetAttribute(bcp_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024);
   if (e != cudaSuccess) return e;
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bcp_tma_kernel, 32, smem);
   if (e != cudaSuccess) return e;

@@ -126,6 +126,23 @@ def test_scenarios_tma_path(cuda_device, case):
     run_and_compare(case, cuda_device, path_mask=3, tile_bytes=16384, tma_stage_bytes=4096)
 
 
+def test_plans_with_different_ring_sizes_interleave(cuda_device):
+    """The TMA kernel's shared-memory ring is sized per plan; executions of plans with large and
+    small rings may alternate in any order."""
+    case = scenario_cases()[3]
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device)
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    big = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3,
+                       tma_stage_bytes=32768, tma_stages=6, tile_bytes=16384)
+    small = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3,
+                         tma_stage_bytes=2048, tma_stages=2, tile_bytes=16384)
+    for plan in (big, small, big, small, big):
+        dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+        bcp.bcp_reshard(plan, src, dst)
+        torch.cuda.synchronize()
+        assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
+
+
 def test_side_stream_and_plan_reuse(cuda_device):
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
