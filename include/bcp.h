@@ -129,7 +129,11 @@ typedef struct {
                                its own (256-thread CTAs); default 2 when this path has at least 128 MiB
                                to move, else 1                                                          */
   uint32_t tma_min_row_bytes; /* TMA path: shortest row (or run) staged through TMA; default 512; multiple of 16 */
-  uint32_t reserved[3];    /* must be 0 */
+  uint32_t allow_replicas;  /* 0 default: two saved entries of one FQN that hold the same element are an
+                               error; 1: saved entries with IDENTICAL boxes are replicas (a checkpoint saved
+                               without de-duplication): the first in input order is read, the others are
+                               ignored; boxes that overlap only partly are still BCP_ERR_OVERLAP        */
+  uint32_t reserved[2];    /* must be 0 */
 } bcp_plan_opts;
 
 typedef struct bcp_plan bcp_plan_t;
@@ -225,8 +229,9 @@ BCP_API int bcp_dedup_assign(const uint64_t* shard_bytes, const uint64_t* holder
  * host memory, caller-owned, read only during the call.  For every target entry the
  * planner finds all source entries of the same FQN whose boxes intersect it, checks that
  * they cover it exactly once, and lowers every intersection to work units
- * (bcp_tile).  Source entries of one FQN must be pairwise disjoint; target entries may
- * overlap one another as boxes (replicas) but not as byte ranges.
+ * (bcp_tile).  Source entries of one FQN must be pairwise disjoint (but see
+ * bcp_plan_opts.allow_replicas); target entries may overlap one another as boxes (replicas)
+ * but not as byte ranges.
  * On success *out_plan owns host (and, after the first bcp_reshard, device) copies of the
  * work list; release it with bcp_plan_destroy.  A plan holds no buffer addresses and can
  * be executed any number of times on any buffers of the planned sizes.

@@ -68,15 +68,19 @@ def check_family(entries: Sequence) -> Tuple[Tuple[int, ...], int]:
     return tuple(int(g) for g in e0.global_shape), int(e0.itemsize)
 
 
-def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payloads: Sequence[np.ndarray]):
+def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payloads: Sequence[np.ndarray],
+             first_wins: bool = False):
     """Full global tensor from saved shards, plus how many shards supplied each element.
 
     Sec. 3.2: shard i covers the box offsets_i + lengths_i of the global shape; an irregular
     shard covers elements [flat_begin, flat_end) of the flattened local box.
+    first_wins: replicated shards are allowed and the earliest entry supplies the value
+    (entries are assigned last to first, so the first one overwrites the rest).
     """
     T = np.zeros(tuple(global_shape), dtype=_UINT[itemsize])
     cover = np.zeros(tuple(global_shape), dtype=np.uint8)
-    for e, data in zip(entries, payloads):
+    pairs = list(zip(entries, payloads))
+    for e, data in (reversed(pairs) if first_wins else pairs):
         b = _box(e)
         if e.kind == FLAT_SLICE:
             a, z = int(e.flat_begin), int(e.flat_end)
@@ -94,7 +98,7 @@ def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payl
     return T, cover
 
 
-def take(T: np.ndarray, cover: np.ndarray, e) -> np.ndarray:
+def take(T: np.ndarray, cover: np.ndarray, e, replicas_ok: bool = False) -> np.ndarray:
     """Bytes of the wanted shard e cut out of the assembled tensor (uint8, C order)."""
     b = _box(e)
     if e.kind == FLAT_SLICE:
@@ -104,7 +108,7 @@ def take(T: np.ndarray, cover: np.ndarray, e) -> np.ndarray:
         vals, cov = T[b].ravel(), cover[b].ravel()
     if cov.size and cov.min() < 1:
         raise OracleError(f"{e.fqn}: wanted element held by no saved shard")
-    if cov.size and cov.max() > 1:
+    if cov.size and cov.max() > 1 and not replicas_ok:
         raise OracleError(f"{e.fqn}: element held by more than one saved shard")
     return np.ascontiguousarray(vals).view(np.uint8)
 
@@ -116,16 +120,19 @@ def group_by_fqn(entries: Iterable) -> Dict[str, List]:
     return g
 
 
-def reshard_fqn(src_entries: Sequence, src_payloads: Sequence[np.ndarray], dst_entries: Sequence) -> List[np.ndarray]:
+def reshard_fqn(src_entries: Sequence, src_payloads: Sequence[np.ndarray], dst_entries: Sequence,
+                allow_replicas: bool = False) -> List[np.ndarray]:
     """Bytes of every wanted shard of ONE FQN, given the payloads of its saved shards."""
     shape, itemsize = check_family(list(src_entries) + list(dst_entries))
-    T, cover = assemble(shape, itemsize, src_entries, src_payloads)
-    return [take(T, cover, d) for d in dst_entries]
+    T, cover = assemble(shape, itemsize, src_entries, src_payloads, first_wins=allow_replicas)
+    return [take(T, cover, d, replicas_ok=allow_replicas) for d in dst_entries]
 
 
 def reshard(src_metas: Sequence, src_blobs: Sequence[np.ndarray], dst_metas: Sequence,
-            dst_buf_bytes: Sequence[int], fill_byte: int = 0) -> List[np.ndarray]:
-    """Every target rank buffer (uint8 arrays); bytes no entry names keep `fill_byte`."""
+            dst_buf_bytes: Sequence[int], fill_byte: int = 0, allow_replicas: bool = False) -> List[np.ndarray]:
+    """Every target rank buffer (uint8 arrays); bytes no entry names keep `fill_byte`.
+    allow_replicas: saved shards may be stored more than once (a checkpoint written without
+    de-duplication); the first entry in input order supplies the bytes."""
     out = [np.full(int(n), fill_byte, dtype=np.uint8) for n in dst_buf_bytes]
     src_by, dst_by = group_by_fqn(src_metas), group_by_fqn(dst_metas)
     for fqn, dsts in dst_by.items():
@@ -135,7 +142,7 @@ def reshard(src_metas: Sequence, src_blobs: Sequence[np.ndarray], dst_metas: Seq
                 continue
             raise OracleError(f"{fqn}: wanted but never saved")
         payloads = [_payload(src_blobs[s.buf_index], s) for s in srcs]
-        for d, data in zip(dsts, reshard_fqn(srcs, payloads, dsts)):
+        for d, data in zip(dsts, reshard_fqn(srcs, payloads, dsts, allow_replicas)):
             buf = out[d.buf_index]
             if d.byte_offset + d.byte_length > buf.size:
                 raise OracleError(f"{fqn}: target byte range outside its buffer")

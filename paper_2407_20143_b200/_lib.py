@@ -43,7 +43,8 @@ class PlanOptsC(C.Structure):
         ("unroll", C.c_uint32),
         ("worker", C.c_uint32),
         ("tma_min_row_bytes", C.c_uint32),
-        ("reserved", C.c_uint32 * 3),
+        ("allow_replicas", C.c_uint32),
+        ("reserved", C.c_uint32 * 2),
     ]
 
 

@@ -487,7 +487,7 @@ int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_by
     std::vector<Item> items;
     bcp_plan_stats_t st;
     memset(&st, 0, sizeof st);
-    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, &items, &st))
+    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt.allow_replicas != 0, &items, &st))
       return rc;
     bcp_plan_t* p = finish_plan(items, opt, st, std::vector<uint64_t>(src_buf_bytes, src_buf_bytes + n_src_bufs),
                               std::vector<uint64_t>(dst_buf_bytes, dst_buf_bytes + n_dst_bufs));

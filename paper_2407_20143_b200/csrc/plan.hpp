@@ -38,6 +38,7 @@ struct Options {
   uint32_t unroll = 4;
   uint32_t worker = 0;  // 0: chosen from the work list
   uint32_t tma_min_row_bytes = 512;
+  uint32_t allow_replicas = 0;
 };
 
 // A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source
@@ -60,7 +61,7 @@ void decompose(const int64_t* lengths, uint32_t ndim, int64_t a, int64_t b, std:
 // counters of `stats`.
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    std::vector<Item>* items, bcp_plan_stats_t* stats);
+                    bool allow_replicas, std::vector<Item>* items, bcp_plan_stats_t* stats);
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
 // tiles = [TMA units..., other CTA-wide units..., warp units...].

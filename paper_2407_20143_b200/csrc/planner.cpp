@@ -50,6 +50,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->unroll) o.unroll = in->unroll;
     if (in->worker) o.worker = in->worker;
     if (in->tma_min_row_bytes) o.tma_min_row_bytes = in->tma_min_row_bytes;
+    o.allow_replicas = in->allow_replicas;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -68,6 +69,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.tma_ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "tma_ctas_per_sm must be in [1, 16]");
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
+  if (o.allow_replicas > 1) return fail(BCP_ERR_INVALID, "allow_replicas must be 0 or 1");
   if (o.worker > 2) return fail(BCP_ERR_INVALID, "worker must be 0, 1 or 2");
   if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
     return fail(BCP_ERR_INVALID, "tma_min_row_bytes must be a multiple of 16 in [16, 65536]");
@@ -345,7 +347,7 @@ struct SegKey {  // identity of a matched segment on the saved side (for the uni
 
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    std::vector<Item>* items, bcp_plan_stats_t* stats) {
+                    bool allow_replicas, std::vector<Item>* items, bcp_plan_stats_t* stats) {
   if ((n_src && !src) || (n_dst && !dst) || (n_src_bufs && !src_buf_bytes) || (n_dst_bufs && !dst_buf_bytes))
     return fail(BCP_ERR_INVALID, "bcp_plan: NULL array with non-zero count");
   std::unordered_map<std::string, uint32_t> ids;
@@ -409,6 +411,24 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
     n_se += f.src.size();
     n_de += f.dst.size();
     const uint32_t nd = f.ndim;
+    if (allow_replicas && f.src.size() > 1) {
+      // identical boxes are replicas of one shard: keep the one that came first in the input
+      std::sort(f.src.begin(), f.src.end(), [nd](const Entry& a, const Entry& b) {
+        for (uint32_t k = 0; k < nd; ++k) {
+          if (a.off[k] != b.off[k]) return a.off[k] < b.off[k];
+          if (a.len[k] != b.len[k]) return a.len[k] < b.len[k];
+        }
+        return a.meta < b.meta;
+      });
+      size_t kept = 0;
+      for (size_t i = 0; i < f.src.size(); ++i) {
+        bool same = kept > 0;
+        for (uint32_t k = 0; same && k < nd; ++k)
+          same = f.src[i].off[k] == f.src[kept - 1].off[k] && f.src[i].len[k] == f.src[kept - 1].len[k];
+        if (!same) f.src[kept++] = f.src[i];
+      }
+      f.src.resize(kept);
+    }
     // saved boxes of one tensor must be pairwise disjoint (each element is stored once)
     std::sort(f.src.begin(), f.src.end(), [](const Entry& a, const Entry& b) { return a.off[0] < b.off[0]; });
     for (size_t i = 0; i < f.src.size(); ++i) {

@@ -169,6 +169,24 @@ def test_hundred_thousand_tiny_tensors(cuda_device):
     assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
 
 
+def test_replicated_saved_side(cuda_device):
+    """A checkpoint written without de-duplication: replicas allowed, the first one is read."""
+    from workloads.configs import MIXED, small_gpt
+    from workloads.layouts import Parallelism, ReshardCase, build_state
+
+    g = small_gpt()
+    case = ReshardCase("replicated-source", build_state(g, Parallelism(tp=2, dp=2, pp=2, zero="zero1"), MIXED, dedup=False),
+                       build_state(g, Parallelism(tp=1, dp=3, pp=4, zero="zero1"), MIXED, dedup=False), "index", 5)
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device)
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON,
+                       allow_replicas=True)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, allow_replicas=1)
+    dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(plan, src, dst)
+    torch.cuda.synchronize()
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
+
+
 def test_deserialized_plan_executes(cuda_device):
     """A plan image written by one plan object runs identically when rebuilt (plan cache)."""
     case = CONFIGS["cfg1"]("index")

@@ -206,6 +206,59 @@ def test_plans_partitioned_by_target_rank_cover_everything():
         assert np.array_equal(g, w)
 
 
+# ---- replicated saved shards (a checkpoint written without de-duplication) ------------------------------
+def _replicated_case():
+    """The hybrid scenario with its saved side NOT de-duplicated: every holder stores its copy."""
+    from workloads.configs import MIXED, small_gpt
+    from workloads.layouts import Parallelism, ReshardCase, build_state
+
+    g = small_gpt()
+    src = build_state(g, Parallelism(tp=2, dp=2, pp=2, zero="zero1"), MIXED, dedup=False)
+    dst = build_state(g, Parallelism(tp=1, dp=3, pp=4, zero="zero1"), MIXED, dedup=False)
+    return ReshardCase("replicated-source", src, dst, "index", 5)
+
+
+def test_replicas_are_an_error_unless_allowed():
+    case = _replicated_case()
+    assert _plan_err(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes) == api.ERR_OVERLAP
+    blobs = np_bufs(fills.fill_state(case.src, case.key_ids, "index", case.seed, "cpu"))
+    with pytest.raises(orc.OracleError):
+        orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, allow_replicas=1)
+    got, _ = run_tiles(plan.tiles(), blobs, case.dst.buf_bytes)
+    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, allow_replicas=True)
+    assert all(np.array_equal(g, w) for g, w in zip(got, want))
+    # consistent replicas: same result as the closed-form fill of the wanted side
+    closed = np_bufs(fills.fill_state(case.dst, case.key_ids, "index", case.seed, "cpu", poison=0xA5))
+    assert all(np.array_equal(g, w) for g, w in zip(got, closed))
+    assert plan.stats()["bytes_src_unique"] < case.src.total_bytes
+
+
+def test_first_replica_wins_and_partial_overlap_stays_an_error():
+    a = _m(boff=0)
+    b = _m(boff=64)  # same box, different bytes
+    blob = np.concatenate([np.full(64, 1, np.uint8), np.full(64, 2, np.uint8)])
+    plan = bcp.bcp_plan([a, b], [128], [_m()], [64], allow_replicas=1)
+    got, _ = run_tiles(plan.tiles(), [blob], [64])
+    want = orc.reshard([a, b], [blob], [_m()], [64], allow_replicas=True)
+    assert np.array_equal(got[0], want[0]) and set(got[0]) == {1}
+    plan = bcp.bcp_plan([b, a], [128], [_m()], [64], allow_replicas=1)  # input order decides, not byte order
+    got, _ = run_tiles(plan.tiles(), [blob], [64])
+    assert set(got[0]) == {2} and np.array_equal(got[0], orc.reshard([b, a], [blob], [_m()], [64], allow_replicas=True)[0])
+    assert _plan_err([_m(ln=(3, 4)), _m(off=(2, 0), ln=(2, 4), boff=48)], [80], [_m()], [64], allow_replicas=1) == api.ERR_OVERLAP
+
+
+def test_single_run_larger_than_4_gib_is_cut_without_overflow():
+    n = 6 * (1 << 30) + 48
+    m = ShardMeta("huge", 1, 3, (n,), (0,), (n,), 0, 16)
+    plan = bcp.bcp_plan([m], [n + 16], [ShardMeta("huge", 1, 3, (n,), (0,), (n,), 0, 0)], [n])
+    tiles = plan.tiles()
+    assert sum(t.rows * t.row_bytes for t in tiles) == n and plan.stats()["bytes_copied"] == n
+    order = sorted(tiles, key=lambda t: t.dst_off)
+    assert order[0].dst_off == 0 and all(a.dst_off + a.row_bytes == b.dst_off for a, b in zip(order, order[1:]))
+    assert all(t.src_off == t.dst_off + 16 for t in tiles) and order[-1].dst_off + order[-1].row_bytes == n
+
+
 # ---- plan images (plan cache across processes, Sec. 4.1) ----------------------------------------------
 def _tile_tuple(t):
     return (t.src_off, t.dst_off, t.src_pitch, t.dst_pitch, t.row_bytes, t.rows, t.src_buf, t.dst_buf, t.flags)
