@@ -332,6 +332,35 @@ BCP_API int bcp_unpack(const void* blob, uint64_t blob_bytes, const bcp_pack_met
 BCP_API int bcp_pack_cache_clear(void);
 
 /*
+ * Safetensors export (the paper's system exports checkpoints in the Safetensors format for
+ * the Hugging Face ecosystem, Sec. 7).  An image is: 8 bytes little-endian header length,
+ * the JSON header (every tensor's dtype, shape and [begin, end) offsets into the byte buffer;
+ * padded with spaces so that the buffer starts on an 8-byte boundary), then the tensors back
+ * to back in the order given.  dtype is one of BOOL U8 I8 F8_E5M2 F8_E4M3 I16 U16 F16 BF16 I32
+ * U32 F32 F64 I64 U64; a tensor's byte length is prod(shape) * size of the dtype.
+ *
+ * bcp_safetensors_layout (host only) writes the first 8 + N bytes of the image to header_out
+ * and every tensor's byte range INSIDE THE IMAGE to out_metas (usable as bcp_pack metas);
+ * with header_cap too small it still reports *header_bytes, *file_bytes and out_metas and
+ * returns BCP_ERR_CAPACITY.
+ * bcp_safetensors_export builds the whole image in device memory at `file` (capacity
+ * file_cap bytes): the tensors (device pointers, any alignment) are packed by the copy kernels
+ * and the header is copied over the front, all on `stream`, asynchronously.  The pageable
+ * header is staged by the runtime before the call returns.
+ */
+typedef struct {
+  const char* name;   /* host, NUL-terminated, unique, not "__metadata__" */
+  const char* dtype;  /* host, NUL-terminated                                */
+  uint32_t ndim;      /* 0..BCP_MAX_NDIM                                     */
+  uint32_t reserved;
+  int64_t shape[BCP_MAX_NDIM];
+} bcp_export_entry;
+BCP_API int bcp_safetensors_layout(const bcp_export_entry* entries, size_t n, void* header_out, size_t header_cap,
+                                   size_t* header_bytes, bcp_pack_meta* out_metas, uint64_t* file_bytes);
+BCP_API int bcp_safetensors_export(const bcp_export_entry* entries, const void* const* tensors, size_t n, void* file,
+                                   uint64_t file_cap, uint64_t* file_bytes, void* stream);
+
+/*
  * Asynchronous save / load staging through a pool of pinned host buffers with ping-pong
  * use (Sec. 4.2: the save pipeline copies shards to a pinned memory pool with ping-pong
  * buffering so that only a short step blocks training; loading mirrors it).

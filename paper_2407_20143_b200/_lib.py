@@ -70,6 +70,11 @@ class PlanStatsC(C.Structure):
         ("plan_ms", C.c_double)]
 
 
+class ExportEntryC(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("dtype", C.c_char_p), ("ndim", C.c_uint32), ("reserved", C.c_uint32),
+                ("shape", C.c_int64 * BCP_MAX_NDIM)]
+
+
 class PackMetaC(C.Structure):
     _fields_ = [("byte_offset", C.c_uint64), ("byte_length", C.c_uint64)]
 
@@ -98,6 +103,10 @@ _PROTOS = {
     "bcp_pack": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
     "bcp_unpack": (C.c_int, [_VP, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
     "bcp_pack_cache_clear": (C.c_int, []),
+    "bcp_safetensors_layout": (C.c_int, [C.POINTER(ExportEntryC), C.c_size_t, _VP, C.c_size_t, C.POINTER(C.c_size_t),
+                                         C.POINTER(PackMetaC), C.POINTER(C.c_uint64)]),
+    "bcp_safetensors_export": (C.c_int, [C.POINTER(ExportEntryC), C.POINTER(_VP), C.c_size_t, _VP, C.c_uint64,
+                                         C.POINTER(C.c_uint64), _VP]),
     "bcp_stager_create": (C.c_int, [C.c_uint64, C.c_uint32, C.POINTER(_VP)]),
     "bcp_stager_destroy": (C.c_int, [_VP]),
     "bcp_stager_save": (C.c_int, [_VP, C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, C.c_uint64, _VP,

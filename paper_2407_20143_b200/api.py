@@ -222,6 +222,44 @@ def bcp_unpack(blob, metas: Sequence[Tuple[int, int]], tensors: Sequence, blob_b
     _check(L.lib().bcp_unpack(bp, nb, _pack_metas(metas), len(tensors), _ptrs(tensors), _stream(stream)))
 
 
+def _export_entries(entries: Sequence[Tuple[str, str, Sequence[int]]]):
+    arr = (L.ExportEntryC * max(1, len(entries)))()
+    keep = []
+    for c, (name, dtype, shape) in zip(arr, entries):
+        nb, db = name.encode(), dtype.encode()
+        keep += [nb, db]
+        c.name, c.dtype, c.ndim = nb, db, len(shape)
+        for k, x in enumerate(shape):
+            c.shape[k] = x
+    return arr, keep
+
+
+def bcp_safetensors_layout(entries: Sequence[Tuple[str, str, Sequence[int]]]) -> Tuple[bytes, List[Tuple[int, int]], int]:
+    """(header bytes, per-tensor (offset, length) inside the image, image size) for tensors given
+    as (name, safetensors dtype string, shape)."""
+    arr, keep = _export_entries(entries)
+    n = len(entries)
+    hb, fb = C.c_size_t(), C.c_uint64()
+    metas = (L.PackMetaC * max(1, n))()
+    L.lib().bcp_safetensors_layout(arr, n, None, 0, C.byref(hb), metas, C.byref(fb))
+    buf = (C.c_uint8 * max(1, hb.value))()
+    _check(L.lib().bcp_safetensors_layout(arr, n, buf, hb.value, C.byref(hb), metas, C.byref(fb)))
+    del keep
+    return bytes(buf[: hb.value]), [(m.byte_offset, m.byte_length) for m in metas[:n]], fb.value
+
+
+def bcp_safetensors_export(entries: Sequence[Tuple[str, str, Sequence[int]]], tensors: Sequence, file, file_cap: Optional[int] = None,
+                           stream=None) -> int:
+    """Build a Safetensors image of `tensors` in the device buffer `file`; returns its size in bytes."""
+    arr, keep = _export_entries(entries)
+    cap = file_cap if file_cap is not None else file.numel() * file.element_size()
+    fp = file if isinstance(file, int) else file.data_ptr()
+    fb = C.c_uint64()
+    _check(L.lib().bcp_safetensors_export(arr, _ptrs(tensors), len(entries), fp, cap, C.byref(fb), _stream(stream)))
+    del keep
+    return fb.value
+
+
 class Stager:
     """Pinned ping-pong pool for asynchronous save / load staging (bcp_stager_* calls)."""
 
