@@ -60,7 +60,7 @@ def parse_args():
                     help="also time asynchronous save staging of every target rank through the pinned ping-pong pool")
     ap.add_argument("--cpu-sample-gb", type=float, default=4.0,
                     help="bytes read+written by one pass of the CPU oracle over its sample of the workload")
-    ap.add_argument("--cpu-passes", type=int, default=5)
+    ap.add_argument("--cpu-passes", type=int, default=40, help="timed passes of the oracle over its sample (about 10 s)")
     for o in ("tile-bytes", "small-bytes", "block-threads", "ctas-per-sm", "order", "path-mask", "cache-hints"):
         ap.add_argument("--" + o, type=int, default=0)
     return ap.parse_args()
