@@ -160,7 +160,7 @@ typedef struct {
                                    src_off, dst_off, row_bytes and both pitches                  */
 #define BCP_TILE_ZERO 0x8u      /* no source: write zero bytes (pack padding)                    */
 #define BCP_TILE_SMALL 0x10u    /* executed by one warp                                          */
-#define BCP_TILE_TMA 0x20u      /* eligible for the TMA staging path                             */
+#define BCP_TILE_TMA 0x20u      /* executed by the TMA staging kernel                            */
 #define BCP_TILE_TMA2D 0x40u    /* rows of a rectangle staged with 2-D tensor-map copies: reserved[0] =
                                    rectangle index + 1, reserved[1] = first row inside the rectangle,
                                    reserved[2] = rows per box                                    */
@@ -174,7 +174,7 @@ typedef struct {
   uint64_t n_tiles;          /* CTA-wide work units                                   */
   uint64_t n_small_tiles;    /* warp work units                                       */
   uint64_t n_strided_tiles;  /* work units with rows > 1                              */
-  uint64_t n_tma_tiles;      /* work units eligible for the TMA path                  */
+  uint64_t n_tma_tiles;      /* work units executed by the TMA staging kernel         */
   uint64_t bytes_copied;     /* payload bytes the list writes = sum of target bytes   */
   uint64_t bytes_src_unique; /* distinct source bytes the list reads                  */
   uint64_t bytes_misaligned; /* payload in units whose access granularity is < 16 B   */

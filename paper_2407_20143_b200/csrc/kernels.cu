@@ -1,6 +1,8 @@
-// sm_100a kernels that execute the resharding work list.
+// Register (LDG/STG) kernels that execute the resharding work list, or the part of it that the
+// TMA staging kernel (tma_kernel.cu) does not take: pieces that are not 16-byte aligned in two
+// dimensions, rows too short for bulk copies, zero fills, and units under 4 KiB.
 //
-// One persistent kernel runs the whole list (Sec. 3.3 Step 5 of arXiv 2407.20143: every
+// One persistent kernel runs its whole list (Sec. 3.3 Step 5 of arXiv 2407.20143: every
 // matched segment is copied into its target shard).  CTAs draw work units from an atomic
 // ticket counter; a unit is either one CTA-wide tile (up to tile_bytes of payload, a run or a
 // strided rectangle) or a batch of small tiles, one per warp.  Every tile carries the widest
