@@ -241,6 +241,25 @@ def test_reshard_host(cuda_device):
         assert all(np.array_equal(d.numpy(), w) for d, w in zip(dst, want))
 
 
+@pytest.mark.parametrize("name", ["dp150-to-dp75", "hybrid", "llama-tp8-to-tp2"])
+def test_reshard_host_scenarios(cuda_device, name):
+    """Host-buffer path on layouts with many buffers (600 saved ranks, two of them empty), replicas
+    and strided pieces; pageable host memory works too, pinned is only faster."""
+    case = [c for c in scenario_cases() if c.name == name][0]
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, "cpu")
+    dst = [torch.full((n,), POISON, dtype=torch.uint8) for n in case.dst.buf_bytes]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    bcp.bcp_reshard_host(plan, [s.data_ptr() if s.numel() else 0 for s in src], [d.data_ptr() if d.numel() else 0 for d in dst])
+    want = orc.reshard(case.src.metas, [s.numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=0)
+    assert all(np.array_equal(d.numpy(), w) for d, w in zip(dst, want))
+    # the same plan still serves device buffers afterwards
+    dsrc = [s.to(cuda_device) for s in src]
+    ddst = [torch.zeros(n, dtype=torch.uint8, device=cuda_device) for n in case.dst.buf_bytes]
+    bcp.bcp_reshard(plan, [s.data_ptr() if s.numel() else 0 for s in dsrc], [d.data_ptr() if d.numel() else 0 for d in ddst])
+    torch.cuda.synchronize()
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(ddst, want))
+
+
 # ---- pack / unpack ---------------------------------------------------------------------------------
 def _pack_check(device, sizes, align, offsets=None, misalign=0):
     g = torch.Generator(device="cpu").manual_seed(len(sizes) * 7919 + align + misalign)
