@@ -127,5 +127,27 @@ def scenario_cases() -> List[ReshardCase]:
                      Parallelism(dp=128, zero="fsdp"), Parallelism(dp=64, zero="fsdp"), OPTIM_ONLY),
         reshard_case("moe-ep8-to-ep4", moe_model("moe-s", 2, 64, 16, 48, 256), Parallelism(ep=8),
                      Parallelism(ep=4), MOE_KINDS),
+        # odd sizes: vocabulary 50257 and hidden 1000 split three ways (uneven), bf16 rows cut at odd
+        # element counts, so two-dimensional pieces are only 2-byte aligned
+        reshard_case("odd-gpt-tp3-to-tp2", gpt_model("gpt-odd", L=1, H=1000, F=4000, V=50257, P=77), Parallelism(tp=3),
+                     Parallelism(tp=2), PARAMS_ONLY),
+        stacked_experts_case(),
     ]
     return out
+
+
+def stacked_experts_case() -> ReshardCase:
+    """Experts stacked in one 3-D tensor [E, F, H]: saved split along dim 0 over 4 ranks, wanted
+    as six flat slices of the whole stack (boundaries inside rows of the middle experts)."""
+    from .meta import FLAT_SLICE, ShardMeta, ShardedState
+
+    E, F, H, isz = 8, 24, 40, 4
+    shape = (E, F, H)
+    src = ShardedState([ShardMeta("experts.w", isz, DTYPE_F32, shape, (2 * r, 0, 0), (2, F, H), r, 256) for r in range(4)],
+                       [256 + 2 * F * H * isz] * 4)
+    n = E * F * H
+    cut = -(-n // 6)
+    dst = ShardedState([ShardMeta("experts.w", isz, DTYPE_F32, shape, (0, 0, 0), shape, r, 0, FLAT_SLICE, r * cut,
+                                  min(n, (r + 1) * cut)) for r in range(6)],
+                       [(min(n, (r + 1) * cut) - r * cut) * isz for r in range(6)])
+    return ReshardCase("stacked-experts-3d", src, dst, "index", 3)
