@@ -556,9 +556,8 @@ bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vect
   }
   if (t.flags & BCP_TILE_TMA) {
     if (zero || t.row_bytes < 16) return false;
-    if (g < 4) {  // shifted run: one row, aligned superset inside the source buffer
-      if (t.rows != 1) return false;
-      if (((t.src_off + t.row_bytes + 15) & ~uint64_t(15)) > sb[t.src_buf]) return false;
+    if (g < 4) {  // shifted run or rectangle: the aligned superset of the last row stays inside the source buffer
+      if (((t.src_off + uint64_t(t.rows - 1) * t.src_pitch + t.row_bytes + 15) & ~uint64_t(15)) > sb[t.src_buf]) return false;
     }
   }
   return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;

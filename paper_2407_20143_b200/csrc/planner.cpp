@@ -521,11 +521,11 @@ struct Cutter {
       small.push_back(t);
     } else {
       // TMA staging: whole 16-byte units between 16-byte aligned addresses (runs and rectangles),
-      // or a run of any alignment whose 16-byte aligned superset stays inside the source buffer
+      // or a run / rectangle of any alignment whose 16-byte aligned supersets stay inside the source buffer
       bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= opt.tma_min_row_bytes;
-      if (eligible && g < 4) {
-        const uint64_t end16 = (src_off + row_bytes + 15) & ~uint64_t(15);
-        eligible = rows == 1 && src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
+      if (eligible && g < 4) {  // the superset of the last row must not reach past the source buffer
+        const uint64_t end16 = (src_off + (rows - 1) * (rows > 1 ? it.src_pitch : 0) + row_bytes + 15) & ~uint64_t(15);
+        eligible = src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
       }
       if (eligible) {
         t.flags |= BCP_TILE_TMA;

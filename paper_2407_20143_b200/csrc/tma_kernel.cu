@@ -15,7 +15,9 @@
 // element cuts of ZeRO / FSDP flat shards, odd shapes), are staged too: the bulk load fetches
 // the 16-byte aligned superset of the source piece, and the warp itself copies the payload out
 // of shared memory with coalesced stores of the run's natural width (1, 2, 4 or 8 bytes), so
-// global reads stay full-width and writes stay contiguous whatever the relative shift.
+// global reads stay full-width and writes stay contiguous whatever the relative shift.  Strided
+// rectangles with such offsets or pitches are handled the same way, several rows per stage,
+// each row in a slot of its own.
 //
 // Rectangles with short rows can instead be staged with 2-D tensor-map copies
 // (cp.async.bulk.tensor.2d): one command moves a box of up to 256 rows, where the per-row form
@@ -120,6 +122,7 @@ struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memor
   uint32_t width;  // 0: aligned chunk, stored with bulk copies; 1..4: shifted run, log2 of the store width + 1;
                    // kTensor: one box of a tensor map (src / dst hold the descriptors, rows = box rows, shift = first row)
 };
+constexpr uint32_t kShiftedRows = 4;  // width codes 5..8: several shifted rows per chunk, `shift` = bytes per row slot
 constexpr uint32_t kTensor = 9;
 
 // Cuts the current tile into chunks.  All lanes hold the same state.
@@ -149,17 +152,37 @@ struct TileCursor {
       if (r == rows) live = false;
       return true;
     }
-    if (width) {  // shifted run (rows == 1): pieces that leave room for the aligned superset
+    if (width) {  // shifted run or rectangle: every row is fetched as its 16-byte aligned superset
+      const uint32_t slot = (row_bytes + 45u) & ~15u;  // room for the superset of a row, whatever its shift
+      if (rows > 1 && slot <= stage_bytes) {           // several whole rows, one slot each
+        const uint32_t k = min(stage_bytes / slot, rows - r);
+        out->src = s + uint64_t(r) * sp;
+        out->dst = d + uint64_t(r) * dp;
+        out->rows = k;
+        out->row_bytes = row_bytes;
+        out->sp = sp;
+        out->dp = dp;
+        out->shift = slot;
+        out->width = width + kShiftedRows;
+        r += k;
+        if (r == rows) live = false;
+        return true;
+      }
+      // pieces of one row that leave room for the aligned superset
       const uint32_t n = min(stage_bytes - 32, row_bytes - c);
-      out->src = s + c;
-      out->dst = d + c;
+      out->src = s + uint64_t(r) * sp + c;
+      out->dst = d + uint64_t(r) * dp + c;
       out->rows = 1;
       out->row_bytes = n;
       out->sp = out->dp = 0;
       out->shift = uint32_t(reinterpret_cast<uintptr_t>(out->src) & 15);
       out->width = width;
       c += n;
-      if (c == row_bytes) live = false;
+      if (c == row_bytes) {
+        c = 0;
+        ++r;
+      }
+      if (r == rows) live = false;
       return true;
     }
     if (row_bytes > stage_bytes || rows == 1) {  // pieces of one row
@@ -254,7 +277,8 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
       // a run that is not 16-byte aligned on both sides and in length is staged as a shifted run
       const uint32_t bits = a.x | a.z | c.x;  // low bits of src_off | dst_off | row_bytes (bases are 16-byte aligned)
       cur.width = 0;
-      if (cur.rows == 1 && (bits & 15)) cur.width = (bits & 1) ? 1 : (bits & 2) ? 2 : (bits & 4) ? 3 : 4;
+      const uint32_t all = bits | b.x | b.z;  // ... and of both pitches
+      if (all & 15) cur.width = (all & 1) ? 1 : (all & 2) ? 2 : (all & 4) ? 3 : 4;
       const uint4 e = __ldg(reinterpret_cast<const uint4*>(t) + 3);  // flags, reserved[0..2]
       if (e.x & BCP_TILE_TMA2D) {  // s / d name the rectangle's descriptors instead of addresses
         cur.width = kTensor;
@@ -282,6 +306,26 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
         tensor_load_2d(base, ch.src, 0, int(ch.shift), bar);
       }
       __syncwarp();
+      return;
+    }
+    if (ch.width > kShiftedRows) {  // shifted rows: one superset per row, each into its own slot
+      uint32_t mine = 0;
+      for (uint32_t r = lane; r < ch.rows; r += 32) {
+        const uint32_t sh = uint32_t(reinterpret_cast<uintptr_t>(ch.src + uint64_t(r) * ch.sp) & 15);
+        mine += (sh + ch.row_bytes + 15u) & ~15u;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+      if (lane == 0) {
+        held[stage] = ch;
+        mbar_expect_tx(bar, mine);
+      }
+      __syncwarp();
+      for (uint32_t r = lane; r < ch.rows; r += 32) {
+        const char* a = ch.src + uint64_t(r) * ch.sp;
+        const uint32_t sh = uint32_t(reinterpret_cast<uintptr_t>(a) & 15);
+        bulk_load(base + r * ch.shift, a - sh, (sh + ch.row_bytes + 15u) & ~15u, bar);
+      }
       return;
     }
     if (ch.width) {  // aligned superset of a shifted run, one bulk copy
@@ -339,6 +383,19 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
     if (h.width == kTensor) {
       if (lane == 0) tensor_store_2d(h.dst, 0, int(h.shift), base);
+    } else if (h.width > kShiftedRows) {  // shifted rows: the warp copies row after row out of its slot
+      for (uint32_t r = 0; r < h.rows; ++r) {
+        const uint32_t sh = uint32_t(reinterpret_cast<uintptr_t>(h.src + uint64_t(r) * h.sp) & 15);
+        const unsigned char* p = stage_mem + stage * stage_bytes + r * h.shift + sh;
+        char* q = h.dst + uint64_t(r) * h.dp;
+        switch (h.width - kShiftedRows) {
+          case 4: warp_store_out<uint2>(p, q, h.row_bytes, lane); break;
+          case 3: warp_store_out<unsigned int>(p, q, h.row_bytes, lane); break;
+          case 2: warp_store_out<unsigned short>(p, q, h.row_bytes, lane); break;
+          default: warp_store_out<unsigned char>(p, q, h.row_bytes, lane); break;
+        }
+      }
+      __syncwarp();
     } else if (h.width) {  // shifted run: the warp copies the payload out of the stage
       const unsigned char* p = stage_mem + stage * stage_bytes + h.shift;
       switch (h.width) {

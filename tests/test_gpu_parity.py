@@ -350,7 +350,7 @@ def _free_gb():
 
 
 @pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6),
-                                                ("cfg4odd", 0.5e9), ("narrow", 0.6e9)])
+                                                ("cfg4odd", 0.5e9), ("narrow", 0.6e9), ("oddgpt", 0.6e9)])
 def test_full_size_config(cuda_device, name, max_fqn_bytes):
     case = (CONFIGS.get(name) or STRESS[name])()
     need = (sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)) / 1e9 + 8

@@ -76,7 +76,16 @@ def narrow_rows(layers: int = 4, cols: int = 256) -> ReshardCase:
                         seed=20150)
 
 
-STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows}
+def odd_gpt(layers: int = 12) -> ReshardCase:
+    """Unscored stress: a GPT with hidden 3000, FFN 12000 and the 50257-token vocabulary, bf16
+    parameters, TP3 -> TP2: the splits are uneven and row-parallel weights are cut at odd element
+    counts, so most two-dimensional pieces are only 2-, 4- or 8-byte aligned."""
+    m = gpt_model("gpt-odd", L=layers, H=3000, F=12000, V=50257, P=1024)
+    return reshard_case(f"odd-gpt-tp3-to-tp2-L{layers}", m, Parallelism(tp=3), Parallelism(tp=2), PARAMS_ONLY, "index",
+                        seed=20151)
+
+
+STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows, "oddgpt": odd_gpt}
 
 CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
     "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
