@@ -295,6 +295,8 @@ def main():
     stream = torch.cuda.current_stream()
 
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(a.steps)]
+    # inputs far larger than the 126 MB L2 need no flush; small workloads get one before every step
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if b_min < (1 << 30) else None
     with ClockSampler(local_rank) as clocks:
         clocks.wait_first_sample()
         for _ in range(max(a.warmup, 3)):
@@ -307,6 +309,8 @@ def main():
         clocks.mark_begin()
         t_begin.record(stream)
         for e0, e1 in evs:
+            if flush is not None:
+                flush.zero_()  # evict the previous step's lines: this workload would fit in L2
             e0.record(stream)
             bcp.bcp_reshard(plan, src, dst, stream)
             e1.record(stream)
@@ -316,7 +320,8 @@ def main():
     D.barrier()
     total_ms = t_begin.elapsed_time(t_end)
     launch_ms = sorted(e0.elapsed_time(e1) for e0, e1 in evs)
-    ms_step = D.max_over_ranks(total_ms / a.steps, dev)
+    # with flushes between the steps only the steps themselves count
+    ms_step = D.max_over_ranks((sum(launch_ms) if flush is not None else total_ms) / a.steps, dev)
     bcp.bcp_plan_device_status(plan)
     value = b_min * ws / (ms_step * 1e-3) / 1e9
 
@@ -345,7 +350,8 @@ def main():
         "config": {"workload": case.name, "src_bytes": st["bytes_src_unique"], "dst_bytes": st["bytes_copied"],
                    "bytes_per_step": b_min, "bytes_counted": "unique source bytes read + target bytes written",
                    "src_ranks": len(case.src.buf_bytes), "dst_ranks": len(case.dst.buf_bytes),
-                   "work_units": st["n_tiles"] + st["n_small_tiles"], "l2": "inputs_exceed_l2", "fill": case.fill,
+                   "work_units": st["n_tiles"] + st["n_small_tiles"],
+                   "l2": "inputs_exceed_l2" if flush is None else "flushed_before_every_step_512MiB", "fill": case.fill,
                    "multi_gpu": "replicas only", "plan_opts": opts, "plan_ms": plan_ms},
         "gbps_b_moved": b_moved * ws / (ms_step * 1e-3) / 1e9,
         "pct_of_8tbs_nominal": value / ws / 8000.0 * 100.0,
