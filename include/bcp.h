@@ -133,7 +133,12 @@ typedef struct {
                                error; 1: saved entries with IDENTICAL boxes are replicas (a checkpoint saved
                                without de-duplication): the first in input order is read, the others are
                                ignored; boxes that overlap only partly are still BCP_ERR_OVERLAP        */
-  uint32_t reserved[2];    /* must be 0 */
+  uint32_t tma_wait_ms;     /* TMA path: how long a CTA waits for one stage to fill before it gives up and
+                               raises BCP_ERR_DEVICE_TIMEOUT (measured with the device's global timer);
+                               default 2000                                                             */
+  uint32_t test_stall;      /* test hook, 0 in normal use: 1 makes the first CTA of the TMA kernel arm its
+                               first stage for more bytes than it loads, so that exactly one bounded wait
+                               runs out and the time-out path can be exercised without any fault          */
 } bcp_plan_opts;
 
 typedef struct bcp_plan bcp_plan_t;

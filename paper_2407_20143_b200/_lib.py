@@ -44,7 +44,8 @@ class PlanOptsC(C.Structure):
         ("worker", C.c_uint32),
         ("tma_min_row_bytes", C.c_uint32),
         ("allow_replicas", C.c_uint32),
-        ("reserved", C.c_uint32 * 2),
+        ("tma_wait_ms", C.c_uint32),
+        ("test_stall", C.c_uint32),
     ]
 
 

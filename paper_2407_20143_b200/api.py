@@ -153,7 +153,7 @@ def bcp_plan(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas: Seque
     if opts:
         o = L.PlanOptsC()
         for k, v in opts.items():
-            if not hasattr(o, k) or k == "reserved":
+            if not hasattr(o, k):
                 raise BcpError(ERR_INVALID, f"unknown plan option {k}")
             setattr(o, k, v)
     h = C.c_void_p()

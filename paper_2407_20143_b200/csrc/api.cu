@@ -167,7 +167,8 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
     t.stage_bytes = p->opt.tma_stage_bytes;
     t.n_stages = p->opt.tma_stages;
     t.grid = uint32_t(n_tma < p->tma_grid ? n_tma : p->tma_grid);
-    t.wait_limit = 1u << 20;
+    t.wait_ns = uint64_t(p->opt.tma_wait_ms) * 1000000ull;
+    t.test_stall = p->opt.test_stall;
     t.cache_hints = p->opt.cache_hints;
     t.maps = p->d_maps;
     BCP_CUDA(launch_tma(t, stream));

@@ -41,7 +41,8 @@ struct TmaLaunchArgs {
   uint32_t stage_bytes;   // shared-memory stage, multiple of 128
   uint32_t n_stages;      // 2..8
   uint32_t grid;
-  uint32_t wait_limit;    // mbarrier polls before a CTA gives up
+  uint64_t wait_ns;       // how long a CTA waits for one stage before it gives up (global timer)
+  uint32_t test_stall;    // test hook: CTA 0 over-arms its first stage so that one wait runs out
   uint32_t cache_hints;   // 3: evict-first stores; 4: evict-first loads too; else none
   const void* maps;       // device: two 128-byte tensor maps (source view, target view) per tensor-map rectangle
 };

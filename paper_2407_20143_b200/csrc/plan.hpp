@@ -39,6 +39,8 @@ struct Options {
   uint32_t worker = 0;  // 0: chosen from the work list
   uint32_t tma_min_row_bytes = 512;
   uint32_t allow_replicas = 0;
+  uint32_t tma_wait_ms = 2000;
+  uint32_t test_stall = 0;
 };
 
 // A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source

@@ -35,8 +35,6 @@ int fail(int code, const char* fmt, ...) {
 int parse_options(const bcp_plan_opts* in, Options* out) {
   Options o;
   if (in) {
-    for (uint32_t r : in->reserved)
-      if (r) return fail(BCP_ERR_INVALID, "bcp_plan_opts.reserved must be zero");
     if (in->tile_bytes) o.tile_bytes = in->tile_bytes;
     if (in->small_bytes) o.small_bytes = in->small_bytes;
     if (in->block_threads) o.block_threads = in->block_threads;
@@ -51,6 +49,8 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->worker) o.worker = in->worker;
     if (in->tma_min_row_bytes) o.tma_min_row_bytes = in->tma_min_row_bytes;
     o.allow_replicas = in->allow_replicas;
+    if (in->tma_wait_ms) o.tma_wait_ms = in->tma_wait_ms;
+    o.test_stall = in->test_stall;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -70,6 +70,8 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.cache_hints < 1 || o.cache_hints > 4) return fail(BCP_ERR_INVALID, "cache_hints must be in [1, 4]");
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
   if (o.allow_replicas > 1) return fail(BCP_ERR_INVALID, "allow_replicas must be 0 or 1");
+  if (o.test_stall > 1) return fail(BCP_ERR_INVALID, "test_stall must be 0 or 1");
+  if (o.tma_wait_ms > 60000) return fail(BCP_ERR_INVALID, "tma_wait_ms must not exceed 60000");
   if (o.worker > 2) return fail(BCP_ERR_INVALID, "worker must be 0, 1 or 2");
   if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
     return fail(BCP_ERR_INVALID, "tma_min_row_bytes must be a multiple of 16 in [16, 65536]");

@@ -42,6 +42,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -232,7 +238,8 @@ __device__ __forceinline__ void warp_store_out(const unsigned char* smem, char* 
 __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles,
                                                      const void* const* __restrict__ src, void* const* __restrict__ dst,
                                                      Control* ctrl, uint32_t stage_bytes, uint32_t n_stages,
-                                                     uint32_t wait_limit, uint32_t hints, const unsigned char* maps) {
+                                                     uint64_t wait_ns, uint32_t hints, const unsigned char* maps,
+                                                     uint32_t test_stall) {
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full[kMaxStages];
   __shared__ Chunk held[kMaxStages];
@@ -296,6 +303,7 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     return cur.next(stage_bytes, ch);
   };
 
+  uint32_t issued = 0, stored = 0;  // chunks whose load / store has been issued
   auto issue_load = [&](uint32_t stage, const Chunk& ch) {
     const uint32_t bar = smem_u32(&full[stage]);
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
@@ -340,7 +348,8 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     }
     if (lane == 0) {
       held[stage] = ch;
-      mbar_expect_tx(bar, ch.rows * ch.row_bytes);
+      // test hook: the very first stage of CTA 0 is armed for 16 bytes that never arrive
+      mbar_expect_tx(bar, ch.rows * ch.row_bytes + ((test_stall && blockIdx.x == 0 && issued == 0) ? 16u : 0u));
     }
     __syncwarp();
     for (uint32_t r = lane; r < ch.rows; r += 32) {
@@ -352,7 +361,6 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     }
   };
 
-  uint32_t issued = 0, stored = 0;  // chunks whose load / store has been issued
   Chunk ch;
   while (issued + 1 < n_stages && produce(&ch)) {  // prologue: S-1 loads in flight
     issue_load(issued % n_stages, ch);
@@ -362,18 +370,21 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     const uint32_t stage = stored % n_stages;
     const uint32_t parity = (stored / n_stages) & 1;
     const uint32_t bar = smem_u32(&full[stage]);
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-      if (++spins >= wait_limit) {
-        failed = true;
-        break;
+    if (!mbar_try_wait(bar, parity)) {  // bounded by the global timer, whatever one poll costs
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(bar, parity)) {
+        if (global_timer_ns() - t0 > wait_ns) {
+          failed = true;
+          break;
+        }
       }
     }
     if (failed) {
       // give the loads still in flight a bounded chance to land before the CTA leaves
+      const uint64_t t0 = global_timer_ns();
       for (uint32_t k = stored + 1; k < issued; ++k) {
         const uint32_t b2 = smem_u32(&full[k % n_stages]);
-        for (uint32_t w = 0; w < wait_limit && !mbar_try_wait(b2, (k / n_stages) & 1); ++w) {
+        while (!mbar_try_wait(b2, (k / n_stages) & 1) && global_timer_ns() - t0 <= wait_ns) {
         }
       }
       break;
@@ -469,7 +480,8 @@ cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream) {
   if (a.n_stages < 2 || a.n_stages > kMaxStages || a.stage_bytes % 128 || a.stage_bytes == 0) return cudaErrorInvalidValue;
   const size_t smem = size_t(a.stage_bytes) * a.n_stages;
   bcp_tma_kernel<<<a.grid, 32, smem, stream>>>(a.tiles, a.n_tiles, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages,
-                                               a.wait_limit, a.cache_hints, static_cast<const unsigned char*>(a.maps));
+                                               a.wait_ns, a.cache_hints, static_cast<const unsigned char*>(a.maps),
+                                               a.test_stall);
   return cudaGetLastError();
 }
 

@@ -143,6 +143,36 @@ def test_plans_with_different_ring_sizes_interleave(cuda_device):
         assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)) and guards_intact(backs, case.dst.buf_bytes)
 
 
+def test_bounded_wait_runs_out_and_is_reported(cuda_device):
+    """Failure detection without a fault: a test hook arms one stage of one CTA for bytes that
+    never arrive; that CTA's bounded wait gives up after 20 ms, the kernel ends, the status call
+    reports BCP_ERR_DEVICE_TIMEOUT, and the context and the library stay usable."""
+    from paper_2407_20143_b200 import api
+
+    case = _dim1_split_case((4096, 8192), 2, 1, 1)  # 64 MB, all aligned runs
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device)
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    stalled = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3,
+                           test_stall=1, tma_wait_ms=20)
+    dst, _ = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(stalled, src, dst)
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.bcp_plan_device_status(stalled)
+    assert e.value.code == api.ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()  # no sticky error: the kernel returned normally
+    got = dst[0].cpu().numpy()
+    missing = int((got != want[0]).sum())
+    assert 0 < missing <= 2 * 65536 + 32768, "only the unit the stalled CTA held may be incomplete"
+    bcp.bcp_plan_device_status(stalled)  # the status word was cleared by the report
+    # an ordinary plan on the same device right afterwards is exact
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3)
+    dst2, backs = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(plan, src, dst2)
+    torch.cuda.synchronize()
+    bcp.bcp_plan_device_status(plan)
+    assert np.array_equal(dst2[0].cpu().numpy(), want[0]) and guards_intact(backs, case.dst.buf_bytes)
+
+
 def test_side_stream_and_plan_reuse(cuda_device):
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
