@@ -30,6 +30,11 @@
  *   - `stream` arguments are CUDA stream handles (cudaStream_t) passed as void*;
  *     NULL is the legacy default stream.
  *   - Nothing here throws, aborts or traps the device.
+ *   - Threads: a plan, a stager and the fixed scratch of bcp_pack_static each serve one
+ *     call at a time; different plans may be used from different threads concurrently.
+ *     bcp_pack / bcp_unpack serialise themselves (their cache of work lists is shared).
+ *   - Source and target buffers of one call must not overlap: sources are read through the
+ *     read-only data path.
  */
 #ifndef BCP_H_
 #define BCP_H_
