@@ -513,12 +513,9 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
         avail = psutil.virtual_memory().available
     except Exception:
         avail = None
-    free, _ = torch.cuda.mem_get_info()
     reason = None
     if avail is not None and avail < (h2d + d2h) * ws * 1.15 + (8 << 30):
         reason = f"host memory: {avail / 1e9:.0f} GB available, {(h2d + d2h) * ws / 1e9:.0f} GB of pinned buffers needed"
-    if free < h2d + d2h + (2 << 30):
-        reason = f"device memory: {free / 1e9:.0f} GB free, {(h2d + d2h) / 1e9:.0f} GB of staging needed"
     ok = D.max_over_ranks(1.0 if reason else 0.0, dev) == 0.0
     if not ok:
         return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -540,8 +537,13 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     D.barrier()
     ms = D.max_over_ranks(e0.elapsed_time(e1) / a.e2e_steps, dev)
     same = all(bool(torch.equal(h[: 1 << 20], d[: 1 << 20].cpu())) for h, d in zip(hdst, dst))
-    return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same}
+    # pinned buffers are addressed by the kernels directly: every unit's source bytes cross PCIe when
+    # it is copied (replica reads cross again), every target byte crosses once on its way out
+    moved_in = plan.stats()["bytes_copied"]
+    return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": moved_in, "d2h_bytes_per_step": d2h,
+            "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same,
+            "mode": "pinned host buffers read and written in place by the kernels (no staging copy)",
+            "host_buffer_bytes": {"sources": h2d, "targets": d2h}}
 
 
 if __name__ == "__main__":

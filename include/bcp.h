@@ -290,12 +290,17 @@ BCP_API int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n
                 void* const* dst_bufs, size_t n_dst_bufs, void* stream);
 
 /*
- * Same operation with HOST buffers (host pointers to host memory, pinned for full speed):
- * copies the source blobs to plan-owned device staging memory, runs the kernels and
- * copies the target buffers back, then waits for completion.  Work is pipelined per target
- * buffer over three streams (`stream` for the kernels, two plan-owned streams for uploads and
- * downloads), so that downloads of finished target buffers overlap the uploads still
- * needed by later ones.  Target bytes not named by any target entry come back as zero.
+ * Same operation with HOST buffers (host pointers to host memory); returns when every target
+ * buffer is complete.  Target bytes not named by any target entry come back as zero.
+ *   - If every buffer is page-locked memory the device can address (cudaHostAlloc,
+ *     cudaHostRegister, torch pin_memory), nothing is staged: the kernels read the sources
+ *     and write the targets in place, so data crosses PCIe in both directions at the same
+ *     time and each byte crosses once per use.
+ *   - Otherwise the source blobs are copied to plan-owned device staging memory, the kernels
+ *     run there and the target buffers are copied back; the work is pipelined per target
+ *     buffer over three streams (`stream` for the kernels, two plan-owned streams for uploads
+ *     and downloads), so that downloads of finished target buffers overlap the uploads still
+ *     needed by later ones.
  */
 BCP_API int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
                      void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);

@@ -19,6 +19,7 @@ struct bcp_plan {
   size_t n_tma = 0, n_big = 0;
   std::vector<uint64_t> src_bytes, dst_bytes;
   std::vector<Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
+  std::vector<Gap> gaps;    // target bytes no entry names (zeroed by the host-buffer call)
   std::vector<CUtensorMap> h_maps;
   CUtensorMap* d_maps = nullptr;
   // device side, created by the first execution
@@ -486,13 +487,15 @@ int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_by
   if (int rc = parse_options(opts, &opt)) return rc;
   try {
     std::vector<Item> items;
+    std::vector<Gap> gaps;
     bcp_plan_stats_t st;
     memset(&st, 0, sizeof st);
-    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt.allow_replicas != 0, &items, &st))
+    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt.allow_replicas != 0, &items, &gaps, &st))
       return rc;
     bcp_plan_t* p = finish_plan(items, opt, st, std::vector<uint64_t>(src_buf_bytes, src_buf_bytes + n_src_bufs),
                               std::vector<uint64_t>(dst_buf_bytes, dst_buf_bytes + n_dst_bufs));
     if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
+    p->gaps = std::move(gaps);
     if (p->tiles.size() > 0xFFFF0000ull) {
       delete p;
       return fail(BCP_ERR_INVALID, "work list too long for one launch");
@@ -518,7 +521,7 @@ struct ImageHeader {
   uint32_t version, tile_size;
   Options opt;
   bcp_plan_stats_t stats;
-  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects;
+  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects, n_gaps;
 };
 uint64_t fnv1a(const unsigned char* p, size_t n) {
   uint64_t h = 1469598103934665603ull;
@@ -578,7 +581,8 @@ bool rect_ok(const Rect& r, const std::vector<uint64_t>& sb, const std::vector<u
 int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n) {
   if (!plan || !n) return fail(BCP_ERR_INVALID, "bcp_plan_serialize: NULL argument");
   const size_t need = sizeof(ImageHeader) + (plan->src_bytes.size() + plan->dst_bytes.size()) * sizeof(uint64_t) +
-                      plan->tiles.size() * sizeof(bcp_tile) + plan->rects.size() * sizeof(Rect) + sizeof(uint64_t);
+                      plan->tiles.size() * sizeof(bcp_tile) + plan->rects.size() * sizeof(Rect) + plan->gaps.size() * sizeof(Gap) +
+                      sizeof(uint64_t);
   *n = need;
   if (!out || cap < need) return fail(BCP_ERR_CAPACITY, "bcp_plan_serialize: image needs %zu bytes, room for %zu", need, out ? cap : size_t(0));
   ImageHeader h;
@@ -594,6 +598,7 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   h.n_big = plan->n_big;
   h.n_tiles = plan->tiles.size();
   h.n_rects = plan->rects.size();
+  h.n_gaps = plan->gaps.size();
   unsigned char* p = static_cast<unsigned char*>(out);
   memcpy(p, &h, sizeof h);
   p += sizeof h;
@@ -605,6 +610,8 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   p += h.n_tiles * sizeof(bcp_tile);
   if (h.n_rects) memcpy(p, plan->rects.data(), h.n_rects * sizeof(Rect));
   p += h.n_rects * sizeof(Rect);
+  if (h.n_gaps) memcpy(p, plan->gaps.data(), h.n_gaps * sizeof(Gap));
+  p += h.n_gaps * sizeof(Gap);
   const uint64_t sum = fnv1a(static_cast<unsigned char*>(out), size_t(p - static_cast<unsigned char*>(out)));
   memcpy(p, &sum, sizeof sum);
   return BCP_OK;
@@ -619,11 +626,11 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   if (h.version != uint32_t(bcp_version()) || h.tile_size != sizeof(bcp_tile))
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image of library version %u, this is %d", h.version, bcp_version());
   const uint64_t lim = uint64_t(1) << 32;
-  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_rects >= lim || h.n_tma > h.n_tiles ||
+  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_rects >= lim || h.n_gaps >= lim || h.n_tma > h.n_tiles ||
       h.n_big > h.n_tiles - h.n_tma)
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: implausible counts");
   const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) +
-                        h.n_rects * sizeof(Rect) + sizeof(uint64_t);
+                        h.n_rects * sizeof(Rect) + h.n_gaps * sizeof(Gap) + sizeof(uint64_t);
   if (need != n) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image is %zu bytes, its header implies %llu", n, (unsigned long long)need);
   const unsigned char* base = static_cast<const unsigned char*>(image);
   uint64_t sum;
@@ -655,11 +662,20 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
     q += h.n_tiles * sizeof(bcp_tile);
     p->rects.resize(h.n_rects);
     if (h.n_rects) memcpy(p->rects.data(), q, h.n_rects * sizeof(Rect));
+    q += h.n_rects * sizeof(Rect);
+    p->gaps.resize(h.n_gaps);
+    if (h.n_gaps) memcpy(p->gaps.data(), q, h.n_gaps * sizeof(Gap));
     p->n_tma = h.n_tma;
     p->n_big = h.n_big;
   } catch (const std::bad_alloc&) {
     delete p;
     return fail(BCP_ERR_NOMEM, "out of host memory");
+  }
+  for (const Gap& g : p->gaps) {  // gaps are zeroed in host memory: they must stay inside their buffer
+    if (g.buf >= p->dst_bytes.size() || g.off > p->dst_bytes[g.buf] || g.len > p->dst_bytes[g.buf] - g.off) {
+      delete p;
+      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: a gap lies outside its target buffer");
+    }
   }
   for (size_t i = 0; i < p->rects.size(); ++i) {
     if (!rect_ok(p->rects[i], p->src_bytes, p->dst_bytes)) {
@@ -705,8 +721,36 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
   for (size_t i = 0; i < n_dst_bufs; ++i)
     if (plan->dst_bytes[i] && !dst_host[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
   if (int rc = bind_device(plan)) return rc;
-  if (int rc = prepare_host_path(plan)) return rc;
   bcp_plan_t* p = plan;
+  // Pinned (or registered) host memory is addressable from the device: then the kernels read the
+  // sources and write the targets in place, over PCIe in both directions at once, and no staging
+  // copy exists at all.  Anything else goes through device staging buffers.
+  {
+    std::vector<const void*> dsrc(n_src_bufs, nullptr);
+    std::vector<void*> ddst(n_dst_bufs, nullptr);
+    bool mapped = true;
+    auto device_view = [&](const void* host, void** out) {
+      cudaPointerAttributes a;
+      if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+      }
+      if (a.type != cudaMemoryTypeHost || !a.devicePointer || (reinterpret_cast<uintptr_t>(a.devicePointer) & 15)) return false;
+      *out = a.devicePointer;
+      return true;
+    };
+    for (size_t i = 0; mapped && i < n_src_bufs; ++i)
+      if (p->src_bytes[i]) mapped = device_view(src_host[i], const_cast<void**>(&dsrc[i]));
+    for (size_t i = 0; mapped && i < n_dst_bufs; ++i)
+      if (p->dst_bytes[i]) mapped = device_view(dst_host[i], &ddst[i]);
+    if (mapped) {
+      for (const Gap& g : p->gaps) memset(static_cast<char*>(dst_host[g.buf]) + g.off, 0, g.len);
+      if (int rc = execute(p, dsrc.data(), n_src_bufs, ddst.data(), n_dst_bufs, stream)) return rc;
+      BCP_CUDA(cudaStreamSynchronize(stream));
+      return BCP_OK;
+    }
+  }
+  if (int rc = prepare_host_path(plan)) return rc;
   // device-side pointer table: the staging buffers
   for (size_t i = 0; i < n_src_bufs; ++i) p->h_ptrs[i] = p->stage_src[i];
   for (size_t i = 0; i < n_dst_bufs; ++i) p->h_ptrs[n_src_bufs + i] = p->stage_dst[i];

@@ -50,6 +50,12 @@ struct Rect {
   uint32_t row_bytes, src_buf, dst_buf, box_rows;
 };
 
+// Bytes of a target buffer that no target entry names.
+struct Gap {
+  uint64_t off, len;
+  uint32_t buf, pad;
+};
+
 int parse_options(const bcp_plan_opts* in, Options* out);
 
 // Irregular-tensor decomposition (Sec. 3.2): boxes relative to the local tensor, flat order.
@@ -63,7 +69,7 @@ void decompose(const int64_t* lengths, uint32_t ndim, int64_t a, int64_t b, std:
 // counters of `stats`.
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    bool allow_replicas, std::vector<Item>* items, bcp_plan_stats_t* stats);
+                    bool allow_replicas, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats);
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
 // tiles = [TMA units..., other CTA-wide units..., warp units...].

@@ -349,7 +349,7 @@ struct SegKey {  // identity of a matched segment on the saved side (for the uni
 
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    bool allow_replicas, std::vector<Item>* items, bcp_plan_stats_t* stats) {
+                    bool allow_replicas, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
   if ((n_src && !src) || (n_dst && !dst) || (n_src_bufs && !src_buf_bytes) || (n_dst_bufs && !dst_buf_bytes))
     return fail(BCP_ERR_INVALID, "bcp_plan: NULL array with non-zero count");
   std::unordered_map<std::string, uint32_t> ids;
@@ -405,6 +405,17 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       if (rs[i].buf == rs[i - 1].buf && rs[i].lo < rs[i - 1].hi)
         return fail(BCP_ERR_DST_ALIAS, "dst[%u] %s and dst[%u] %s write overlapping bytes of buffer %u", rs[i - 1].meta,
                     dst[rs[i - 1].meta].fqn, rs[i].meta, dst[rs[i].meta].fqn, rs[i].buf);
+    if (gaps) {  // what no entry names: between the sorted ranges, and whole buffers without entries
+      size_t i = 0;
+      for (uint32_t b = 0; b < n_dst_bufs; ++b) {
+        uint64_t pos = 0;
+        for (; i < rs.size() && rs[i].buf == b; ++i) {
+          if (rs[i].lo > pos) gaps->push_back(Gap{pos, rs[i].lo - pos, b, 0});
+          pos = rs[i].hi;
+        }
+        if (dst_buf_bytes[b] > pos) gaps->push_back(Gap{pos, dst_buf_bytes[b] - pos, b, 0});
+      }
+    }
   }
   std::vector<SegKey> segs;
   uint64_t n_inter = 0, n_se = 0, n_de = 0;
