@@ -141,6 +141,11 @@ typedef struct {
   uint32_t tma_wait_ms;     /* TMA path: how long a CTA waits for one stage to fill before it gives up and
                                raises BCP_ERR_DEVICE_TIMEOUT (measured with the device's global timer);
                                default 2000                                                             */
+  uint32_t fanout;          /* 0 default (= 1); 1: TMA units that read the same source bytes (replicas of a
+                               target shard; needs order 1) are grouped, the source is staged once and
+                               written to every member's target (fewer L2 reads; over PCIe, fewer reads
+                               at all); 2: every unit is staged on its own (bcp_reshard_host still groups
+                               when it works in place)                                                     */
   uint32_t test_stall;      /* test hook, 0 in normal use: 1 makes the first CTA of the TMA kernel arm its
                                first stage for more bytes than it loads, so that exactly one bounded wait
                                runs out and the time-out path can be exercised without any fault          */
@@ -174,6 +179,11 @@ typedef struct {
 #define BCP_TILE_TMA2D 0x40u    /* rows of a rectangle staged with 2-D tensor-map copies: reserved[0] =
                                    rectangle index + 1, reserved[1] = first row inside the rectangle,
                                    reserved[2] = rows per box                                    */
+#define BCP_TILE_FOLLOW 0x80u   /* TMA unit with the same source bytes as the unit before it in the list
+                                   (a replica of a target shard): the CTA that stages the first unit of
+                                   such a group writes every member's target from the one staged copy,
+                                   and whoever draws a follower's ticket skips it                 */
+#define BCP_TILE_FAN_SHIFT 8    /* bits 8..10 of a group's first unit: how many followers it has (0..7) */
 
 typedef struct {
   uint64_t n_src_entries;    /* after decomposing flat slices                        */

@@ -45,6 +45,7 @@ class PlanOptsC(C.Structure):
         ("tma_min_row_bytes", C.c_uint32),
         ("allow_replicas", C.c_uint32),
         ("tma_wait_ms", C.c_uint32),
+        ("fanout", C.c_uint32),
         ("test_stall", C.c_uint32),
     ]
 

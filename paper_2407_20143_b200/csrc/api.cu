@@ -25,6 +25,7 @@ struct bcp_plan {
   // device side, created by the first execution
   int device = -1;
   bcp_tile* d_tiles = nullptr;
+  bcp_tile* d_fan_tiles = nullptr;  // the same list with replica groups marked (in-place host path)
   void** d_ptrs = nullptr;  // source table followed by target table
   Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel
   uint32_t grid = 0, tma_grid = 0;
@@ -197,7 +198,8 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
   return BCP_OK;
 }
 
-int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, size_t nd, cudaStream_t stream) {
+int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, size_t nd, cudaStream_t stream,
+            const bcp_tile* list = nullptr) {
   if (!p) return fail(BCP_ERR_INVALID, "plan is NULL");
   if (ns != p->src_bytes.size() || nd != p->dst_bytes.size())
     return fail(BCP_ERR_INVALID, "buffer counts (%zu, %zu) differ from the planned (%zu, %zu)", ns, nd, p->src_bytes.size(),
@@ -224,7 +226,7 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
     for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
     if (int rc = upload_tables(p, stream)) return rc;
   }
-  if (int rc = launch_units(p, p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
+  if (int rc = launch_units(p, list ? list : p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
   p->last_stream = stream;
   p->ran = true;
   return BCP_OK;
@@ -356,7 +358,9 @@ int prepare_host_path(bcp_plan_t* p) {
   for (const bcp_tile& t : p->tiles) {
     const uint32_t d = t.dst_buf;
     if (!(t.flags & BCP_TILE_ZERO)) need[d][t.src_buf] = 1;
-    ((t.flags & BCP_TILE_TMA) ? tma : (t.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(t);
+    bcp_tile u = t;
+    u.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));  // groups are per target buffer here: every unit is staged on its own
+    ((u.flags & BCP_TILE_TMA) ? tma : (u.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(u);
   }
   std::vector<bcp_tile> flat;
   flat.reserve(p->tiles.size());
@@ -683,6 +687,18 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
       return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: rectangle %zu is inconsistent with the recorded buffers", i);
     }
   }
+  {  // replica groups must be exactly what the planner would mark: a follower is never staged itself
+    std::vector<bcp_tile> again(p->tiles.begin(), p->tiles.begin() + p->n_tma);
+    for (bcp_tile& t : again) t.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));
+    if (p->opt.fanout == 1 && p->opt.order == 1) mark_followers(again.data(), again.size());
+    bool ok = true;
+    for (size_t i = 0; ok && i < p->tiles.size(); ++i)
+      ok = i < p->n_tma ? again[i].flags == p->tiles[i].flags : !(p->tiles[i].flags & (BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT)));
+    if (!ok) {
+      delete p;
+      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: replica groups of the work list are inconsistent");
+    }
+  }
   for (size_t i = 0; i < p->tiles.size(); ++i) {
     const bcp_tile& t = p->tiles[i];
     const bool in_tma = i < p->n_tma, in_small = i >= p->n_tma + p->n_big;
@@ -744,8 +760,15 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
     for (size_t i = 0; mapped && i < n_dst_bufs; ++i)
       if (p->dst_bytes[i]) mapped = device_view(dst_host[i], &ddst[i]);
     if (mapped) {
+      // over PCIe every read costs: stage each source piece once and write all its replicas from it
+      if (!p->d_fan_tiles && p->n_tma && p->opt.order == 1 && p->opt.fanout != 1) {
+        std::vector<bcp_tile> fan(p->tiles);
+        mark_followers(fan.data(), p->n_tma);
+        BCP_CUDA(cudaMalloc(&p->d_fan_tiles, fan.size() * sizeof(bcp_tile)));
+        BCP_CUDA(cudaMemcpy(p->d_fan_tiles, fan.data(), fan.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
+      }
       for (const Gap& g : p->gaps) memset(static_cast<char*>(dst_host[g.buf]) + g.off, 0, g.len);
-      if (int rc = execute(p, dsrc.data(), n_src_bufs, ddst.data(), n_dst_bufs, stream)) return rc;
+      if (int rc = execute(p, dsrc.data(), n_src_bufs, ddst.data(), n_dst_bufs, stream, p->d_fan_tiles)) return rc;
       BCP_CUDA(cudaStreamSynchronize(stream));
       return BCP_OK;
     }
@@ -825,6 +848,7 @@ int bcp_plan_destroy(bcp_plan_t* plan) {
     for (void* q : plan->stage_dst) cudaFree(q);
     cudaFree(plan->d_host_tiles);
     cudaFree(plan->d_tiles);
+    cudaFree(plan->d_fan_tiles);
     cudaFree(plan->d_ptrs);
     cudaFree(plan->d_ctrl);
     cudaFree(plan->d_maps);

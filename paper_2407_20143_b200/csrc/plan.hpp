@@ -41,6 +41,7 @@ struct Options {
   uint32_t allow_replicas = 0;
   uint32_t tma_wait_ms = 2000;
   uint32_t test_stall = 0;
+  uint32_t fanout = 1;  // 1 on, 2 off
 };
 
 // A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source
@@ -73,6 +74,9 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
 // tiles = [TMA units..., other CTA-wide units..., warp units...].
+// Mark groups of TMA units (ordered by source address) that read the same source bytes.
+void mark_followers(bcp_tile* tma, size_t n);
+
 // src_bytes: sizes of the source buffers (bounds for over-reading aligned supersets).
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
                  std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,

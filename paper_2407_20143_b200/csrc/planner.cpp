@@ -51,6 +51,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     o.allow_replicas = in->allow_replicas;
     if (in->tma_wait_ms) o.tma_wait_ms = in->tma_wait_ms;
     o.test_stall = in->test_stall;
+    if (in->fanout) o.fanout = in->fanout;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -71,6 +72,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.unroll != 4 && o.unroll != 8) return fail(BCP_ERR_INVALID, "unroll must be 4 or 8");
   if (o.allow_replicas > 1) return fail(BCP_ERR_INVALID, "allow_replicas must be 0 or 1");
   if (o.test_stall > 1) return fail(BCP_ERR_INVALID, "test_stall must be 0 or 1");
+  if (o.fanout != 1 && o.fanout != 2) return fail(BCP_ERR_INVALID, "fanout must be 0, 1 or 2");
   if (o.tma_wait_ms > 60000) return fail(BCP_ERR_INVALID, "tma_wait_ms must not exceed 60000");
   if (o.worker > 2) return fail(BCP_ERR_INVALID, "worker must be 0, 1 or 2");
   if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
@@ -635,6 +637,29 @@ struct Cutter {
 
 }  // namespace
 
+// Read once, write many: TMA units that read exactly the same source bytes (the replicas of a
+// target shard) sit next to each other in a list ordered by source address.  All but the first
+// of such a group (up to 8 members) are marked as followers and the first one records how many
+// follow; the kernel stages the source once and stores it to every member's target.
+void mark_followers(bcp_tile* tma, size_t n) {
+  size_t head = 0;
+  for (size_t i = 1; i < n; ++i) {
+    const bcp_tile& a = tma[i - 1];
+    bcp_tile& b = tma[i];
+    const uint32_t plain = ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));
+    // (equal flags include the access width, so one copy-out width suits every member's target)
+    const bool same = a.src_buf == b.src_buf && a.src_off == b.src_off && a.rows == b.rows && a.row_bytes == b.row_bytes &&
+                      a.src_pitch == b.src_pitch && (a.flags & plain) == (b.flags & plain) && (b.flags & BCP_TILE_TMA) &&
+                      (!(b.flags & BCP_TILE_TMA2D) || a.reserved[2] == b.reserved[2]);
+    if (same && i - head < 8) {
+      b.flags |= BCP_TILE_FOLLOW;
+      tma[head].flags = (tma[head].flags & ~(7u << BCP_TILE_FAN_SHIFT)) | (uint32_t(i - head) << BCP_TILE_FAN_SHIFT);
+    } else {
+      head = i;
+    }
+  }
+}
+
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
                  std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,
                  bcp_plan_stats_t* stats) {
@@ -725,6 +750,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
       std::sort(v->begin(), v->end(), by_dst);
     }
   }
+  if (opt.order == 1 && opt.fanout == 1) mark_followers(c.tma.data(), c.tma.size());
   stats->n_tiles = c.tma.size() + c.big.size();
   stats->n_small_tiles = c.small.size();
   *n_tma = c.tma.size();

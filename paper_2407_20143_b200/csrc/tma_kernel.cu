@@ -119,6 +119,8 @@ __device__ __forceinline__ void bulk_wait_read() {
 
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+constexpr int kMaxFan = 7;  // followers a unit can carry (targets written from the same staged bytes)
+
 struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memory
   const char* src;
   char* dst;
@@ -127,6 +129,16 @@ struct Chunk {  // what one stage holds: rows x row_bytes, dense in shared memor
   uint32_t shift;  // shifted run only: payload starts `shift` bytes into the stage
   uint32_t width;  // 0: aligned chunk, stored with bulk copies; 1..4: shifted run, log2 of the store width + 1;
                    // kTensor: one box of a tensor map (src / dst hold the descriptors, rows = box rows, shift = first row)
+  // replicas: nf further targets receive the same bytes; their addresses live in fan slot `slot`, and
+  // this chunk starts at row r0, byte c0 of the unit
+  uint32_t nf, slot, r0, c0;
+};
+
+// Follower targets of one unit (same geometry as the head, own address / descriptor and pitch).
+struct Fan {
+  char* dst[kMaxFan];      // target base address (tensor-map rectangles: target descriptor)
+  uint64_t pitch[kMaxFan];
+  uint32_t row0[kMaxFan];  // tensor-map rectangles: first row of the unit inside the follower's rectangle
 };
 constexpr uint32_t kShiftedRows = 4;  // width codes 5..8: several shifted rows per chunk, `shift` = bytes per row slot
 constexpr uint32_t kTensor = 9;
@@ -140,7 +152,15 @@ struct TileCursor {
   uint32_t r, c;  // next row, next byte inside the row
   uint32_t width;  // 0 aligned tile; 1..4 log2(access width) + 1 of a shifted run; kTensor: tensor-map rectangle
   uint32_t box_rows, row0;  // tensor-map rectangle: rows per box, first row of this unit inside the rectangle
+  uint32_t nf, slot;        // followers of this unit and the fan slot that holds their targets
   bool live;
+
+  __device__ __forceinline__ void fan(Chunk* out, uint32_t row, uint32_t col) const {
+    out->nf = nf;
+    out->slot = slot;
+    out->r0 = row;
+    out->c0 = col;
+  }
 
   __device__ __forceinline__ bool next(uint32_t stage_bytes, Chunk* out) {
     if (!live) return false;
@@ -154,6 +174,7 @@ struct TileCursor {
       out->sp = out->dp = 0;
       out->shift = row0 + r;
       out->width = kTensor;
+      fan(out, r, 0);
       r += min(box_rows, rows - r);
       if (r == rows) live = false;
       return true;
@@ -170,6 +191,7 @@ struct TileCursor {
         out->dp = dp;
         out->shift = slot;
         out->width = width + kShiftedRows;
+        fan(out, r, 0);
         r += k;
         if (r == rows) live = false;
         return true;
@@ -183,6 +205,7 @@ struct TileCursor {
       out->sp = out->dp = 0;
       out->shift = uint32_t(reinterpret_cast<uintptr_t>(out->src) & 15);
       out->width = width;
+      fan(out, r, c);
       c += n;
       if (c == row_bytes) {
         c = 0;
@@ -198,6 +221,7 @@ struct TileCursor {
       out->rows = 1;
       out->row_bytes = n;
       out->sp = out->dp = 0;
+      fan(out, r, c);
       c += n;
       if (c == row_bytes) {
         c = 0;
@@ -211,6 +235,7 @@ struct TileCursor {
       out->row_bytes = row_bytes;
       out->sp = sp;
       out->dp = dp;
+      fan(out, r, 0);
       r += k;
     }
     if (r == rows) live = false;
@@ -243,6 +268,8 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full[kMaxStages];
   __shared__ Chunk held[kMaxStages];
+  __shared__ Fan fans[kMaxStages + 1];  // chunks in flight span at most n_stages units
+  uint32_t fan_next = 0;
   const uint32_t lane = threadIdx.x;
   const uint64_t pol = policy_evict_first();
   const bool hint_st = hints >= 3, hint_ld = hints >= 4;  // 3: stores evict-first; 4: loads too
@@ -270,6 +297,11 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
         return false;
       }
       const bcp_tile* t = tiles + ticket;
+      const uint4 e = __ldg(reinterpret_cast<const uint4*>(t) + 3);  // flags, reserved[0..2]
+      if (e.x & BCP_TILE_FOLLOW) {  // written by the CTA that stages the head of its group
+        if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
+        continue;
+      }
       const uint4 a = __ldg(reinterpret_cast<const uint4*>(t));
       const uint4 b = __ldg(reinterpret_cast<const uint4*>(t) + 1);
       const uint4 c = __ldg(reinterpret_cast<const uint4*>(t) + 2);
@@ -281,12 +313,10 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
       cur.rows = c.y;
       cur.r = cur.c = 0;
       cur.live = cur.rows > 0 && cur.row_bytes > 0;
-      // a run that is not 16-byte aligned on both sides and in length is staged as a shifted run
-      const uint32_t bits = a.x | a.z | c.x;  // low bits of src_off | dst_off | row_bytes (bases are 16-byte aligned)
+      // a piece that is not 16-byte aligned on both sides, in length and in its pitches is staged shifted
+      const uint32_t all = a.x | a.z | c.x | b.x | b.z;  // low bits (bases are 16-byte aligned)
       cur.width = 0;
-      const uint32_t all = bits | b.x | b.z;  // ... and of both pitches
       if (all & 15) cur.width = (all & 1) ? 1 : (all & 2) ? 2 : (all & 4) ? 3 : 4;
-      const uint4 e = __ldg(reinterpret_cast<const uint4*>(t) + 3);  // flags, reserved[0..2]
       if (e.x & BCP_TILE_TMA2D) {  // s / d name the rectangle's descriptors instead of addresses
         cur.width = kTensor;
         cur.s = reinterpret_cast<const char*>(maps + uint64_t(e.y - 1) * 256);
@@ -297,6 +327,30 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
           tensormap_acquire(cur.s);
           tensormap_acquire(cur.d);
         }
+      }
+      // followers: the head's flags say how many of the units right behind it read the same source bytes
+      cur.nf = (e.x >> BCP_TILE_FAN_SHIFT) & 7u;
+      if (cur.nf) {
+        cur.slot = fan_next;
+        fan_next = fan_next == n_stages ? 0 : fan_next + 1;
+        if (lane < cur.nf) {
+          const bcp_tile* f = tiles + ticket + 1 + lane;
+          const uint4 fe = __ldg(reinterpret_cast<const uint4*>(f) + 3);
+          const uint4 fa = __ldg(reinterpret_cast<const uint4*>(f));
+          const uint4 fb = __ldg(reinterpret_cast<const uint4*>(f) + 1);
+          const uint4 fc = __ldg(reinterpret_cast<const uint4*>(f) + 2);
+          Fan& fn = fans[cur.slot];
+          fn.pitch[lane] = uint64_t(fb.z) | (uint64_t(fb.w) << 32);
+          if (fe.x & BCP_TILE_TMA2D) {
+            fn.dst[lane] = const_cast<char*>(reinterpret_cast<const char*>(maps + uint64_t(fe.y - 1) * 256 + 128));
+            fn.row0[lane] = fe.z;
+            tensormap_acquire(fn.dst[lane]);
+          } else {
+            fn.dst[lane] = static_cast<char*>(dst[fc.w]) + (uint64_t(fa.z) | (uint64_t(fa.w) << 32));
+            fn.row0[lane] = 0;
+          }
+        }
+        __syncwarp();
       }
       if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);  // consumed when this tile is used up
     }
@@ -392,38 +446,54 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     __syncwarp();
     const Chunk h = held[stage];
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
-    if (h.width == kTensor) {
-      if (lane == 0) tensor_store_2d(h.dst, 0, int(h.shift), base);
-    } else if (h.width > kShiftedRows) {  // shifted rows: the warp copies row after row out of its slot
-      for (uint32_t r = 0; r < h.rows; ++r) {
-        const uint32_t sh = uint32_t(reinterpret_cast<uintptr_t>(h.src + uint64_t(r) * h.sp) & 15);
-        const unsigned char* p = stage_mem + stage * stage_bytes + r * h.shift + sh;
-        char* q = h.dst + uint64_t(r) * h.dp;
-        switch (h.width - kShiftedRows) {
-          case 4: warp_store_out<uint2>(p, q, h.row_bytes, lane); break;
-          case 3: warp_store_out<unsigned int>(p, q, h.row_bytes, lane); break;
-          case 2: warp_store_out<unsigned short>(p, q, h.row_bytes, lane); break;
-          default: warp_store_out<unsigned char>(p, q, h.row_bytes, lane); break;
+    // the head's target, then every follower's, all from the same staged bytes
+    for (uint32_t m = 0; m <= h.nf; ++m) {
+      char* mdst = h.dst;
+      uint64_t mdp = h.dp;
+      uint32_t mrow = h.shift;
+      if (m) {
+        const Fan& fn = fans[h.slot];
+        mdp = fn.pitch[m - 1];
+        mdst = fn.dst[m - 1];
+        if (h.width == kTensor) {
+          mrow = fn.row0[m - 1] + h.r0;
+        } else {
+          mdst += uint64_t(h.r0) * mdp + h.c0;
         }
       }
-      __syncwarp();
-    } else if (h.width) {  // shifted run: the warp copies the payload out of the stage
-      const unsigned char* p = stage_mem + stage * stage_bytes + h.shift;
-      switch (h.width) {
-        case 4: warp_store_out<uint2>(p, h.dst, h.row_bytes, lane); break;
-        case 3: warp_store_out<unsigned int>(p, h.dst, h.row_bytes, lane); break;
-        case 2: warp_store_out<unsigned short>(p, h.dst, h.row_bytes, lane); break;
-        default: warp_store_out<unsigned char>(p, h.dst, h.row_bytes, lane); break;
+      if (h.width == kTensor) {
+        if (lane == 0) tensor_store_2d(mdst, 0, int(mrow), base);
+      } else if (h.width > kShiftedRows) {  // shifted rows: the warp copies row after row out of its slot
+        for (uint32_t r = 0; r < h.rows; ++r) {
+          const uint32_t sh = uint32_t(reinterpret_cast<uintptr_t>(h.src + uint64_t(r) * h.sp) & 15);
+          const unsigned char* p = stage_mem + stage * stage_bytes + r * h.shift + sh;
+          char* q = mdst + uint64_t(r) * mdp;
+          switch (h.width - kShiftedRows) {
+            case 4: warp_store_out<uint2>(p, q, h.row_bytes, lane); break;
+            case 3: warp_store_out<unsigned int>(p, q, h.row_bytes, lane); break;
+            case 2: warp_store_out<unsigned short>(p, q, h.row_bytes, lane); break;
+            default: warp_store_out<unsigned char>(p, q, h.row_bytes, lane); break;
+          }
+        }
+      } else if (h.width) {  // shifted run: the warp copies the payload out of the stage
+        const unsigned char* p = stage_mem + stage * stage_bytes + h.shift;
+        switch (h.width) {
+          case 4: warp_store_out<uint2>(p, mdst, h.row_bytes, lane); break;
+          case 3: warp_store_out<unsigned int>(p, mdst, h.row_bytes, lane); break;
+          case 2: warp_store_out<unsigned short>(p, mdst, h.row_bytes, lane); break;
+          default: warp_store_out<unsigned char>(p, mdst, h.row_bytes, lane); break;
+        }
+      } else {  // aligned rows: one bulk store per row
+        for (uint32_t r = lane; r < h.rows; r += 32) {
+          if (hint_st) {
+            bulk_store_hint(mdst + uint64_t(r) * mdp, base + r * h.row_bytes, h.row_bytes, pol);
+          } else {
+            bulk_store(mdst + uint64_t(r) * mdp, base + r * h.row_bytes, h.row_bytes);
+          }
+        }
       }
-      __syncwarp();
     }
-    for (uint32_t r = lane; r < (h.width ? 0u : h.rows); r += 32) {
-      if (hint_st) {
-        bulk_store_hint(h.dst + uint64_t(r) * h.dp, base + r * h.row_bytes, h.row_bytes, pol);
-      } else {
-        bulk_store(h.dst + uint64_t(r) * h.dp, base + r * h.row_bytes, h.row_bytes);
-      }
-    }
+    if (h.width && h.width != kTensor) __syncwarp();
     bulk_commit();
     ++stored;
     // the stage of the previous store is free once that store has read its shared memory
@@ -464,8 +534,12 @@ cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_
   int optin = 0;
   e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  if (smem + 1024 > size_t(optin)) return cudaErrorInvalidValue;  // 1 KiB of static shared memory and slack
-  e = cudaFuncSetAttribute(bcp_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024);
+  cudaFuncAttributes fa;
+  e = cudaFuncGetAttributes(&fa, bcp_tma_kernel);
+  if (e != cudaSuccess) return e;
+  const int room = optin - int(fa.sharedSizeBytes);  // what the kernel's static shared memory leaves
+  if (room <= 0 || smem > size_t(room)) return cudaErrorInvalidValue;
+  e = cudaFuncSetAttribute(bcp_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, room);
   if (e != cudaSuccess) return e;
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bcp_tma_kernel, 32, smem);
   if (e != cudaSuccess) return e;

@@ -88,7 +88,8 @@ def test_big_random_misaligned(cuda_device, itemsize, seed, path_mask):
                                   dict(path_mask=1, worker=2, unroll=8, ctas_per_sm=4, tile_bytes=16384),
                                   dict(path_mask=3), dict(path_mask=3, tma_stage_bytes=4096, tma_stages=2, tile_bytes=32768),
                                   dict(path_mask=3, tma_stage_bytes=32768, tma_stages=6, tma_ctas_per_sm=1),
-                                  dict(path_mask=7), dict(path_mask=7, tile_bytes=8192, tma_stage_bytes=4096)])
+                                  dict(path_mask=7), dict(path_mask=7, tile_bytes=8192, tma_stage_bytes=4096),
+                                  dict(path_mask=7, fanout=2), dict(path_mask=3, fanout=1, tile_bytes=4096, tma_stage_bytes=2048, tma_stages=2)])
 def test_launch_options(cuda_device, opts):
     run_and_compare(CONFIGS["cfg1"]("index"), cuda_device, **opts)
     run_and_compare(big_random_case(11, itemsize=2), cuda_device, **opts)
@@ -124,6 +125,7 @@ def test_wide_strided_rows(cuda_device, opts):
 @pytest.mark.parametrize("case", scenario_cases()[:4] + scenario_cases()[8:10], ids=lambda c: c.name)
 def test_scenarios_tma_path(cuda_device, case):
     run_and_compare(case, cuda_device, path_mask=3, tile_bytes=16384, tma_stage_bytes=4096)
+    run_and_compare(case, cuda_device, path_mask=7, tile_bytes=8192, tma_min_row_bytes=64, fanout=1)
 
 
 def test_plans_with_different_ring_sizes_interleave(cuda_device):

@@ -37,7 +37,7 @@ def test_struct_sizes_match_header():
 
     assert C.sizeof(_lib.TileC) == 64
     assert C.sizeof(_lib.ShardMetaC) == 8 + 16 + 3 * 64 + 16 + 8 + 16
-    assert C.sizeof(_lib.PlanOptsC) == 64
+    assert C.sizeof(_lib.PlanOptsC) == 68
 
 
 # ---- decomposition (Sec. 3.2) ----------------------------------------------------------------------
@@ -257,6 +257,38 @@ def test_single_run_larger_than_4_gib_is_cut_without_overflow():
     order = sorted(tiles, key=lambda t: t.dst_off)
     assert order[0].dst_off == 0 and all(a.dst_off + a.row_bytes == b.dst_off for a, b in zip(order, order[1:]))
     assert all(t.src_off == t.dst_off + 16 for t in tiles) and order[-1].dst_off + order[-1].row_bytes == n
+
+
+def test_replica_units_follow_their_head():
+    """Units that read the same source bytes are grouped (read once, write many): followers sit
+    right behind a head with identical source geometry, at most 7 per head."""
+    case = scenario_cases()[2]  # dp4 -> dp8: every parameter shard is wanted by 8 data-parallel ranks
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3, tile_bytes=4096,
+                        tma_min_row_bytes=64, fanout=1)
+    tiles = plan.tiles()
+    heads = [i for i, t in enumerate(tiles) if (t.flags >> 8) & 7]
+    for i in heads:  # a head announces exactly the followers behind it
+        k = (tiles[i].flags >> 8) & 7
+        assert all(tiles[i + j].flags & api.TILE_FOLLOW for j in range(1, k + 1))
+        assert i + k + 1 == len(tiles) or not (tiles[i + k + 1].flags & api.TILE_FOLLOW)
+    n_follow, run = 0, 1
+    for prev, t in zip(tiles, tiles[1:]):
+        if t.flags & api.TILE_FOLLOW:
+            n_follow += 1
+            run += 1
+            assert run <= 8 and t.flags & api.TILE_TMA and prev.flags & api.TILE_TMA
+            assert (prev.src_buf, prev.src_off, prev.rows, prev.row_bytes, prev.src_pitch) == \
+                   (t.src_buf, t.src_off, t.rows, t.row_bytes, t.src_pitch)
+            assert (prev.dst_buf, prev.dst_off) != (t.dst_buf, t.dst_off)
+        else:
+            run = 1
+    assert n_follow > 0 and not (tiles[0].flags & api.TILE_FOLLOW)
+    assert not any(t.flags & api.TILE_FOLLOW for t in bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas,
+                                                                  case.dst.buf_bytes, path_mask=3, order=2, fanout=1).tiles())
+    assert not any(t.flags & api.TILE_FOLLOW for t in bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas,
+                                                                  case.dst.buf_bytes, path_mask=3, fanout=2).tiles())
+    again = bcp.Plan.deserialize(plan.serialize())
+    assert [_tile_tuple(t) for t in again.tiles()] == [_tile_tuple(t) for t in tiles]
 
 
 # ---- plan images (plan cache across processes, Sec. 4.1) ----------------------------------------------
