@@ -151,7 +151,7 @@ typedef struct {
                                runs out and the time-out path can be exercised without any fault          */
 } bcp_plan_opts;
 
-typedef struct bcp_plan bcp_plan_t;
+typedef struct bcp_plan_s bcp_plan_t;
 
 /*
  * One unit of the flat work list the planner produces and the kernels execute:

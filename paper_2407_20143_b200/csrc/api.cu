@@ -12,7 +12,7 @@
 
 using namespace bcp;
 
-struct bcp_plan {
+struct bcp_plan_s {
   Options opt;
   bcp_plan_stats_t stats;
   std::vector<bcp_tile> tiles;  // TMA units, then other CTA-wide units, then warp units
@@ -352,7 +352,7 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
 int prepare_host_path(bcp_plan_t* p) {
   if (p->s_h2d) return BCP_OK;
   const size_t ns = p->src_bytes.size(), nd = p->dst_bytes.size();
-  p->groups.assign(nd, bcp_plan::Group());
+  p->groups.assign(nd, bcp_plan_s::Group());
   std::vector<std::vector<bcp_tile>> tma(nd), big(nd), small(nd);
   std::vector<std::vector<char>> need(nd, std::vector<char>(ns, 0));
   for (const bcp_tile& t : p->tiles) {
@@ -365,7 +365,7 @@ int prepare_host_path(bcp_plan_t* p) {
   std::vector<bcp_tile> flat;
   flat.reserve(p->tiles.size());
   for (size_t d = 0; d < nd; ++d) {
-    bcp_plan::Group& g = p->groups[d];
+    bcp_plan_s::Group& g = p->groups[d];
     g.first = flat.size();
     g.n_tma = tma[d].size();
     g.n_big = big[d].size();
@@ -590,7 +590,7 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   *n = need;
   if (!out || cap < need) return fail(BCP_ERR_CAPACITY, "bcp_plan_serialize: image needs %zu bytes, room for %zu", need, out ? cap : size_t(0));
   ImageHeader h;
-  memset(&h, 0, sizeof h);
+  memset(static_cast<void*>(&h), 0, sizeof h);  // padding bytes too: images are compared and checksummed
   memcpy(h.magic, kMagic, 8);
   h.version = uint32_t(bcp_version());
   h.tile_size = sizeof(bcp_tile);
@@ -787,7 +787,7 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
   // download it.  Uploads, kernels and downloads sit on three streams, so the download of one
   // target buffer overlaps the uploads for the next (PCIe is full duplex).
   for (uint32_t d : p->order) {
-    const bcp_plan::Group& g = p->groups[d];
+    const bcp_plan_s::Group& g = p->groups[d];
     for (uint32_t sb : g.needs) {
       if (uploaded[sb]) continue;
       uploaded[sb] = 1;
