@@ -255,6 +255,9 @@ BCP_API int bcp_dedup_assign(const uint64_t* shard_bytes, const uint64_t* holder
  * On success *out_plan owns host (and, after the first bcp_reshard, device) copies of the
  * work list; release it with bcp_plan_destroy.  A plan holds no buffer addresses and can
  * be executed any number of times on any buffers of the planned sizes.
+ * Work lists of more than 32k units are built by several host threads (at most 8; the
+ * environment variable BCP_PLAN_THREADS, 1..64, overrides the count); the plan does not
+ * depend on how many.
  */
 BCP_API int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes,
              size_t n_src_bufs, const bcp_shard_meta* dst, size_t n_dst,

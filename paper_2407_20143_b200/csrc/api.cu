@@ -15,7 +15,7 @@ using namespace bcp;
 struct bcp_plan_s {
   Options opt;
   bcp_plan_stats_t stats;
-  std::vector<bcp_tile> tiles;  // TMA units, then other CTA-wide units, then warp units
+  TileVec tiles;  // TMA units, then other CTA-wide units, then warp units
   size_t n_tma = 0, n_big = 0;
   std::vector<uint64_t> src_bytes, dst_bytes;
   std::vector<Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
@@ -762,7 +762,7 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
     if (mapped) {
       // over PCIe every read costs: stage each source piece once and write all its replicas from it
       if (!p->d_fan_tiles && p->n_tma && p->opt.order == 1 && p->opt.fanout != 1) {
-        std::vector<bcp_tile> fan(p->tiles);
+        std::vector<bcp_tile> fan(p->tiles.begin(), p->tiles.end());
         mark_followers(fan.data(), p->n_tma);
         BCP_CUDA(cudaMalloc(&p->d_fan_tiles, fan.size() * sizeof(bcp_tile)));
         BCP_CUDA(cudaMemcpy(p->d_fan_tiles, fan.data(), fan.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));

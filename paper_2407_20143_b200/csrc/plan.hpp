@@ -3,7 +3,10 @@
 
 #include <cstdarg>
 #include <cstdint>
+#include <memory>
+#include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "bcp.h"
@@ -77,9 +80,32 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
 // Mark groups of TMA units (ordered by source address) that read the same source bytes.
 void mark_followers(bcp_tile* tma, size_t n);
 
+// A work list can hold a million units: a vector whose resize() leaves the new elements
+// uninitialised, so that the threads which fill it are the first to touch its pages.
+template <class T>
+struct NoInitAlloc : std::allocator<T> {
+  template <class U>
+  struct rebind {
+    using other = NoInitAlloc<U>;
+  };
+  NoInitAlloc() = default;
+  template <class U>
+  NoInitAlloc(const NoInitAlloc<U>&) {}
+  template <class U>
+  void construct(U* p) {
+    ::new (static_cast<void*>(p)) U;
+  }
+  template <class U, class... A>
+  void construct(U* p, A&&... a) {
+    ::new (static_cast<void*>(p)) U(std::forward<A>(a)...);
+  }
+};
+using TileVec = std::vector<bcp_tile, NoInitAlloc<bcp_tile>>;
+
 // src_bytes: sizes of the source buffers (bounds for over-reading aligned supersets).
-void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
-                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,
-                 bcp_plan_stats_t* stats);
+// Large lists are built by several host threads (at most 8; the environment variable
+// BCP_PLAN_THREADS overrides the count); the result does not depend on how many.
+void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes, TileVec* tiles,
+                 size_t* n_tma, size_t* n_big, std::vector<Rect>* rects, bcp_plan_stats_t* stats);
 
 }  // namespace bcp

@@ -7,10 +7,15 @@
 //            FQN; each matching segment becomes one piece of the load plan.
 // Everything here is int64 arithmetic on the host; no CUDA.
 #include <algorithm>
+#include <atomic>
 #include <chrono>
+#include <cstdlib>
+#include <memory>
+#include <thread>
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <string_view>
 #include <unordered_map>
 
 #include "plan.hpp"
@@ -215,7 +220,8 @@ int check_meta(const bcp_shard_meta& m, const char* side, size_t i, const uint64
   return BCP_OK;
 }
 
-void expand(const bcp_shard_meta& m, uint32_t meta_index, int64_t count, std::vector<Entry>* out) {
+void expand(const bcp_shard_meta& m, uint32_t meta_index, int64_t count, std::vector<Entry>* out,
+            std::vector<RelBox>* scratch) {
   if (count == 0) return;
   if (m.kind == BCP_BOX) {
     Entry e;
@@ -230,7 +236,8 @@ void expand(const bcp_shard_meta& m, uint32_t meta_index, int64_t count, std::ve
     out->push_back(e);
     return;
   }
-  std::vector<RelBox> boxes;
+  std::vector<RelBox>& boxes = *scratch;
+  boxes.clear();
   decompose(m.lengths, m.ndim, m.flat_begin, m.flat_end, &boxes);
   uint64_t pos = m.byte_offset;  // sub-boxes occupy consecutive byte ranges, in flat order
   for (const RelBox& b : boxes) {
@@ -340,11 +347,16 @@ void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t isz, const in
   }
 }
 
-struct SegKey {  // identity of a matched segment on the saved side (for the unique-bytes count)
-  uint32_t fam, src;
-  int64_t off[BCP_MAX_NDIM], len[BCP_MAX_NDIM];
-  bool operator<(const SegKey& o) const { return memcmp(this, &o, sizeof *this) < 0; }
-  bool operator==(const SegKey& o) const { return memcmp(this, &o, sizeof *this) == 0; }
+// Identity of a matched segment on the saved side (for the unique-bytes count): the saved box
+// and the positions of the segment's first and last element in that box's C order, which fix
+// the segment's box.
+struct SegKey {
+  uint64_t src, first, last, bytes;
+  bool operator<(const SegKey& o) const {
+    if (src != o.src) return src < o.src;
+    return first != o.first ? first < o.first : last < o.last;
+  }
+  bool operator==(const SegKey& o) const { return src == o.src && first == o.first && last == o.last; }
 };
 
 }  // namespace
@@ -354,10 +366,11 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
                     bool allow_replicas, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
   if ((n_src && !src) || (n_dst && !dst) || (n_src_bufs && !src_buf_bytes) || (n_dst_bufs && !dst_buf_bytes))
     return fail(BCP_ERR_INVALID, "bcp_plan: NULL array with non-zero count");
-  std::unordered_map<std::string, uint32_t> ids;
+  std::unordered_map<std::string_view, uint32_t> ids;  // keys point into the caller's metas
   std::vector<Family> fams;
   auto family_of = [&](const bcp_shard_meta& m, const char* side, size_t i, uint32_t* id) -> int {
-    auto it = ids.find(m.fqn);
+    const std::string_view name(m.fqn);
+    auto it = ids.find(name);
     if (it == ids.end()) {
       Family f;
       f.fqn = m.fqn;
@@ -366,7 +379,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       f.ndim = m.ndim;
       for (uint32_t k = 0; k < BCP_MAX_NDIM; ++k) f.shape[k] = k < m.ndim ? m.global_shape[k] : 1;
       *id = uint32_t(fams.size());
-      ids.emplace(m.fqn, *id);
+      ids.emplace(name, *id);
       fams.push_back(std::move(f));
       return BCP_OK;
     }
@@ -379,12 +392,13 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
     *id = it->second;
     return BCP_OK;
   };
+  std::vector<RelBox> scratch;
   for (size_t i = 0; i < n_src; ++i) {
     int64_t n;
     uint32_t f;
     if (int rc = check_meta(src[i], "src", i, src_buf_bytes, n_src_bufs, &n)) return rc;
     if (int rc = family_of(src[i], "src", i, &f)) return rc;
-    expand(src[i], uint32_t(i), n, &fams[f].src);
+    expand(src[i], uint32_t(i), n, &fams[f].src, &scratch);
   }
   // target byte ranges must not overlap inside a buffer
   {
@@ -399,7 +413,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       uint32_t f;
       if (int rc = check_meta(dst[i], "dst", i, dst_buf_bytes, n_dst_bufs, &n)) return rc;
       if (int rc = family_of(dst[i], "dst", i, &f)) return rc;
-      expand(dst[i], uint32_t(i), n, &fams[f].dst);
+      expand(dst[i], uint32_t(i), n, &fams[f].dst, &scratch);
       if (n > 0) rs.push_back(Range{dst[i].byte_offset, dst[i].byte_offset + dst[i].byte_length, dst[i].buf_index, uint32_t(i)});
     }
     std::sort(rs.begin(), rs.end(), [](const Range& a, const Range& b) { return a.buf != b.buf ? a.buf < b.buf : a.lo < b.lo; });
@@ -419,8 +433,9 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       }
     }
   }
-  std::vector<SegKey> segs;
-  uint64_t n_inter = 0, n_se = 0, n_de = 0;
+  std::vector<SegKey> segs;      // matched segments of the family at hand
+  std::vector<int64_t> reach;    // reach[i] = largest end (along dim 0) among the family's saved boxes 0..i
+  uint64_t n_inter = 0, n_se = 0, n_de = 0, uniq = 0;
   for (uint32_t fi = 0; fi < fams.size(); ++fi) {
     Family& f = fams[fi];
     n_se += f.src.size();
@@ -455,10 +470,16 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
                       f.src[j].meta);
       }
     }
+    reach.resize(f.src.size());
+    for (size_t i = 0; i < f.src.size(); ++i)
+      reach[i] = std::max(i ? reach[i - 1] : INT64_MIN, f.src[i].off[0] + f.src[i].len[0]);
+    segs.clear();
     for (const Entry& d : f.dst) {
       int64_t covered = 0;
       const int64_t dend0 = d.off[0] + d.len[0];
-      for (uint32_t si = 0; si < f.src.size(); ++si) {
+      // boxes before `first` all end at or before the wanted box's first row
+      const uint32_t first = uint32_t(std::upper_bound(reach.begin(), reach.end(), d.off[0]) - reach.begin());
+      for (uint32_t si = first; si < f.src.size(); ++si) {
         const Entry& s = f.src[si];
         if (s.off[0] >= dend0) break;  // sorted by first offset
         int64_t o[BCP_MAX_NDIM], l[BCP_MAX_NDIM];
@@ -466,13 +487,10 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
         covered += volume(l, 0, nd);
         ++n_inter;
         lower(s, d, nd, f.itemsize, o, l, items);
-        SegKey key;
-        memset(&key, 0, sizeof key);
-        key.fam = fi;
-        key.src = si;
+        SegKey key = {si, 0, 0, uint64_t(volume(l, 0, nd)) * f.itemsize};
         for (uint32_t k = 0; k < nd; ++k) {
-          key.off[k] = o[k];
-          key.len[k] = l[k];
+          key.first = key.first * uint64_t(s.len[k]) + uint64_t(o[k] - s.off[k]);
+          key.last = key.last * uint64_t(s.len[k]) + uint64_t(o[k] + l[k] - 1 - s.off[k]);
         }
         segs.push_back(key);
       }
@@ -480,11 +498,11 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
         return fail(BCP_ERR_UNCOVERED, "%s: dst[%u] wants %lld elements, saved entries hold %lld of them", f.fqn, d.meta,
                     (long long)d.vol, (long long)covered);
     }
+    // distinct source bytes: a segment wanted by several target entries (replicas) counts once
+    std::sort(segs.begin(), segs.end());
+    segs.erase(std::unique(segs.begin(), segs.end()), segs.end());
+    for (const SegKey& k : segs) uniq += k.bytes;
   }
-  std::sort(segs.begin(), segs.end());
-  segs.erase(std::unique(segs.begin(), segs.end()), segs.end());
-  uint64_t uniq = 0;
-  for (const SegKey& k : segs) uniq += uint64_t(volume(k.len, 0, fams[k.fam].ndim)) * fams[k.fam].itemsize;
   stats->n_src_entries = n_se;
   stats->n_dst_entries = n_de;
   stats->n_fqns = fams.size();
@@ -502,12 +520,64 @@ inline uint32_t gran_log2(uint64_t bits) {
   return g;  // 0..4 -> 1..16 bytes
 }
 
+// Host threads for large work lists.  The result never depends on the count.
+unsigned plan_threads(size_t n_units) {
+  if (n_units < 32768) return 1;
+  unsigned n = 0;
+  if (const char* e = getenv("BCP_PLAN_THREADS")) n = unsigned(strtoul(e, nullptr, 10));
+  if (!n) n = std::min(8u, std::thread::hardware_concurrency());
+  return std::max(1u, std::min(n, 64u));
+}
+
+// job(0) .. job(n_jobs - 1), handed out by a counter to the caller and up to threads - 1 helpers.
+// Jobs must not throw; if helpers cannot be started the caller does all the work.
+template <class F>
+void parallel_jobs(size_t n_jobs, unsigned threads, F&& job) {
+  std::atomic<size_t> next{0};
+  auto worker = [&] {
+    for (size_t j; (j = next.fetch_add(1)) < n_jobs;) job(j);
+  };
+  std::vector<std::thread> pool;
+  if (threads > 1 && n_jobs > 1) {
+    try {
+      pool.reserve(threads - 1);
+      for (unsigned t = 1; t < threads && t < n_jobs; ++t) pool.emplace_back(worker);
+    } catch (...) {
+    }
+  }
+  worker();
+  for (std::thread& t : pool) t.join();
+}
+
+enum { kTma = 0, kBig = 1, kSmall = 2 };  // unit classes, in the order of the final list
+
+struct Tally {
+  uint64_t bytes_copied = 0, bytes_misaligned = 0, n_strided = 0;
+  uint64_t tma_bytes = 0;   // payload of the TMA class ...
+  uint64_t tma_busy = 0;    // ... in shifted runs and rectangles with rows under 2 KiB (the warp issues a lot)
+  uint64_t tma_boxed = 0;   // ... in tensor-map boxes
+  void add(const Tally& o) {
+    bytes_copied += o.bytes_copied, bytes_misaligned += o.bytes_misaligned, n_strided += o.n_strided;
+    tma_bytes += o.tma_bytes, tma_busy += o.tma_busy, tma_boxed += o.tma_boxed;
+  }
+};
+
+// Cuts items into units.  Used twice: a counting pass (out[] null) that sizes the arrays, then
+// a writing pass in which every block of items starts at its own, precomputed positions.
 struct Cutter {
   const Options& opt;
   const std::vector<uint64_t>* src_bytes;  // source buffer sizes (may be null: unknown)
-  std::vector<bcp_tile> tma, big, small;
-  std::vector<Rect> rects;
-  bcp_plan_stats_t* st;
+  bool demote;                             // small job: TMA-eligible units go to the register kernel
+  bcp_tile* out[3];
+  Rect* rects_out;
+  size_t pos[3];
+  size_t rect_pos;
+  Tally st;
+
+  void put(int cls, const bcp_tile& t) {
+    if (out[cls]) out[cls][pos[cls]] = t;
+    ++pos[cls];
+  }
 
   void emit(const Item& it, uint64_t src_off, uint64_t dst_off, uint64_t rows, uint64_t row_bytes) {
     bcp_tile t;
@@ -528,28 +598,31 @@ struct Cutter {
     t.flags = g;
     if (it.zero) t.flags |= BCP_TILE_ZERO;
     const uint64_t payload = rows * row_bytes;
-    if (g < 4) st->bytes_misaligned += payload;
-    if (rows > 1) ++st->n_strided_tiles;
-    st->bytes_copied += payload;
+    if (g < 4) st.bytes_misaligned += payload;
+    if (rows > 1) ++st.n_strided;
+    st.bytes_copied += payload;
     if (payload < opt.small_bytes) {
       t.flags |= BCP_TILE_SMALL;
-      small.push_back(t);
-    } else {
-      // TMA staging: whole 16-byte units between 16-byte aligned addresses (runs and rectangles),
-      // or a run / rectangle of any alignment whose 16-byte aligned supersets stay inside the source buffer
-      bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= opt.tma_min_row_bytes;
-      if (eligible && g < 4) {  // the superset of the last row must not reach past the source buffer
-        const uint64_t end16 = (src_off + (rows - 1) * (rows > 1 ? it.src_pitch : 0) + row_bytes + 15) & ~uint64_t(15);
-        eligible = src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
-      }
-      if (eligible) {
+      put(kSmall, t);
+      return;
+    }
+    // TMA staging: whole 16-byte units between 16-byte aligned addresses (runs and rectangles),
+    // or a run / rectangle of any alignment whose 16-byte aligned supersets stay inside the source buffer
+    bool eligible = !it.zero && opt.path_mask != 1 && row_bytes >= opt.tma_min_row_bytes;
+    if (eligible && g < 4) {  // the superset of the last row must not reach past the source buffer
+      const uint64_t end16 = (src_off + (rows - 1) * (rows > 1 ? it.src_pitch : 0) + row_bytes + 15) & ~uint64_t(15);
+      eligible = src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
+    }
+    if (eligible) {
+      st.tma_bytes += payload;
+      if (g < 4 || (rows > 1 && row_bytes < 2048)) st.tma_busy += payload;
+      if (!demote) {
         t.flags |= BCP_TILE_TMA;
-        ++st->n_tma_tiles;
-        tma.push_back(t);
-      } else {
-        big.push_back(t);
+        put(kTma, t);
+        return;
       }
     }
+    put(kBig, t);
   }
 
   // contiguous run: peel a ragged head / tail when source and target are co-aligned, then
@@ -591,11 +664,15 @@ struct Cutter {
     const uint64_t box_rows = std::min<uint64_t>(256, cap / it.row_bytes);
     if (box_rows == 0) return false;
     const uint64_t rpt = std::max<uint64_t>(box_rows, opt.tile_bytes / it.row_bytes / box_rows * box_rows);
-    Rect rc;
-    rc.src_off = it.src_off, rc.dst_off = it.dst_off, rc.src_pitch = it.src_pitch, rc.dst_pitch = it.dst_pitch;
-    rc.rows = it.rows, rc.row_bytes = uint32_t(it.row_bytes), rc.src_buf = it.src_buf, rc.dst_buf = it.dst_buf;
-    rc.box_rows = uint32_t(box_rows);
-    rects.push_back(rc);
+    if (!demote) {
+      if (rects_out) {
+        Rect& rc = rects_out[rect_pos];
+        rc.src_off = it.src_off, rc.dst_off = it.dst_off, rc.src_pitch = it.src_pitch, rc.dst_pitch = it.dst_pitch;
+        rc.rows = it.rows, rc.row_bytes = uint32_t(it.row_bytes), rc.src_buf = it.src_buf, rc.dst_buf = it.dst_buf;
+        rc.box_rows = uint32_t(box_rows);
+      }
+      ++rect_pos;
+    }
     for (uint64_t r = 0; r < it.rows; r += rpt) {
       const uint64_t nr = std::min(rpt, it.rows - r);
       bcp_tile t;
@@ -605,14 +682,20 @@ struct Cutter {
       t.src_pitch = it.src_pitch, t.dst_pitch = it.dst_pitch;
       t.rows = uint32_t(nr), t.row_bytes = uint32_t(it.row_bytes);
       t.src_buf = it.src_buf, t.dst_buf = it.dst_buf;
-      t.flags = 4u | BCP_TILE_TMA | BCP_TILE_TMA2D;
-      t.reserved[0] = uint32_t(rects.size());  // index + 1
+      t.flags = 4u;
+      ++st.n_strided;
+      st.bytes_copied += nr * it.row_bytes;
+      st.tma_bytes += nr * it.row_bytes;
+      st.tma_boxed += nr * it.row_bytes;
+      if (demote) {
+        put(kBig, t);
+        continue;
+      }
+      t.flags |= BCP_TILE_TMA | BCP_TILE_TMA2D;
+      t.reserved[0] = uint32_t(rect_pos);  // index + 1
       t.reserved[1] = uint32_t(r);
       t.reserved[2] = uint32_t(box_rows);
-      ++st->n_strided_tiles;
-      ++st->n_tma_tiles;
-      st->bytes_copied += nr * it.row_bytes;
-      tma.push_back(t);
+      put(kTma, t);
     }
     return true;
   }
@@ -660,9 +743,50 @@ void mark_followers(bcp_tile* tma, size_t n) {
   }
 }
 
-void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes,
-                 std::vector<bcp_tile>* tiles, size_t* n_tma, size_t* n_big, std::vector<Rect>* rects,
-                 bcp_plan_stats_t* stats) {
+namespace {
+
+// Sort key of a unit: (a_buf, a_off) is the side the list is ordered by, (b_buf, b_off) breaks
+// ties between units that read the same source bytes (replicas); idx = position before sorting.
+struct Key {
+  uint64_t a_off, b_off;
+  uint32_t a_buf, b_buf, idx, pad;
+};
+inline bool key_less(const Key& x, const Key& y) {
+  if (x.a_buf != y.a_buf) return x.a_buf < y.a_buf;
+  if (x.a_off != y.a_off) return x.a_off < y.a_off;
+  return x.b_buf != y.b_buf ? x.b_buf < y.b_buf : x.b_off < y.b_off;
+}
+
+// Merge sort over `threads` chunks; returns whichever of the two arrays holds the result.
+// Every merge of two runs is itself split into parts (cut one run evenly, find the matching
+// cut of the other by binary search), so that all rounds keep every thread busy.
+Key* sort_keys(Key* k, Key* tmp, size_t n, unsigned threads) {
+  const size_t chunks = std::max<size_t>(1, std::min<size_t>(threads, n / 8192));
+  auto bound = [&](size_t i) { return n * std::min(i, chunks) / chunks; };
+  parallel_jobs(chunks, threads, [&](size_t c) { std::sort(k + bound(c), k + bound(c + 1), key_less); });
+  Key *from = k, *to = tmp;
+  for (size_t w = 1; w < chunks; w *= 2) {
+    const size_t pairs = (chunks + 2 * w - 1) / (2 * w);
+    const size_t parts = std::max<size_t>(1, (threads + pairs - 1) / pairs);
+    parallel_jobs(pairs * parts, threads, [&](size_t job) {
+      const size_t j = job / parts, part = job % parts;
+      const size_t lo = bound(2 * j * w), mid = bound(2 * j * w + w), hi = bound(2 * j * w + 2 * w);
+      const Key *a = from + lo, *b = from + mid;
+      const size_t na = mid - lo, nb = hi - mid;
+      auto cut_b = [&](size_t ia) { return ia >= na ? nb : size_t(std::lower_bound(b, b + nb, a[ia], key_less) - b); };
+      const size_t a0 = na * part / parts, a1 = na * (part + 1) / parts;
+      const size_t b0 = part == 0 ? 0 : cut_b(a0), b1 = part + 1 == parts ? nb : cut_b(a1);
+      std::merge(a + a0, a + a1, b + b0, b + b1, to + lo + a0 + b0, key_less);
+    });
+    std::swap(from, to);
+  }
+  return from;
+}
+
+}  // namespace
+
+void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes, TileVec* tiles,
+                 size_t* n_tma, size_t* n_big, std::vector<Rect>* rects, bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
@@ -682,53 +806,77 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     }
     merged.push_back(it);
   }
-  stats->n_items = merged.size();
-  stats->bytes_copied = 0;
-  stats->bytes_misaligned = 0;
-  stats->n_strided_tiles = 0;
-  stats->n_tma_tiles = 0;
-  Cutter c{opt, src_bytes, {}, {}, {}, {}, stats};
-  for (const Item& it : merged) c.cut(it);
-  if (opt.path_mask == 0) {  // small jobs are launch-bound: keep them in one kernel
-    uint64_t eligible = 0;
-    for (const bcp_tile& t : c.tma) eligible += uint64_t(t.rows) * t.row_bytes;
-    if (eligible < (128u << 20)) {
-      for (bcp_tile& t : c.tma) {
-        t.flags &= ~(BCP_TILE_TMA | BCP_TILE_TMA2D);
-        t.reserved[0] = t.reserved[1] = t.reserved[2] = 0;
-      }
-      c.rects.clear();
-      c.big.insert(c.big.end(), c.tma.begin(), c.tma.end());
-      c.tma.clear();
-      stats->n_tma_tiles = 0;
+  const size_t n_items = merged.size();
+  stats->n_items = n_items;
+
+  // Pass 1: how many units of each class (and rectangles) every item gives.  A rough unit count
+  // decides whether helpers are worth starting.
+  uint64_t rough = 0;
+  for (const Item& it : merged) rough += it.rows * it.row_bytes / opt.tile_bytes + (it.row_bytes >= opt.tile_bytes ? it.rows : 1);
+  const unsigned threads = plan_threads(size_t(std::min<uint64_t>(rough, SIZE_MAX)));
+  struct Count {
+    size_t n[3], rects;
+  };
+  std::vector<Count> cnt(n_items + 1);
+  const size_t kBlock = 16;
+  std::vector<Tally> tally((n_items + kBlock - 1) / kBlock);
+  parallel_jobs(tally.size(), threads, [&](size_t j) {
+    Cutter c{opt, src_bytes, false, {nullptr, nullptr, nullptr}, nullptr, {0, 0, 0}, 0, Tally()};
+    for (size_t i = j * kBlock; i < std::min(n_items, (j + 1) * kBlock); ++i) {
+      const Count before = {{c.pos[0], c.pos[1], c.pos[2]}, c.rect_pos};
+      c.cut(merged[i]);
+      cnt[i] = {{c.pos[0] - before.n[0], c.pos[1] - before.n[1], c.pos[2] - before.n[2]}, c.rect_pos - before.rects};
     }
+    tally[j] = c.st;
+  });
+  Tally all;
+  for (const Tally& t : tally) all.add(t);
+  // small jobs are launch-bound: keep them in one kernel
+  const bool demote = opt.path_mask == 0 && all.tma_bytes < (128u << 20);
+  if (demote) {
+    for (size_t i = 0; i < n_items; ++i) cnt[i].n[kBig] += cnt[i].n[kTma], cnt[i].n[kTma] = 0, cnt[i].rects = 0;
+    all.tma_bytes = all.tma_busy = all.tma_boxed = 0;
   }
-  auto by_src = [](const bcp_tile& a, const bcp_tile& b) {
-    if (a.src_buf != b.src_buf) return a.src_buf < b.src_buf;
-    if (a.src_off != b.src_off) return a.src_off < b.src_off;
-    return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
-  };
-  auto by_dst = [](const bcp_tile& a, const bcp_tile& b) {
-    return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
-  };
+  Count run = {{0, 0, 0}, 0};  // counts -> positions of each item's first unit inside its class
+  for (size_t i = 0; i <= n_items; ++i) {
+    const Count c = i < n_items ? cnt[i] : Count{{0, 0, 0}, 0};
+    cnt[i] = run;
+    for (int k = 0; k < 3; ++k) run.n[k] += c.n[k];
+    run.rects += c.rects;
+  }
+  const size_t total = run.n[0] + run.n[1] + run.n[2];
+
+  // Pass 2: write the units, blocks of items of about equal size in parallel
+  std::unique_ptr<bcp_tile[]> raw(new bcp_tile[total ? total : 1]);
+  bcp_tile* const cls[3] = {raw.get(), raw.get() + run.n[0], raw.get() + run.n[0] + run.n[1]};
+  std::vector<Rect> rc(run.rects);
+  std::vector<size_t> cuts(1, 0);  // item index where each block starts
+  {
+    auto units_before = [&](size_t i) { return cnt[i].n[0] + cnt[i].n[1] + cnt[i].n[2]; };
+    const size_t per_block = std::max<size_t>(4096, total / (size_t(threads) * 8) + 1);
+    for (size_t i = 1; i < n_items; ++i)
+      if (units_before(i) - units_before(cuts.back()) >= per_block) cuts.push_back(i);
+    cuts.push_back(n_items);
+  }
+  parallel_jobs(cuts.size() - 1, threads, [&](size_t j) {
+    const Count& at = cnt[cuts[j]];
+    Cutter c{opt, src_bytes, demote, {cls[0], cls[1], cls[2]}, rc.data(), {at.n[0], at.n[1], at.n[2]}, at.rects, Tally()};
+    for (size_t i = cuts[j]; i < cuts[j + 1]; ++i) c.cut(merged[i]);
+  });
+  stats->bytes_copied = all.bytes_copied;
+  stats->bytes_misaligned = all.bytes_misaligned;
+  stats->n_strided_tiles = all.n_strided;
+  stats->n_tma_tiles = run.n[kTma];
+
   // Stage geometry of the TMA kernel when the caller left it open.  Long aligned runs only need
   // a few copy commands per stage, so two CTAs with 32 KiB stages per SM are enough; shifted
   // runs (copied out of shared memory by the warp itself) and rectangles with rows under 2 KiB
   // (one copy command per row) are limited by what one warp can issue and want four CTAs with
   // 16 KiB stages.  Both fill 192 KiB of shared memory per SM.
   {
-    uint64_t total = 0, busy = 0, boxed = 0;
-    for (const bcp_tile& t : c.tma) {
-      const uint64_t n = uint64_t(t.rows) * t.row_bytes;
-      total += n;
-      if (t.flags & BCP_TILE_TMA2D) {
-        boxed += n;
-      } else if ((t.flags & BCP_TILE_GRAN_MASK) < 4 || (t.rows > 1 && t.row_bytes < 2048)) {
-        busy += n;
-      }
-    }
-    const bool many_busy = busy * 8 >= total && total > 0;
-    const bool many_boxed = !many_busy && boxed * 8 >= total && total > 0;  // boxes are at most 16 KiB: deeper ring
+    const uint64_t busy = all.tma_busy, boxed = all.tma_boxed, sum = all.tma_bytes;
+    const bool many_busy = busy * 8 >= sum && sum > 0;
+    const bool many_boxed = !many_busy && boxed * 8 >= sum && sum > 0;  // boxes are at most 16 KiB: deeper ring
     if (!opt.tma_stage_bytes) opt.tma_stage_bytes = (many_busy || many_boxed) ? 16384 : 32768;
     if (!opt.tma_ctas_per_sm) opt.tma_ctas_per_sm = many_busy ? 4 : 2;
     if (!opt.tma_stages) opt.tma_stages = many_boxed ? 4 : 3;
@@ -736,31 +884,43 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   // Register kernel: a CTA per unit for small jobs (fewer, fatter workers start faster); every
   // warp its own worker once the kernel has a lot to move (no barriers, deeper overlap).
   if (!opt.worker) {
-    uint64_t reg_bytes = 0;
-    for (const bcp_tile& t : c.big) reg_bytes += uint64_t(t.rows) * t.row_bytes;
-    for (const bcp_tile& t : c.small) reg_bytes += uint64_t(t.rows) * t.row_bytes;
-    opt.worker = reg_bytes >= (128u << 20) ? 2 : 1;
+    opt.worker = all.bytes_copied - all.tma_bytes >= (128u << 20) ? 2 : 1;
     if (opt.worker == 2 && !opt.ctas_per_sm) opt.ctas_per_sm = 4;
   }
   if (!opt.ctas_per_sm) opt.ctas_per_sm = 2;
-  for (std::vector<bcp_tile>* v : {&c.tma, &c.big, &c.small}) {
-    if (opt.order == 1) {
-      std::sort(v->begin(), v->end(), by_src);
-    } else {
-      std::sort(v->begin(), v->end(), by_dst);
+
+  // Order every class by source address (order 1: the reads of replicas meet in L2) or by target
+  // address, through compact keys, and gather the units into the final list.
+  std::unique_ptr<Key[]> keys(new Key[total ? total : 1]), spare(new Key[total ? total : 1]);
+  const bool by_src = opt.order == 1;
+  const size_t kChunk = 65536;
+  parallel_jobs((total + kChunk - 1) / kChunk, threads, [&](size_t j) {
+    for (size_t i = j * kChunk; i < std::min(total, (j + 1) * kChunk); ++i) {
+      const bcp_tile& t = raw[i];
+      const int k = i < run.n[0] ? 0 : i < run.n[0] + run.n[1] ? 1 : 2;
+      const uint32_t idx = uint32_t(i - (cls[k] - raw.get()));
+      keys[i] = by_src ? Key{t.src_off, t.dst_off, t.src_buf, t.dst_buf, idx, 0} : Key{t.dst_off, 0, t.dst_buf, 0, idx, 0};
     }
-  }
-  if (opt.order == 1 && opt.fanout == 1) mark_followers(c.tma.data(), c.tma.size());
-  stats->n_tiles = c.tma.size() + c.big.size();
-  stats->n_small_tiles = c.small.size();
-  *n_tma = c.tma.size();
-  *n_big = c.big.size();
-  if (rects) *rects = std::move(c.rects);
+  });
   tiles->clear();
-  tiles->reserve(c.tma.size() + c.big.size() + c.small.size());
-  tiles->insert(tiles->end(), c.tma.begin(), c.tma.end());
-  tiles->insert(tiles->end(), c.big.begin(), c.big.end());
-  tiles->insert(tiles->end(), c.small.begin(), c.small.end());
+  tiles->resize(total);
+  size_t base = 0;
+  for (int k = 0; k < 3; ++k) {
+    const size_t n = run.n[k];
+    const Key* sorted = sort_keys(keys.get() + base, spare.get() + base, n, threads);
+    bcp_tile* dst = tiles->data() + base;
+    const bcp_tile* src = cls[k];
+    parallel_jobs((n + kChunk - 1) / kChunk, threads, [&](size_t j) {
+      for (size_t i = j * kChunk; i < std::min(n, (j + 1) * kChunk); ++i) dst[i] = src[sorted[i].idx];
+    });
+    base += n;
+  }
+  if (opt.order == 1 && opt.fanout == 1) mark_followers(tiles->data(), run.n[kTma]);
+  stats->n_tiles = run.n[kTma] + run.n[kBig];
+  stats->n_small_tiles = run.n[kSmall];
+  *n_tma = run.n[kTma];
+  *n_big = run.n[kBig];
+  if (rects) *rects = std::move(rc);
 }
 
 }  // namespace bcp

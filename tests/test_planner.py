@@ -312,6 +312,29 @@ def test_plan_image_round_trip(case):
     assert all(np.array_equal(g, w) for g, w in zip(got, want))
 
 
+def _image_without_clock(plan):
+    """Plan image with the planning-time field and the checksum over it blanked."""
+    import struct
+
+    image = plan.serialize()
+    at = image.find(struct.pack("<d", plan.stats()["plan_ms"]))
+    assert 0 < at < 256
+    return image[:at] + bytes(8) + image[at + 8:-8]
+
+
+@pytest.mark.parametrize("opts", [dict(), dict(order=2, tile_bytes=16384), dict(path_mask=1)], ids=str)
+def test_work_list_does_not_depend_on_the_number_of_planner_threads(opts, monkeypatch):
+    case = CONFIGS["cfg3"]()  # 16 GB, a quarter of a million units: large enough for helper threads
+    images = []
+    for threads in ("1", "3", "8"):
+        monkeypatch.setenv("BCP_PLAN_THREADS", threads)
+        plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+        assert plan.stats()["n_tiles"] > 100_000
+        images.append(_image_without_clock(plan))
+        plan.destroy()
+    assert images[0] == images[1] == images[2]
+
+
 def test_plan_image_is_verified():
     case = scenario_cases()[0]
     plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
