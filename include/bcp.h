@@ -298,6 +298,9 @@ BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, si
  * point.  Executions of one plan must be ordered (same stream, or externally
  * synchronised): they share the plan's device-side pointer tables and ticket counter.
  * Target bytes not named by any target entry are left untouched.
+ * Once a plan has run on a set of buffer addresses, running it again on the same addresses
+ * enqueues kernel launches only (no allocation, no copy, no synchronisation), so the call
+ * may be recorded by a stream capture and replayed from a CUDA graph.
  */
 BCP_API int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs,
                 void* const* dst_bufs, size_t n_dst_bufs, void* stream);

@@ -461,3 +461,34 @@ def _pack_full_rank(case, dst, device):
     torch.cuda.synchronize()
     assert torch.equal(out[:sizes[0]], blob[offs[0]:offs[0] + sizes[0]]) and torch.equal(out[sizes[0]:], blob[offs[1]:offs[1] + sizes[1]])
     bcp.bcp_pack_cache_clear()
+
+
+# ---- CUDA graphs ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,opts", [("cfg1", dict()), ("cfg1", dict(path_mask=7, tma_min_row_bytes=512)),
+                                       ("big_random", dict(path_mask=3, tile_bytes=8192))], ids=str)
+def test_reshard_replays_from_a_cuda_graph(cuda_device, name, opts):
+    """A plan that has run once on some buffers is pure kernel launches on those buffers, so a
+    stream capture records it and a replay reshards whatever the buffers hold by then."""
+    case = CONFIGS["cfg1"]("index") if name == "cfg1" else big_random_case(3, itemsize=2)
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device, poison=0x5A)
+    dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    bcp.bcp_reshard(plan, src, dst)  # binds the plan to the device and uploads its tables
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        bcp.bcp_reshard(plan, src, dst)  # the binding launches on torch's current stream: the capturing one
+    for seed in (case.seed + 1, case.seed + 2):
+        fresh = fills.fill_state(case.src, case.key_ids, "uniform", seed, cuda_device, poison=0x5A)
+        for s, f in zip(src, fresh):
+            s.copy_(f)
+        for b in backs:
+            b.fill_(POISON)
+        want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+        graph.replay()
+        torch.cuda.synchronize()
+        bcp.bcp_plan_device_status(plan)
+        assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want))
+        assert guards_intact(backs, case.dst.buf_bytes)
+    del graph
+    plan.destroy()
