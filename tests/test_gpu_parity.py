@@ -492,3 +492,47 @@ def test_reshard_replays_from_a_cuda_graph(cuda_device, name, opts):
         assert guards_intact(backs, case.dst.buf_bytes)
     del graph
     plan.destroy()
+
+
+# ---- host threads --------------------------------------------------------------------------------
+def test_plans_run_from_several_threads_on_their_own_streams(cuda_device):
+    """Different plans are independent: three host threads, each with its own plan, buffers and
+    stream, execute at the same time (their kernels share the GPU; none waits for another)."""
+    import threading
+
+    torch.cuda.init()
+    cases = [big_random_case(1, itemsize=2), CONFIGS["cfg1"]("index"), big_random_case(6, itemsize=4)]
+    opts = [dict(path_mask=3, tile_bytes=8192), dict(), dict(path_mask=1, tile_bytes=16384)]
+    jobs = []
+    for case, o in zip(cases, opts):
+        src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device, poison=0x5A)
+        want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+        jobs.append((case, o, src, want))
+    torch.cuda.synchronize()
+    failures = []
+
+    def work(case, o, src, want):
+        try:
+            torch.cuda.set_device(cuda_device)
+            stream = torch.cuda.Stream(device=cuda_device)
+            plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **o)
+            for _ in range(8):
+                with torch.cuda.stream(stream):
+                    dst, backs = guarded(case.dst.buf_bytes, cuda_device)
+                bcp.bcp_reshard(plan, src, dst, stream=stream)
+                stream.synchronize()
+                bcp.bcp_plan_device_status(plan, stream=stream)
+                if not all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)):
+                    failures.append(case.name + ": wrong bytes")
+                if not guards_intact(backs, case.dst.buf_bytes):
+                    failures.append(case.name + ": guard band overwritten")
+            plan.destroy()
+        except Exception as e:  # noqa: BLE001 - reported below
+            failures.append(f"{case.name}: {e!r}")
+
+    threads = [threading.Thread(target=work, args=j) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not failures, failures[:3]

@@ -412,3 +412,45 @@ def test_pack_layout_matches_closed_form():
         assert bcp.bcp_pack_layout(sizes, align) == orc.pack_layout(sizes, align)
     with pytest.raises(bcp.BcpError):
         bcp.bcp_pack_layout(sizes, 24)
+
+
+# ---- host threads --------------------------------------------------------------------------------
+def test_planning_from_several_threads_at_once():
+    """Different plans may be built and read from different threads at the same time; error
+    texts are per thread.  (The binding releases the interpreter lock inside every call.)"""
+    import threading
+
+    cases = [random_case(s) for s in range(6)] + [big_random_case(2, itemsize=2), big_random_case(4, itemsize=4)]
+
+    def image(case):
+        plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, tile_bytes=4096)
+        out = _image_without_clock(plan)
+        plan.destroy()
+        return out
+
+    want = [image(c) for c in cases]
+    failures = []
+
+    def work(tid):
+        try:
+            for rep in range(12):
+                k = (tid + rep) % len(cases)
+                if image(cases[k]) != want[k]:
+                    failures.append(f"thread {tid}: plan {k} differs")
+                if tid % 2:  # this thread also fails on purpose; the message must be its own
+                    name = f"t{tid}r{rep}"
+                    try:
+                        bcp.bcp_plan([_m(fqn=name, isz=3)], [64], [_m(fqn=name)], [64])
+                        failures.append("no error raised")
+                    except bcp.BcpError as e:
+                        if e.code != api.ERR_INVALID or name not in str(e):
+                            failures.append(f"thread {tid}: foreign error text {e}")
+        except Exception as e:  # noqa: BLE001 - reported below
+            failures.append(f"thread {tid}: {e!r}")
+
+    threads = [threading.Thread(target=work, args=(t,)) for t in range(6)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not failures, failures[:3]
