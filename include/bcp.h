@@ -149,7 +149,28 @@ typedef struct {
   uint32_t test_stall;      /* test hook, 0 in normal use: 1 makes the first CTA of the TMA kernel arm its
                                first stage for more bytes than it loads, so that exactly one bounded wait
                                runs out and the time-out path can be exercised without any fault          */
+  uint32_t convert;         /* 0 default: entries of one FQN must agree on itemsize and dtype_tag, bytes are
+                               moved unchanged.  BCP_CONVERT_F32_TO_BF16 / BCP_CONVERT_BF16_TO_F32: an FQN
+                               whose saved entries have dtype_tag convert_src_tag and whose wanted entries have
+                               dtype_tag convert_dst_tag (itemsizes 4 and 2, resp. 2 and 4) is converted
+                               element by element while it is resharded; every other FQN is moved unchanged.
+                               The paper moves bytes only; this serves the hand-over of fp32 master weights
+                               to a bf16 evaluation job (and back).                                       */
+  uint32_t convert_src_tag; /* see convert */
+  uint32_t convert_dst_tag;
 } bcp_plan_opts;
+
+/*
+ * Conversions (bcp_plan_opts.convert).  Values are IEEE-754 binary32 and bfloat16 (the upper
+ * 16 bits of a binary32), little endian.
+ * F32_TO_BF16 rounds to nearest, ties to even, on the bit pattern: infinities stay, values
+ * beyond the largest bfloat16 become infinity, subnormals round like any other value (no
+ * flush to zero), and every NaN becomes the quiet NaN 0x7FC0.
+ * BF16_TO_F32 appends 16 zero bits (exact for every input, NaN payloads included).
+ */
+#define BCP_CONVERT_NONE 0u
+#define BCP_CONVERT_F32_TO_BF16 1u
+#define BCP_CONVERT_BF16_TO_F32 2u
 
 typedef struct bcp_plan_s bcp_plan_t;
 
@@ -184,6 +205,10 @@ typedef struct {
                                    such a group writes every member's target from the one staged copy,
                                    and whoever draws a follower's ticket skips it                 */
 #define BCP_TILE_FAN_SHIFT 8    /* bits 8..10 of a group's first unit: how many followers it has (0..7) */
+#define BCP_TILE_CVT_SHIFT 11   /* bits 11..12: BCP_CONVERT_* applied by this unit (0: plain copy).  For a
+                                   converting unit row_bytes counts TARGET bytes; a source row holds the same
+                                   number of elements (twice, resp. half as many bytes)            */
+#define BCP_TILE_CVT_MASK (3u << BCP_TILE_CVT_SHIFT)
 
 typedef struct {
   uint64_t n_src_entries;    /* after decomposing flat slices                        */
@@ -199,6 +224,7 @@ typedef struct {
   uint64_t bytes_src_unique; /* distinct source bytes the list reads                  */
   uint64_t bytes_misaligned; /* payload in units whose access granularity is < 16 B   */
   double plan_ms;            /* host time spent in bcp_plan                           */
+  uint64_t n_cvt_tiles;      /* converting work units (bcp_plan_opts.convert)         */
 } bcp_plan_stats_t;
 
 /* ByteMeta of one tensor inside a packed blob (Sec. 3.2): start offset and length. */
@@ -283,7 +309,7 @@ BCP_API int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_p
 
 /*
  * Host copy of the work list, in execution order (CTA-wide units first, then warp
- * units).  Writes min(cap, count) records to out (may be NULL when cap == 0) and the
+ * units, then converting units).  Writes min(cap, count) records to out (may be NULL when cap == 0) and the
  * full count to *n.
  */
 BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n);

@@ -23,10 +23,17 @@ Entries are duck-typed objects with the attributes fqn, itemsize, dtype_tag, glo
 offsets, lengths, kind (0 box, 1 flat slice), flat_begin, flat_end, buf_index, byte_offset,
 byte_length.
 
+Element conversion while resharding (binary32 <-> bfloat16) is not in the paper, which moves
+bytes only; it is an extension of the library, and the oracle states it from the definition
+of rounding (`f32_to_bf16`: search the two neighbouring bfloat16 values, pick the nearer,
+the even one on a tie), not from a bit trick.
+
 Pins (tests/test_oracle_pins.py): the paper's worked example of an irregular shard, the
 identity / round-trip / exact-cover invariants, textbook reductions to numpy concatenate
 and split, a brute-force per-element index map on tiny inputs, and the closed-form
-index-pattern fill.  No function here is "parity unpinned".
+index-pattern fill; for the conversions, hand-worked bit patterns (tests/golden/
+f32_to_bf16_examples.txt), torch's own cast on everything but NaN, and the half-ulp error
+bound.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -37,6 +44,7 @@ import numpy as np
 
 _UINT = {1: np.uint8, 2: np.uint16, 4: np.uint32, 8: np.uint64}
 FLAT_SLICE = 1
+F32_TO_BF16, BF16_TO_F32 = 1, 2  # conversion kinds
 
 
 class OracleError(ValueError):
@@ -53,6 +61,39 @@ def _payload(blob: np.ndarray, e) -> np.ndarray:
     if raw.size != e.byte_length:
         raise OracleError(f"{e.fqn}: byte range outside its buffer")
     return np.ascontiguousarray(raw).view(_UINT[e.itemsize])
+
+
+def f32_to_bf16(bits: np.ndarray) -> np.ndarray:
+    """binary32 bit patterns (uint32) -> bfloat16 bit patterns (uint16), round to nearest, ties
+    to even.  A bfloat16 is a binary32 whose low 16 bits are zero, and for non-negative floats
+    the order of bit patterns is the order of values, so the two candidates for |x| are the
+    pattern with its low half cleared (`below`) and the next bfloat16 pattern (`above`; past
+    the largest finite one it stands for 2^128, as IEEE 754 rounding prescribes before
+    overflow turns it into infinity).  Distances are taken in float64, where they are exact.
+    NaN (any payload, either sign) -> 0x7FC0."""
+    bits = np.asarray(bits, dtype=np.uint32)
+    sign = bits & np.uint32(0x80000000)
+    mag = bits & np.uint32(0x7FFFFFFF)
+    nan = mag > np.uint32(0x7F800000)
+    below = mag & np.uint32(0xFFFF0000)
+    above = (below.astype(np.uint64) + 0x10000).astype(np.uint32)  # at most 0x7F800000 for finite input
+    value = lambda pattern: pattern.view(np.float32).astype(np.float64)  # noqa: E731
+    with np.errstate(invalid="ignore", over="ignore"):
+        x = value(mag)
+        v_above = np.where(above == np.uint32(0x7F800000), 2.0 ** 128, value(above))
+        d_below, d_above = x - value(below), v_above - x
+        below_is_odd = ((below >> np.uint32(16)) & np.uint32(1)) == 1
+        up = (d_above < d_below) | ((d_above == d_below) & below_is_odd)
+    up &= mag < np.uint32(0x7F800000)  # infinity stays
+    out = np.where(up, above, below) | sign
+    out = np.where(nan, np.uint32(0x7FC00000), out)
+    return (out >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) -> binary32 bit patterns (uint32): a bfloat16 IS the upper
+    half of a binary32, so the value is unchanged when 16 zero bits are appended."""
+    return np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
 
 
 def check_family(entries: Sequence) -> Tuple[Tuple[int, ...], int]:
@@ -121,15 +162,30 @@ def group_by_fqn(entries: Iterable) -> Dict[str, List]:
 
 
 def reshard_fqn(src_entries: Sequence, src_payloads: Sequence[np.ndarray], dst_entries: Sequence,
-                allow_replicas: bool = False) -> List[np.ndarray]:
-    """Bytes of every wanted shard of ONE FQN, given the payloads of its saved shards."""
-    shape, itemsize = check_family(list(src_entries) + list(dst_entries))
+                allow_replicas: bool = False, convert=None) -> List[np.ndarray]:
+    """Bytes of every wanted shard of ONE FQN, given the payloads of its saved shards.
+    convert = (kind, saved dtype_tag, wanted dtype_tag): a tensor saved with the first tag and
+    wanted with the second is converted element by element after it has been assembled."""
+    s0, d0 = src_entries[0], dst_entries[0]
+    if (s0.itemsize, s0.dtype_tag) == (d0.itemsize, d0.dtype_tag):
+        shape, itemsize = check_family(list(src_entries) + list(dst_entries))
+        T, cover = assemble(shape, itemsize, src_entries, src_payloads, first_wins=allow_replicas)
+        return [take(T, cover, d, replicas_ok=allow_replicas) for d in dst_entries]
+    sizes = {F32_TO_BF16: (4, 2), BF16_TO_F32: (2, 4)}
+    if (convert is None or (s0.dtype_tag, d0.dtype_tag) != tuple(convert[1:])
+            or (s0.itemsize, d0.itemsize) != sizes[convert[0]]):
+        raise OracleError(f"{s0.fqn}: saved and wanted entries disagree on dtype")
+    shape, itemsize = check_family(list(src_entries))
+    if check_family(list(dst_entries))[0] != shape:
+        raise OracleError(f"{s0.fqn}: entries disagree on global shape or dtype")
     T, cover = assemble(shape, itemsize, src_entries, src_payloads, first_wins=allow_replicas)
+    T = f32_to_bf16(T) if convert[0] == F32_TO_BF16 else bf16_to_f32(T)
     return [take(T, cover, d, replicas_ok=allow_replicas) for d in dst_entries]
 
 
 def reshard(src_metas: Sequence, src_blobs: Sequence[np.ndarray], dst_metas: Sequence,
-            dst_buf_bytes: Sequence[int], fill_byte: int = 0, allow_replicas: bool = False) -> List[np.ndarray]:
+            dst_buf_bytes: Sequence[int], fill_byte: int = 0, allow_replicas: bool = False,
+            convert=None) -> List[np.ndarray]:
     """Every target rank buffer (uint8 arrays); bytes no entry names keep `fill_byte`.
     allow_replicas: saved shards may be stored more than once (a checkpoint written without
     de-duplication); the first entry in input order supplies the bytes."""
@@ -142,7 +198,7 @@ def reshard(src_metas: Sequence, src_blobs: Sequence[np.ndarray], dst_metas: Seq
                 continue
             raise OracleError(f"{fqn}: wanted but never saved")
         payloads = [_payload(src_blobs[s.buf_index], s) for s in srcs]
-        for d, data in zip(dsts, reshard_fqn(srcs, payloads, dsts, allow_replicas)):
+        for d, data in zip(dsts, reshard_fqn(srcs, payloads, dsts, allow_replicas, convert)):
             buf = out[d.buf_index]
             if d.byte_offset + d.byte_length > buf.size:
                 raise OracleError(f"{fqn}: target byte range outside its buffer")

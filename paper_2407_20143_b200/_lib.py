@@ -47,6 +47,9 @@ class PlanOptsC(C.Structure):
         ("tma_wait_ms", C.c_uint32),
         ("fanout", C.c_uint32),
         ("test_stall", C.c_uint32),
+        ("convert", C.c_uint32),
+        ("convert_src_tag", C.c_uint32),
+        ("convert_dst_tag", C.c_uint32),
     ]
 
 
@@ -69,7 +72,7 @@ class PlanStatsC(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "n_src_entries", "n_dst_entries", "n_fqns", "n_intersections", "n_items", "n_tiles", "n_small_tiles",
         "n_strided_tiles", "n_tma_tiles", "bytes_copied", "bytes_src_unique", "bytes_misaligned")] + [
-        ("plan_ms", C.c_double)]
+        ("plan_ms", C.c_double), ("n_cvt_tiles", C.c_uint64)]
 
 
 class ExportEntryC(C.Structure):

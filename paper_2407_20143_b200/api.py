@@ -21,6 +21,8 @@ class BcpError(RuntimeError):
 ERR_INVALID, ERR_MISMATCH, ERR_OVERLAP, ERR_UNCOVERED, ERR_BOUNDS, ERR_DST_ALIAS = -1, -2, -3, -4, -5, -6
 ERR_CUDA, ERR_NOMEM, ERR_DEVICE_TIMEOUT, ERR_CAPACITY = -7, -8, -9, -10
 TILE_GRAN_MASK, TILE_ZERO, TILE_SMALL, TILE_TMA, TILE_TMA2D, TILE_FOLLOW = 0x7, 0x8, 0x10, 0x20, 0x40, 0x80
+TILE_CVT_SHIFT, TILE_CVT_MASK = 11, 3 << 11
+CONVERT_NONE, CONVERT_F32_TO_BF16, CONVERT_BF16_TO_F32 = 0, 1, 2
 
 
 def _check(rc: int) -> None:

@@ -15,8 +15,9 @@ using namespace bcp;
 struct bcp_plan_s {
   Options opt;
   bcp_plan_stats_t stats;
-  TileVec tiles;  // TMA units, then other CTA-wide units, then warp units
-  size_t n_tma = 0, n_big = 0;
+  TileVec tiles;  // TMA units, then other CTA-wide units, then warp units, then converting units
+  size_t n_tma = 0, n_big = 0, n_cvt = 0;
+  size_t n_small() const { return tiles.size() - n_tma - n_big - n_cvt; }
   std::vector<uint64_t> src_bytes, dst_bytes;
   std::vector<Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
   std::vector<Gap> gaps;    // target bytes no entry names (zeroed by the host-buffer call)
@@ -27,8 +28,8 @@ struct bcp_plan_s {
   bcp_tile* d_tiles = nullptr;
   bcp_tile* d_fan_tiles = nullptr;  // the same list with replica groups marked (in-place host path)
   void** d_ptrs = nullptr;  // source table followed by target table
-  Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel
-  uint32_t grid = 0, tma_grid = 0;
+  Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel, [2] converting kernel
+  uint32_t grid = 0, tma_grid = 0, cvt_grid = 0;
   cudaStream_t last_stream = nullptr;
   bool ran = false;
   std::vector<void*> h_ptrs;
@@ -36,7 +37,7 @@ struct bcp_plan_s {
   // bcp_reshard_host: device staging plus a second copy of the work list grouped by target
   // buffer, so that uploads, kernels and downloads of different target buffers overlap
   struct Group {  // units of one target buffer inside d_host_tiles
-    size_t first = 0, n_tma = 0, n_big = 0, n_small = 0;
+    size_t first = 0, n_tma = 0, n_big = 0, n_small = 0, n_cvt = 0;
     std::vector<uint32_t> needs;  // source buffers its units read
   };
   std::vector<void*> stage_src, stage_dst;
@@ -66,8 +67,8 @@ int bind_device_alloc(bcp_plan_t* p) {
     BCP_CUDA(cudaMalloc(&p->d_maps, p->rects.size() * 2 * sizeof(CUtensorMap)));
     p->h_maps.resize(p->rects.size() * 2);
   }
-  BCP_CUDA(cudaMalloc(&p->d_ctrl, 2 * sizeof(Control)));
-  BCP_CUDA(cudaMemset(p->d_ctrl, 0, 2 * sizeof(Control)));
+  BCP_CUDA(cudaMalloc(&p->d_ctrl, 3 * sizeof(Control)));
+  BCP_CUDA(cudaMemset(p->d_ctrl, 0, 3 * sizeof(Control)));
   if (p->opt.worker == 2) {
     BCP_CUDA(warp_kernel_max_grid(p->opt.ctas_per_sm, &p->grid));
   } else {
@@ -75,6 +76,7 @@ int bind_device_alloc(bcp_plan_t* p) {
   }
   if (p->n_tma)
     BCP_CUDA(tma_kernel_max_grid(p->opt.tma_stage_bytes, p->opt.tma_stages, p->opt.tma_ctas_per_sm, &p->tma_grid));
+  if (p->n_cvt) BCP_CUDA(convert_kernel_max_grid(&p->cvt_grid));
   p->h_ptrs.resize(n_ptrs);
   return BCP_OK;
 }
@@ -156,8 +158,9 @@ int upload_tables(bcp_plan_t* p, cudaStream_t stream) {
   return BCP_OK;
 }
 
-// Enqueue the kernels for a slice of a device work list laid out as [TMA | CTA-wide | warp units].
-int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_big, size_t n_small, cudaStream_t stream) {
+// Enqueue the kernels for a slice of a device work list laid out as [TMA | CTA-wide | warp | converting units].
+int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_big, size_t n_small, size_t n_cvt,
+                 cudaStream_t stream) {
   const size_t ns = p->src_bytes.size();
   if (n_tma) {
     TmaLaunchArgs t;
@@ -195,6 +198,16 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
   a.cache_hints = p->opt.cache_hints;
   a.unroll = p->opt.unroll;
   if (units) BCP_CUDA(launch_copy(a, stream));
+  if (n_cvt) {
+    ConvertLaunchArgs c;
+    c.tiles = tiles + n_tma + n_big + n_small;
+    c.n_units = uint32_t(n_cvt);
+    c.src = a.src;
+    c.dst = a.dst;
+    c.ctrl = p->d_ctrl + 2;
+    c.grid = p->cvt_grid;
+    BCP_CUDA(launch_convert(c, stream));
+  }
   return BCP_OK;
 }
 
@@ -226,7 +239,7 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
     for (size_t i = 0; i < nd; ++i) p->h_ptrs[ns + i] = dst[i];
     if (int rc = upload_tables(p, stream)) return rc;
   }
-  if (int rc = launch_units(p, list ? list : p->d_tiles, p->n_tma, p->n_big, p->tiles.size() - p->n_tma - p->n_big, stream)) return rc;
+  if (int rc = launch_units(p, list ? list : p->d_tiles, p->n_tma, p->n_big, p->n_small(), p->n_cvt, stream)) return rc;
   p->last_stream = stream;
   p->ran = true;
   return BCP_OK;
@@ -240,7 +253,7 @@ bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_s
   p->stats = stats;
   p->src_bytes = std::move(src_bytes);
   p->dst_bytes = std::move(dst_bytes);
-  build_tiles(items, p->opt, &p->src_bytes, &p->tiles, &p->n_tma, &p->n_big, &p->rects, &p->stats);
+  build_tiles(items, p->opt, &p->src_bytes, &p->tiles, &p->n_tma, &p->n_big, &p->n_cvt, &p->rects, &p->stats);
   return p;
 }
 
@@ -353,14 +366,14 @@ int prepare_host_path(bcp_plan_t* p) {
   if (p->s_h2d) return BCP_OK;
   const size_t ns = p->src_bytes.size(), nd = p->dst_bytes.size();
   p->groups.assign(nd, bcp_plan_s::Group());
-  std::vector<std::vector<bcp_tile>> tma(nd), big(nd), small(nd);
+  std::vector<std::vector<bcp_tile>> tma(nd), big(nd), small(nd), cvt(nd);
   std::vector<std::vector<char>> need(nd, std::vector<char>(ns, 0));
   for (const bcp_tile& t : p->tiles) {
     const uint32_t d = t.dst_buf;
     if (!(t.flags & BCP_TILE_ZERO)) need[d][t.src_buf] = 1;
     bcp_tile u = t;
     u.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));  // groups are per target buffer here: every unit is staged on its own
-    ((u.flags & BCP_TILE_TMA) ? tma : (u.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(u);
+    ((u.flags & BCP_TILE_CVT_MASK) ? cvt : (u.flags & BCP_TILE_TMA) ? tma : (u.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(u);
   }
   std::vector<bcp_tile> flat;
   flat.reserve(p->tiles.size());
@@ -370,9 +383,11 @@ int prepare_host_path(bcp_plan_t* p) {
     g.n_tma = tma[d].size();
     g.n_big = big[d].size();
     g.n_small = small[d].size();
+    g.n_cvt = cvt[d].size();
     flat.insert(flat.end(), tma[d].begin(), tma[d].end());
     flat.insert(flat.end(), big[d].begin(), big[d].end());
     flat.insert(flat.end(), small[d].begin(), small[d].end());
+    flat.insert(flat.end(), cvt[d].begin(), cvt[d].end());
     for (uint32_t sb = 0; sb < ns; ++sb)
       if (need[d][sb]) g.needs.push_back(sb);
   }
@@ -432,7 +447,7 @@ void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vec
 
 extern "C" {
 
-int bcp_version(void) { return 100; }
+int bcp_version(void) { return 200; }  // 0.2.0: plan images carry converting units
 
 const char* bcp_last_error(void) { return last_error().c_str(); }
 
@@ -494,7 +509,7 @@ int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_by
     std::vector<Gap> gaps;
     bcp_plan_stats_t st;
     memset(&st, 0, sizeof st);
-    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt.allow_replicas != 0, &items, &gaps, &st))
+    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt, &items, &gaps, &st))
       return rc;
     bcp_plan_t* p = finish_plan(items, opt, st, std::vector<uint64_t>(src_buf_bytes, src_buf_bytes + n_src_bufs),
                               std::vector<uint64_t>(dst_buf_bytes, dst_buf_bytes + n_dst_bufs));
@@ -525,7 +540,7 @@ struct ImageHeader {
   uint32_t version, tile_size;
   Options opt;
   bcp_plan_stats_t stats;
-  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects, n_gaps;
+  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects, n_gaps, n_cvt;
 };
 uint64_t fnv1a(const unsigned char* p, size_t n) {
   uint64_t h = 1469598103934665603ull;
@@ -536,6 +551,18 @@ uint64_t fnv1a(const unsigned char* p, size_t n) {
 bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db, const std::vector<Rect>& rects,
              const Options& opt) {
   if (t.rows == 0 || t.row_bytes == 0 || t.dst_buf >= db.size()) return false;
+  if (const uint32_t kind = (t.flags & BCP_TILE_CVT_MASK) >> BCP_TILE_CVT_SHIFT) {
+    // converting unit: element-aligned on both sides, source rows hold the same number of elements
+    if (kind > BCP_CONVERT_BF16_TO_F32 || (t.flags & ~(BCP_TILE_GRAN_MASK | BCP_TILE_CVT_MASK)) || t.src_buf >= sb.size()) return false;
+    const uint64_t s_isz = kind == BCP_CONVERT_F32_TO_BF16 ? 4 : 2, d_isz = 6 - s_isz;
+    const uint64_t s_row = uint64_t(t.row_bytes) / d_isz * s_isz;
+    if (t.row_bytes % d_isz || t.dst_off % d_isz || t.dst_pitch % d_isz || t.src_off % s_isz || t.src_pitch % s_isz) return false;
+    if (t.rows > 1 && (t.dst_pitch < t.row_bytes || t.src_pitch < s_row)) return false;
+    const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes, span_s = uint64_t(t.rows - 1) * t.src_pitch + s_row;
+    if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
+    if (t.src_off > sb[t.src_buf] || span_s > sb[t.src_buf] - t.src_off) return false;
+    return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
+  }
   const bool zero = t.flags & BCP_TILE_ZERO;
   const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes;
   if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
@@ -600,6 +627,7 @@ int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n)
   h.n_dst_bufs = plan->dst_bytes.size();
   h.n_tma = plan->n_tma;
   h.n_big = plan->n_big;
+  h.n_cvt = plan->n_cvt;
   h.n_tiles = plan->tiles.size();
   h.n_rects = plan->rects.size();
   h.n_gaps = plan->gaps.size();
@@ -631,7 +659,7 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image of library version %u, this is %d", h.version, bcp_version());
   const uint64_t lim = uint64_t(1) << 32;
   if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_rects >= lim || h.n_gaps >= lim || h.n_tma > h.n_tiles ||
-      h.n_big > h.n_tiles - h.n_tma)
+      h.n_big > h.n_tiles - h.n_tma || h.n_cvt > h.n_tiles - h.n_tma - h.n_big)
     return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: implausible counts");
   const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) +
                         h.n_rects * sizeof(Rect) + h.n_gaps * sizeof(Gap) + sizeof(uint64_t);
@@ -671,6 +699,7 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
     if (h.n_gaps) memcpy(p->gaps.data(), q, h.n_gaps * sizeof(Gap));
     p->n_tma = h.n_tma;
     p->n_big = h.n_big;
+    p->n_cvt = h.n_cvt;
   } catch (const std::bad_alloc&) {
     delete p;
     return fail(BCP_ERR_NOMEM, "out of host memory");
@@ -701,9 +730,9 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   }
   for (size_t i = 0; i < p->tiles.size(); ++i) {
     const bcp_tile& t = p->tiles[i];
-    const bool in_tma = i < p->n_tma, in_small = i >= p->n_tma + p->n_big;
+    const bool in_tma = i < p->n_tma, in_cvt = i >= p->tiles.size() - p->n_cvt, in_small = i >= p->n_tma + p->n_big && !in_cvt;
     if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->rects, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
-        bool(t.flags & BCP_TILE_SMALL) != in_small) {
+        bool(t.flags & BCP_TILE_SMALL) != in_small || bool(t.flags & BCP_TILE_CVT_MASK) != in_cvt) {
       delete p;
       return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: work unit %zu is inconsistent with the recorded buffers", i);
     }
@@ -797,7 +826,7 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
     if (!p->dst_bytes[d]) continue;
     for (uint32_t sb : g.needs) BCP_CUDA(cudaStreamWaitEvent(stream, p->ev_src[sb], 0));
     BCP_CUDA(cudaMemsetAsync(p->stage_dst[d], 0, p->dst_bytes[d], stream));
-    if (int rc = launch_units(p, p->d_host_tiles + g.first, g.n_tma, g.n_big, g.n_small, stream)) return rc;
+    if (int rc = launch_units(p, p->d_host_tiles + g.first, g.n_tma, g.n_big, g.n_small, g.n_cvt, stream)) return rc;
     BCP_CUDA(cudaEventRecord(p->ev_dst[d], stream));
     BCP_CUDA(cudaStreamWaitEvent(p->s_d2h, p->ev_dst[d], 0));
     BCP_CUDA(cudaMemcpyAsync(dst_host[d], p->stage_dst[d], p->dst_bytes[d], cudaMemcpyDeviceToHost, p->s_d2h));

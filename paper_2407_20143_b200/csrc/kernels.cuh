@@ -1,4 +1,5 @@
-// Launch interface between the C ABI (api.cu) and the sm_100a kernels (kernels.cu).
+// Launch interface between the C ABI (api.cu) and the sm_100a kernels (kernels.cu, tma_kernel.cu,
+// convert_kernel.cu).
 #pragma once
 
 #include <cuda_runtime.h>
@@ -46,6 +47,21 @@ struct TmaLaunchArgs {
   uint32_t cache_hints;   // 3: evict-first stores; 4: evict-first loads too; else none
   const void* maps;       // device: two 128-byte tensor maps (source view, target view) per tensor-map rectangle
 };
+
+struct ConvertLaunchArgs {
+  const bcp_tile* tiles;  // device: n_units converting units (BCP_TILE_CVT_MASK set)
+  uint32_t n_units;
+  const void* const* src;
+  void* const* dst;
+  Control* ctrl;          // device, separate from the other kernels'
+  uint32_t grid;
+};
+
+// Persistent grid of the converting kernel (256-thread CTAs, every warp a worker).
+cudaError_t convert_kernel_max_grid(uint32_t* grid);
+
+// Enqueue the converting kernel on `stream`.
+cudaError_t launch_convert(const ConvertLaunchArgs& a, cudaStream_t stream);
 
 // Persistent grid of the TMA staging kernel (one warp per CTA) for a stage geometry.
 cudaError_t tma_kernel_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_t ctas_per_sm, uint32_t* grid);

@@ -25,6 +25,9 @@ struct Item {
   uint64_t rows = 1;
   uint32_t src_buf = 0, dst_buf = 0;
   bool zero = false;  // no source: write zeros
+  uint8_t cvt = 0;    // BCP_CONVERT_*: row_bytes counts target bytes, the source row holds the same elements
+  // bytes of one source row
+  uint64_t src_row_bytes() const { return cvt == BCP_CONVERT_F32_TO_BF16 ? row_bytes * 2 : cvt == BCP_CONVERT_BF16_TO_F32 ? row_bytes / 2 : row_bytes; }
 };
 
 struct Options {
@@ -45,6 +48,7 @@ struct Options {
   uint32_t tma_wait_ms = 2000;
   uint32_t test_stall = 0;
   uint32_t fanout = 1;  // 1 on, 2 off
+  uint32_t convert = 0, convert_src_tag = 0, convert_dst_tag = 0;
 };
 
 // A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source
@@ -73,10 +77,10 @@ void decompose(const int64_t* lengths, uint32_t ndim, int64_t a, int64_t b, std:
 // counters of `stats`.
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    bool allow_replicas, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats);
+                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats);
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
-// tiles = [TMA units..., other CTA-wide units..., warp units...].
+// tiles = [TMA units..., other CTA-wide units..., warp units..., converting units...].
 // Mark groups of TMA units (ordered by source address) that read the same source bytes.
 void mark_followers(bcp_tile* tma, size_t n);
 
@@ -106,6 +110,6 @@ using TileVec = std::vector<bcp_tile, NoInitAlloc<bcp_tile>>;
 // Large lists are built by several host threads (at most 8; the environment variable
 // BCP_PLAN_THREADS overrides the count); the result does not depend on how many.
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes, TileVec* tiles,
-                 size_t* n_tma, size_t* n_big, std::vector<Rect>* rects, bcp_plan_stats_t* stats);
+                 size_t* n_tma, size_t* n_big, size_t* n_cvt, std::vector<Rect>* rects, bcp_plan_stats_t* stats);
 
 }  // namespace bcp

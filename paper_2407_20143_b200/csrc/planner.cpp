@@ -57,6 +57,9 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     if (in->tma_wait_ms) o.tma_wait_ms = in->tma_wait_ms;
     o.test_stall = in->test_stall;
     if (in->fanout) o.fanout = in->fanout;
+    o.convert = in->convert;
+    o.convert_src_tag = in->convert_src_tag;
+    o.convert_dst_tag = in->convert_dst_tag;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -80,6 +83,11 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.fanout != 1 && o.fanout != 2) return fail(BCP_ERR_INVALID, "fanout must be 0, 1 or 2");
   if (o.tma_wait_ms > 60000) return fail(BCP_ERR_INVALID, "tma_wait_ms must not exceed 60000");
   if (o.worker > 2) return fail(BCP_ERR_INVALID, "worker must be 0, 1 or 2");
+  if (o.convert > BCP_CONVERT_BF16_TO_F32) return fail(BCP_ERR_INVALID, "convert must be 0, 1 or 2");
+  if (o.convert && o.convert_src_tag == o.convert_dst_tag)
+    return fail(BCP_ERR_INVALID, "convert needs two different dtype tags (convert_src_tag, convert_dst_tag)");
+  if (!o.convert && (o.convert_src_tag || o.convert_dst_tag))
+    return fail(BCP_ERR_INVALID, "convert_src_tag / convert_dst_tag are set but convert is 0");
   if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
     return fail(BCP_ERR_INVALID, "tma_min_row_bytes must be a multiple of 16 in [16, 65536]");
   *out = o;
@@ -172,7 +180,10 @@ struct Entry {  // one regular box with its bytes
 
 struct Family {
   const char* fqn;
-  uint32_t itemsize, dtype_tag, ndim;
+  uint32_t itemsize, dtype_tag, ndim;  // of the saved side (of the wanted side while nothing is saved)
+  uint32_t d_itemsize, d_tag;          // of the wanted side (differs only under a conversion)
+  uint32_t cvt;                        // BCP_CONVERT_* applied to this tensor
+  bool has_src, has_dst;
   int64_t shape[BCP_MAX_NDIM];
   std::vector<Entry> src, dst;
 };
@@ -269,8 +280,8 @@ inline bool intersect(const Entry& a, const Entry& b, uint32_t ndim, int64_t* of
 
 // One matched segment -> copy items.  The segment `off/len` lies inside both the saved box s
 // and the wanted box d, each stored densely in C order.
-void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t isz, const int64_t* off, const int64_t* len,
-           std::vector<Item>* items) {
+void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t s_isz, uint32_t d_isz, uint32_t cvt, const int64_t* off,
+           const int64_t* len, std::vector<Item>* items) {
   // element strides of the containing boxes and byte offsets of the segment's origin
   int64_t ss[BCP_MAX_NDIM], ds[BCP_MAX_NDIM];
   int64_t sacc = 1, dacc = 1;
@@ -282,8 +293,8 @@ void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t isz, const in
   }
   uint64_t so = s.byte_off, dof = d.byte_off;
   for (uint32_t k = 0; k < ndim; ++k) {
-    so += uint64_t(off[k] - s.off[k]) * uint64_t(ss[k]) * isz;
-    dof += uint64_t(off[k] - d.off[k]) * uint64_t(ds[k]) * isz;
+    so += uint64_t(off[k] - s.off[k]) * uint64_t(ss[k]) * s_isz;
+    dof += uint64_t(off[k] - d.off[k]) * uint64_t(ds[k]) * d_isz;
   }
   // dims of extent > 1, outer to inner, with byte strides
   struct Dim {
@@ -292,13 +303,13 @@ void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t isz, const in
   Dim dims[BCP_MAX_NDIM + 1];
   int nd = 0;
   for (uint32_t k = 0; k < ndim; ++k)
-    if (len[k] > 1) dims[nd++] = Dim{uint64_t(len[k]), uint64_t(ss[k]) * isz, uint64_t(ds[k]) * isz};
+    if (len[k] > 1) dims[nd++] = Dim{uint64_t(len[k]), uint64_t(ss[k]) * s_isz, uint64_t(ds[k]) * d_isz};
   // the innermost dim must be a dense run of elements on both sides; otherwise add a run of one element
-  if (nd == 0 || dims[nd - 1].sp != isz || dims[nd - 1].dp != isz) dims[nd++] = Dim{1, isz, isz};
-  // merge a dim into the run while it is dense on both sides
-  uint64_t run = dims[nd - 1].n * isz;
+  if (nd == 0 || dims[nd - 1].sp != s_isz || dims[nd - 1].dp != d_isz) dims[nd++] = Dim{1, s_isz, d_isz};
+  // merge a dim into the run (counted in elements) while it is dense on both sides
+  uint64_t run = dims[nd - 1].n;
   --nd;
-  while (nd > 0 && dims[nd - 1].sp == run && dims[nd - 1].dp == run) {
+  while (nd > 0 && dims[nd - 1].sp == run * s_isz && dims[nd - 1].dp == run * d_isz) {
     run *= dims[nd - 1].n;
     --nd;
   }
@@ -315,7 +326,8 @@ void lower(const Entry& s, const Entry& d, uint32_t ndim, uint32_t isz, const in
   Item it;
   it.src_buf = s.buf;
   it.dst_buf = d.buf;
-  it.row_bytes = run;
+  it.row_bytes = run * d_isz;
+  it.cvt = uint8_t(cvt);
   if (nd == 0) {
     it.src_off = so;
     it.dst_off = dof;
@@ -363,19 +375,24 @@ struct SegKey {
 
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    bool allow_replicas, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
+                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
+  const bool allow_replicas = opt.allow_replicas != 0;
   if ((n_src && !src) || (n_dst && !dst) || (n_src_bufs && !src_buf_bytes) || (n_dst_bufs && !dst_buf_bytes))
     return fail(BCP_ERR_INVALID, "bcp_plan: NULL array with non-zero count");
   std::unordered_map<std::string_view, uint32_t> ids;  // keys point into the caller's metas
   std::vector<Family> fams;
-  auto family_of = [&](const bcp_shard_meta& m, const char* side, size_t i, uint32_t* id) -> int {
+  const char* const kDiffers = "%s[%zu] %s: itemsize, dtype_tag, ndim or global shape differs from an earlier entry";
+  auto family_of = [&](const bcp_shard_meta& m, const char* side, size_t i, bool wanted, uint32_t* id) -> int {
     const std::string_view name(m.fqn);
     auto it = ids.find(name);
     if (it == ids.end()) {
       Family f;
       f.fqn = m.fqn;
-      f.itemsize = m.itemsize;
-      f.dtype_tag = m.dtype_tag;
+      f.itemsize = f.d_itemsize = m.itemsize;
+      f.dtype_tag = f.d_tag = m.dtype_tag;
+      f.cvt = 0;
+      f.has_src = !wanted;
+      f.has_dst = wanted;
       f.ndim = m.ndim;
       for (uint32_t k = 0; k < BCP_MAX_NDIM; ++k) f.shape[k] = k < m.ndim ? m.global_shape[k] : 1;
       *id = uint32_t(fams.size());
@@ -383,21 +400,34 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       fams.push_back(std::move(f));
       return BCP_OK;
     }
-    const Family& f = fams[it->second];
-    bool same = f.itemsize == m.itemsize && f.dtype_tag == m.dtype_tag && f.ndim == m.ndim;
-    for (uint32_t k = 0; same && k < m.ndim; ++k) same = f.shape[k] == m.global_shape[k];
-    if (!same)
-      return fail(BCP_ERR_MISMATCH, "%s[%zu] %s: itemsize, dtype_tag, ndim or global shape differs from an earlier entry",
-                  side, i, m.fqn);
+    Family& f = fams[it->second];
     *id = it->second;
-    return BCP_OK;
+    bool same = f.ndim == m.ndim;
+    for (uint32_t k = 0; same && k < m.ndim; ++k) same = f.shape[k] == m.global_shape[k];
+    if (!same) return fail(BCP_ERR_MISMATCH, kDiffers, side, i, m.fqn);
+    if (!wanted || f.has_dst) {  // later entries of a side repeat that side's dtype
+      const bool ok = wanted ? (f.d_itemsize == m.itemsize && f.d_tag == m.dtype_tag) : (f.itemsize == m.itemsize && f.dtype_tag == m.dtype_tag);
+      return ok ? BCP_OK : fail(BCP_ERR_MISMATCH, kDiffers, side, i, m.fqn);
+    }
+    // first wanted entry of a saved tensor: same dtype, or the pair the caller asked to convert
+    f.has_dst = true;
+    f.d_itemsize = m.itemsize;
+    f.d_tag = m.dtype_tag;
+    if (f.itemsize == m.itemsize && f.dtype_tag == m.dtype_tag) return BCP_OK;
+    const uint32_t s_isz = opt.convert == BCP_CONVERT_F32_TO_BF16 ? 4 : 2, d_isz = 6 - s_isz;
+    if (opt.convert && f.dtype_tag == opt.convert_src_tag && m.dtype_tag == opt.convert_dst_tag && f.itemsize == s_isz &&
+        m.itemsize == d_isz) {
+      f.cvt = opt.convert;
+      return BCP_OK;
+    }
+    return fail(BCP_ERR_MISMATCH, kDiffers, side, i, m.fqn);
   };
   std::vector<RelBox> scratch;
   for (size_t i = 0; i < n_src; ++i) {
     int64_t n;
     uint32_t f;
     if (int rc = check_meta(src[i], "src", i, src_buf_bytes, n_src_bufs, &n)) return rc;
-    if (int rc = family_of(src[i], "src", i, &f)) return rc;
+    if (int rc = family_of(src[i], "src", i, false, &f)) return rc;
     expand(src[i], uint32_t(i), n, &fams[f].src, &scratch);
   }
   // target byte ranges must not overlap inside a buffer
@@ -412,7 +442,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       int64_t n;
       uint32_t f;
       if (int rc = check_meta(dst[i], "dst", i, dst_buf_bytes, n_dst_bufs, &n)) return rc;
-      if (int rc = family_of(dst[i], "dst", i, &f)) return rc;
+      if (int rc = family_of(dst[i], "dst", i, true, &f)) return rc;
       expand(dst[i], uint32_t(i), n, &fams[f].dst, &scratch);
       if (n > 0) rs.push_back(Range{dst[i].byte_offset, dst[i].byte_offset + dst[i].byte_length, dst[i].buf_index, uint32_t(i)});
     }
@@ -486,7 +516,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
         if (!intersect(s, d, nd, o, l)) continue;
         covered += volume(l, 0, nd);
         ++n_inter;
-        lower(s, d, nd, f.itemsize, o, l, items);
+        lower(s, d, nd, f.itemsize, f.d_itemsize, f.cvt, o, l, items);
         SegKey key = {si, 0, 0, uint64_t(volume(l, 0, nd)) * f.itemsize};
         for (uint32_t k = 0; k < nd; ++k) {
           key.first = key.first * uint64_t(s.len[k]) + uint64_t(o[k] - s.off[k]);
@@ -549,16 +579,17 @@ void parallel_jobs(size_t n_jobs, unsigned threads, F&& job) {
   for (std::thread& t : pool) t.join();
 }
 
-enum { kTma = 0, kBig = 1, kSmall = 2 };  // unit classes, in the order of the final list
+enum { kTma = 0, kBig = 1, kSmall = 2, kCvt = 3, kClasses = 4 };  // unit classes, in the order of the final list
 
 struct Tally {
   uint64_t bytes_copied = 0, bytes_misaligned = 0, n_strided = 0;
   uint64_t tma_bytes = 0;   // payload of the TMA class ...
   uint64_t tma_busy = 0;    // ... in shifted runs and rectangles with rows under 2 KiB (the warp issues a lot)
   uint64_t tma_boxed = 0;   // ... in tensor-map boxes
+  uint64_t cvt_bytes = 0;   // target bytes written by converting units
   void add(const Tally& o) {
     bytes_copied += o.bytes_copied, bytes_misaligned += o.bytes_misaligned, n_strided += o.n_strided;
-    tma_bytes += o.tma_bytes, tma_busy += o.tma_busy, tma_boxed += o.tma_boxed;
+    tma_bytes += o.tma_bytes, tma_busy += o.tma_busy, tma_boxed += o.tma_boxed, cvt_bytes += o.cvt_bytes;
   }
 };
 
@@ -568,9 +599,9 @@ struct Cutter {
   const Options& opt;
   const std::vector<uint64_t>* src_bytes;  // source buffer sizes (may be null: unknown)
   bool demote;                             // small job: TMA-eligible units go to the register kernel
-  bcp_tile* out[3];
+  bcp_tile* out[kClasses];
   Rect* rects_out;
-  size_t pos[3];
+  size_t pos[kClasses];
   size_t rect_pos;
   Tally st;
 
@@ -700,7 +731,56 @@ struct Cutter {
     return true;
   }
 
+  // Converting units: rows x row_bytes TARGET bytes each; no staging path, no warp path.
+  void emit_cvt(const Item& it, uint64_t src_off, uint64_t dst_off, uint64_t rows, uint64_t row_bytes) {
+    bcp_tile t;
+    memset(&t, 0, sizeof t);
+    t.src_off = src_off;
+    t.dst_off = dst_off;
+    t.rows = uint32_t(rows);
+    t.row_bytes = uint32_t(row_bytes);
+    t.src_buf = it.src_buf;
+    t.dst_buf = it.dst_buf;
+    if (rows > 1) {
+      t.src_pitch = it.src_pitch;
+      t.dst_pitch = it.dst_pitch;
+      ++st.n_strided;
+    }
+    const uint32_t g = gran_log2(t.src_off | t.dst_off | t.row_bytes | t.src_pitch | t.dst_pitch);
+    t.flags = g | (uint32_t(it.cvt) << BCP_TILE_CVT_SHIFT);
+    if (g < 4) st.bytes_misaligned += rows * row_bytes;
+    st.bytes_copied += rows * row_bytes;
+    st.cvt_bytes += rows * row_bytes;
+    put(kCvt, t);
+  }
+
+  void cut_cvt(const Item& it) {
+    const uint64_t unit = opt.tile_bytes;
+    auto src_bytes_of = [&](uint64_t dst_bytes) { return it.cvt == BCP_CONVERT_F32_TO_BF16 ? dst_bytes * 2 : dst_bytes / 2; };
+    if (it.rows > 1 && it.row_bytes < unit) {  // groups of whole rows
+      const uint64_t rpt = std::max<uint64_t>(1, unit / it.row_bytes);
+      for (uint64_t r = 0; r < it.rows; r += rpt)
+        emit_cvt(it, it.src_off + r * it.src_pitch, it.dst_off + r * it.dst_pitch, std::min(rpt, it.rows - r), it.row_bytes);
+      return;
+    }
+    for (uint64_t r = 0; r < it.rows; ++r) {  // every row is a run, cut so that later units start 256-byte aligned
+      uint64_t so = it.src_off + r * it.src_pitch, dof = it.dst_off + r * it.dst_pitch, n = it.row_bytes;
+      uint64_t first = unit;
+      if (n > unit && (dof & 255)) first = unit - (dof & 255);
+      while (n) {
+        const uint64_t c = std::min(n, first);
+        emit_cvt(it, so, dof, 1, c);
+        so += src_bytes_of(c), dof += c, n -= c;
+        first = unit;
+      }
+    }
+  }
+
   void cut(const Item& it) {
+    if (it.cvt) {
+      cut_cvt(it);
+      return;
+    }
     if (it.rows <= 1 || it.row_bytes == 0) {
       cut_run(it, it.src_off, it.dst_off, it.rows ? it.row_bytes : 0);
       return;
@@ -786,7 +866,7 @@ Key* sort_keys(Key* k, Key* tmp, size_t n, unsigned threads) {
 }  // namespace
 
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes, TileVec* tiles,
-                 size_t* n_tma, size_t* n_big, std::vector<Rect>* rects, bcp_plan_stats_t* stats) {
+                 size_t* n_tma, size_t* n_big, size_t* n_cvt, std::vector<Rect>* rects, bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
   std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
     return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
@@ -797,9 +877,9 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     if (it.rows * it.row_bytes == 0) continue;
     if (!merged.empty()) {
       Item& p = merged.back();
-      if (p.rows == 1 && it.rows == 1 && p.zero == it.zero && p.dst_buf == it.dst_buf &&
+      if (p.rows == 1 && it.rows == 1 && p.zero == it.zero && p.cvt == it.cvt && p.dst_buf == it.dst_buf &&
           p.dst_off + p.row_bytes == it.dst_off &&
-          (it.zero || (p.src_buf == it.src_buf && p.src_off + p.row_bytes == it.src_off))) {
+          (it.zero || (p.src_buf == it.src_buf && p.src_off + p.src_row_bytes() == it.src_off))) {
         p.row_bytes += it.row_bytes;
         continue;
       }
@@ -815,17 +895,18 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   for (const Item& it : merged) rough += it.rows * it.row_bytes / opt.tile_bytes + (it.row_bytes >= opt.tile_bytes ? it.rows : 1);
   const unsigned threads = plan_threads(size_t(std::min<uint64_t>(rough, SIZE_MAX)));
   struct Count {
-    size_t n[3], rects;
+    size_t n[kClasses], rects;
   };
   std::vector<Count> cnt(n_items + 1);
   const size_t kBlock = 16;
   std::vector<Tally> tally((n_items + kBlock - 1) / kBlock);
   parallel_jobs(tally.size(), threads, [&](size_t j) {
-    Cutter c{opt, src_bytes, false, {nullptr, nullptr, nullptr}, nullptr, {0, 0, 0}, 0, Tally()};
+    Cutter c{opt, src_bytes, false, {nullptr, nullptr, nullptr, nullptr}, nullptr, {0, 0, 0, 0}, 0, Tally()};
     for (size_t i = j * kBlock; i < std::min(n_items, (j + 1) * kBlock); ++i) {
-      const Count before = {{c.pos[0], c.pos[1], c.pos[2]}, c.rect_pos};
+      const Count before = {{c.pos[0], c.pos[1], c.pos[2], c.pos[3]}, c.rect_pos};
       c.cut(merged[i]);
-      cnt[i] = {{c.pos[0] - before.n[0], c.pos[1] - before.n[1], c.pos[2] - before.n[2]}, c.rect_pos - before.rects};
+      cnt[i] = {{c.pos[0] - before.n[0], c.pos[1] - before.n[1], c.pos[2] - before.n[2], c.pos[3] - before.n[3]},
+                c.rect_pos - before.rects};
     }
     tally[j] = c.st;
   });
@@ -837,22 +918,23 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     for (size_t i = 0; i < n_items; ++i) cnt[i].n[kBig] += cnt[i].n[kTma], cnt[i].n[kTma] = 0, cnt[i].rects = 0;
     all.tma_bytes = all.tma_busy = all.tma_boxed = 0;
   }
-  Count run = {{0, 0, 0}, 0};  // counts -> positions of each item's first unit inside its class
+  Count run = {{0, 0, 0, 0}, 0};  // counts -> positions of each item's first unit inside its class
   for (size_t i = 0; i <= n_items; ++i) {
-    const Count c = i < n_items ? cnt[i] : Count{{0, 0, 0}, 0};
+    const Count c = i < n_items ? cnt[i] : Count{{0, 0, 0, 0}, 0};
     cnt[i] = run;
-    for (int k = 0; k < 3; ++k) run.n[k] += c.n[k];
+    for (int k = 0; k < kClasses; ++k) run.n[k] += c.n[k];
     run.rects += c.rects;
   }
-  const size_t total = run.n[0] + run.n[1] + run.n[2];
+  const size_t total = run.n[0] + run.n[1] + run.n[2] + run.n[3];
 
   // Pass 2: write the units, blocks of items of about equal size in parallel
   std::unique_ptr<bcp_tile[]> raw(new bcp_tile[total ? total : 1]);
-  bcp_tile* const cls[3] = {raw.get(), raw.get() + run.n[0], raw.get() + run.n[0] + run.n[1]};
+  bcp_tile* const cls[kClasses] = {raw.get(), raw.get() + run.n[0], raw.get() + run.n[0] + run.n[1],
+                                   raw.get() + run.n[0] + run.n[1] + run.n[2]};
   std::vector<Rect> rc(run.rects);
   std::vector<size_t> cuts(1, 0);  // item index where each block starts
   {
-    auto units_before = [&](size_t i) { return cnt[i].n[0] + cnt[i].n[1] + cnt[i].n[2]; };
+    auto units_before = [&](size_t i) { return cnt[i].n[0] + cnt[i].n[1] + cnt[i].n[2] + cnt[i].n[3]; };
     const size_t per_block = std::max<size_t>(4096, total / (size_t(threads) * 8) + 1);
     for (size_t i = 1; i < n_items; ++i)
       if (units_before(i) - units_before(cuts.back()) >= per_block) cuts.push_back(i);
@@ -860,7 +942,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   }
   parallel_jobs(cuts.size() - 1, threads, [&](size_t j) {
     const Count& at = cnt[cuts[j]];
-    Cutter c{opt, src_bytes, demote, {cls[0], cls[1], cls[2]}, rc.data(), {at.n[0], at.n[1], at.n[2]}, at.rects, Tally()};
+    Cutter c{opt, src_bytes, demote, {cls[0], cls[1], cls[2], cls[3]}, rc.data(), {at.n[0], at.n[1], at.n[2], at.n[3]}, at.rects, Tally()};
     for (size_t i = cuts[j]; i < cuts[j + 1]; ++i) c.cut(merged[i]);
   });
   stats->bytes_copied = all.bytes_copied;
@@ -884,7 +966,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   // Register kernel: a CTA per unit for small jobs (fewer, fatter workers start faster); every
   // warp its own worker once the kernel has a lot to move (no barriers, deeper overlap).
   if (!opt.worker) {
-    opt.worker = all.bytes_copied - all.tma_bytes >= (128u << 20) ? 2 : 1;
+    opt.worker = all.bytes_copied - all.tma_bytes - all.cvt_bytes >= (128u << 20) ? 2 : 1;
     if (opt.worker == 2 && !opt.ctas_per_sm) opt.ctas_per_sm = 4;
   }
   if (!opt.ctas_per_sm) opt.ctas_per_sm = 2;
@@ -897,7 +979,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   parallel_jobs((total + kChunk - 1) / kChunk, threads, [&](size_t j) {
     for (size_t i = j * kChunk; i < std::min(total, (j + 1) * kChunk); ++i) {
       const bcp_tile& t = raw[i];
-      const int k = i < run.n[0] ? 0 : i < run.n[0] + run.n[1] ? 1 : 2;
+      const int k = i < run.n[0] ? 0 : i < run.n[0] + run.n[1] ? 1 : i < run.n[0] + run.n[1] + run.n[2] ? 2 : 3;
       const uint32_t idx = uint32_t(i - (cls[k] - raw.get()));
       keys[i] = by_src ? Key{t.src_off, t.dst_off, t.src_buf, t.dst_buf, idx, 0} : Key{t.dst_off, 0, t.dst_buf, 0, idx, 0};
     }
@@ -905,7 +987,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   tiles->clear();
   tiles->resize(total);
   size_t base = 0;
-  for (int k = 0; k < 3; ++k) {
+  for (int k = 0; k < kClasses; ++k) {
     const size_t n = run.n[k];
     const Key* sorted = sort_keys(keys.get() + base, spare.get() + base, n, threads);
     bcp_tile* dst = tiles->data() + base;
@@ -920,6 +1002,8 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   stats->n_small_tiles = run.n[kSmall];
   *n_tma = run.n[kTma];
   *n_big = run.n[kBig];
+  *n_cvt = run.n[kCvt];
+  stats->n_cvt_tiles = run.n[kCvt];
   if (rects) *rects = std::move(rc);
 }
 

@@ -13,7 +13,7 @@ import torch
 import paper_2407_20143_b200 as bcp
 from oracle import reshard_oracle as orc
 from workloads import fills
-from workloads.configs import CONFIGS, STRESS, scenario_cases
+from workloads.configs import CONFIGS, STRESS, convert_cases, scenario_cases
 from workloads.meta import ShardMeta
 from workloads.random_cases import big_random_case, many_tiny_case, random_case
 
@@ -34,8 +34,9 @@ def guards_intact(backs, sizes, poison=POISON):
 
 def run_and_compare(case, device, fill="index", runs=1, stream=None, **opts):
     src = fills.fill_state(case.src, case.key_ids, fill, case.seed, device, poison=0x5A)
-    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
-    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON,
+                       convert=case.convert)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts, **case.plan_opts)
     for _ in range(runs):
         dst, backs = guarded(case.dst.buf_bytes, device)
         bcp.bcp_reshard(plan, src, dst, stream=stream)
@@ -536,3 +537,64 @@ def test_plans_run_from_several_threads_on_their_own_streams(cuda_device):
     for t in threads:
         t.join()
     assert not failures, failures[:3]
+
+
+# ---- element conversion (extension) --------------------------------------------------------------
+@pytest.mark.parametrize("fill", ["index", "uniform"])
+@pytest.mark.parametrize("case", convert_cases(), ids=lambda c: c.name)
+def test_converting_reshard(cuda_device, case, fill):
+    st = run_and_compare(case, cuda_device, fill, runs=2, tile_bytes=4096 if fill == "index" else 65536)
+    assert st["n_cvt_tiles"] > 0
+
+
+def test_converting_reshard_every_bit_pattern_and_alignment(cuda_device):
+    """All 2^32 binary32 patterns are too many; all 2^16 upper halves times the lower halves around
+    the halfway point are not (every exponent, every tie, NaNs, infinities), and rows that start
+    at every element phase exercise the leading / body / tail split of the kernel."""
+    hi = np.arange(1 << 16, dtype=np.uint64) << 16
+    lows = np.array([0x0000, 0x0001, 0x7FFF, 0x8000, 0x8001, 0xFFFF], dtype=np.uint64)
+    bits = (hi[:, None] | lows[None, :]).reshape(-1).astype(np.uint32)  # 393,216 values
+    n = bits.size
+    rows, cols = 96, n // 96
+    src_meta = [ShardMeta("x", 4, 2, (rows, cols), (0, 0), (rows, cols), 0, 0)]
+    # wanted: column blocks of odd widths, so that row starts fall on every phase of 16 bytes
+    cuts = [0, 1, 4, 9, 16, 23, 1000, 1003, cols]
+    dst_meta, pos = [], 0
+    for a, b in zip(cuts, cuts[1:]):
+        m = ShardMeta("x", 2, 1, (rows, cols), (0, a), (rows, b - a), 0, pos)
+        dst_meta.append(m)
+        pos += m.byte_length + (2 if (b - a) % 2 else 6)  # odd gaps: targets start at odd element offsets too
+    blob = torch.from_numpy(bits.view(np.uint8).copy()).to(cuda_device)
+    want = orc.reshard(src_meta, [bits.view(np.uint8)], dst_meta, [pos], fill_byte=POISON, convert=(1, 2, 1))[0]
+    plan = bcp.bcp_plan(src_meta, [n * 4], dst_meta, [pos], convert=1, convert_src_tag=2, convert_dst_tag=1, tile_bytes=8192)
+    dst, backs = guarded([pos], cuda_device)
+    bcp.bcp_reshard(plan, [blob], dst)
+    torch.cuda.synchronize()
+    bcp.bcp_plan_device_status(plan)
+    assert np.array_equal(dst[0].cpu().numpy(), want) and guards_intact(backs, [pos])
+    plan.destroy()
+    # and back: every bfloat16 pattern widened
+    h = np.arange(1 << 16, dtype=np.uint32).astype(np.uint16)
+    src_meta = [ShardMeta("h", 2, 1, (1 << 16,), (0,), (1 << 16,), 0, 0)]
+    dst_meta = [ShardMeta("h", 4, 2, (1 << 16,), (a,), (b - a,), 0, 4 * a + 4) for a, b in ((0, 3), (3, 40001), (40001, 1 << 16))]
+    total = 4 * (1 << 16) + 4
+    want = orc.reshard(src_meta, [h.view(np.uint8)], dst_meta, [total], fill_byte=POISON, convert=(2, 1, 2))[0]
+    plan = bcp.bcp_plan(src_meta, [h.nbytes], dst_meta, [total], convert=2, convert_src_tag=1, convert_dst_tag=2)
+    dst, backs = guarded([total], cuda_device)
+    bcp.bcp_reshard(plan, [torch.from_numpy(h.view(np.uint8).copy()).to(cuda_device)], dst)
+    torch.cuda.synchronize()
+    assert np.array_equal(dst[0].cpu().numpy(), want) and guards_intact(backs, [total])
+    plan.destroy()
+
+
+def test_converting_reshard_from_host_buffers(cuda_device):
+    case = convert_cases()[1]
+    src = [s.cpu() for s in fills.fill_state(case.src, case.key_ids, "uniform", case.seed, "cpu")]
+    want = orc.reshard(case.src.metas, [s.numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=0, convert=case.convert)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **case.plan_opts)
+    for pinned in (False, True):
+        a = [s.pin_memory() if pinned else s for s in src]
+        dst = [torch.full((n,), POISON, dtype=torch.uint8, pin_memory=pinned) for n in case.dst.buf_bytes]
+        bcp.bcp_reshard_host(plan, a, dst)
+        assert all(np.array_equal(d.numpy(), w) for d, w in zip(dst, want))
+    plan.destroy()

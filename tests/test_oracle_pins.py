@@ -221,3 +221,92 @@ def test_pack_is_join_with_zero_padding():
         assert offs == list(np.cumsum([0] + [-(-n // align) * align for n in sizes[:-1]]))
         back = orc.unpack(blob, table)
         assert all(np.array_equal(a, b) for a, b in zip(back, ts))
+
+
+# ---- element conversion (extension; the paper moves bytes only) ----------------------------------
+def _conversion_examples():
+    import os
+
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "f32_to_bf16_examples.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    return [(int(r[0], 16), int(r[1], 16)) for r in rows]
+
+
+def test_conversion_hand_worked_examples():
+    ex = _conversion_examples()
+    assert len(ex) >= 20
+    got = orc.f32_to_bf16(np.array([a for a, _ in ex], dtype=np.uint32))
+    assert [int(g) for g in got] == [b for _, b in ex]
+    # widening appends sixteen zero bits
+    assert [int(x) for x in orc.bf16_to_f32(np.array([0x3F80, 0xC049, 0x0001, 0x7FC0, 0xFFFF], dtype=np.uint16))] == [
+        0x3F800000, 0xC0490000, 0x00010000, 0x7FC00000, 0xFFFF0000]
+
+
+def _patterns():
+    rng = np.random.default_rng(11)
+    sweep = np.arange(0, 1 << 32, 16381, dtype=np.uint64).astype(np.uint32)  # every exponent, both signs
+    ties = (np.arange(0, 1 << 16, dtype=np.uint64) << 16 | 0x8000).astype(np.uint32)  # every halfway point
+    return np.concatenate([rng.integers(0, 1 << 32, 400_000, dtype=np.uint64).astype(np.uint32), sweep, ties, ties - 1, ties + 1])
+
+
+def test_conversion_agrees_with_the_library_cast():
+    """torch's own binary32 -> bfloat16 cast on everything but NaN (NaN encodings are not fixed by IEEE 754)."""
+    import torch
+
+    bits = _patterns()
+    bits = bits[(bits & 0x7FFFFFFF) <= 0x7F800000]
+    lib = torch.from_numpy(bits.view(np.float32).copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(orc.f32_to_bf16(bits), lib)
+    back = torch.from_numpy(lib.view(np.int16).copy()).view(torch.bfloat16).to(torch.float32).numpy().view(np.uint32)
+    assert np.array_equal(orc.bf16_to_f32(lib), back)
+
+
+def test_conversion_error_bound_fixed_points_and_order():
+    bits = _patterns()
+    finite = bits[(bits & 0x7FFFFFFF) < 0x7F800000]
+    out = orc.f32_to_bf16(finite)
+    x = finite.view(np.float32).astype(np.float64)
+    with np.errstate(over="ignore"):
+        y = orc.bf16_to_f32(out).view(np.float32).astype(np.float64)
+    # half a unit in the last place of the result: 2^-8 relative for normal numbers, 2^-134 absolute below
+    ok = np.isfinite(y)
+    assert np.all(np.abs(y[ok] - x[ok]) <= np.maximum(np.abs(x[ok]) * 2.0 ** -8, 2.0 ** -134))
+    assert np.all(np.abs(x[~ok]) >= (2.0 - 2.0 ** -8) * 2.0 ** 127)  # only values past the last halfway point overflow
+    assert np.all((y == 0) | (np.sign(y) == np.sign(x)))
+    # every bfloat16 is a fixed point (all 65,536 patterns but the NaNs)
+    h = np.arange(1 << 16, dtype=np.uint32).astype(np.uint16)
+    h = h[(h & 0x7FFF) <= 0x7F80]
+    assert np.array_equal(orc.f32_to_bf16(orc.bf16_to_f32(h)), h)
+    # rounding never reverses the order of two values
+    pos = np.sort(finite[finite < 0x7F800000])
+    assert np.all(np.diff(orc.f32_to_bf16(pos).astype(np.int64)) >= 0)
+    # NaNs: one canonical pattern
+    assert set(orc.f32_to_bf16(np.array([0x7F800001, 0x7FFFFFFF, 0xFFC00000, 0xFF800001], dtype=np.uint32)).tolist()) == {0x7FC0}
+
+
+def test_conversion_commutes_with_resharding():
+    """Converting reshard == plain reshard of the saved type into the wanted layout, then the library cast,
+    element by element (no NaN in this fill)."""
+    import torch
+    from workloads.configs import convert_cases
+    from workloads.meta import DTYPE_BF16, DTYPE_F32
+
+    for case in convert_cases():
+        blobs = filled(case, case.src, "uniform")
+        got = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, convert=case.convert)
+        narrow = case.convert[0] == orc.F32_TO_BF16
+        # the same wanted boxes in the saved type, packed back to back
+        same, pos = [], 0
+        for m in case.dst.metas:
+            k = ShardMeta(m.fqn, 4 if narrow else 2, DTYPE_F32 if narrow else DTYPE_BF16, m.global_shape, m.offsets, m.lengths,
+                          0, pos, m.kind, m.flat_begin, m.flat_end)
+            same.append(k)
+            pos += k.byte_length
+        plain = orc.reshard(case.src.metas, blobs, same, [pos])[0]
+        for m, k in zip(case.dst.metas, same):
+            raw = plain[k.byte_offset:k.byte_offset + k.byte_length]
+            if narrow:
+                want = torch.from_numpy(raw.view(np.float32).copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint8)
+            else:
+                want = torch.from_numpy(raw.view(np.int16).copy()).view(torch.bfloat16).to(torch.float32).numpy().view(np.uint8)
+            assert np.array_equal(got[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length], want), (case.name, m.fqn)

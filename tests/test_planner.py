@@ -12,7 +12,7 @@ import paper_2407_20143_b200 as bcp
 from paper_2407_20143_b200 import _lib, api
 from oracle import reshard_oracle as orc
 from workloads import fills
-from workloads.configs import CONFIGS, EXPECTED_TOTALS, scenario_cases
+from workloads.configs import CONFIGS, EXPECTED_TOTALS, convert_cases, scenario_cases
 from workloads.meta import BOX, FLAT_SLICE, ShardMeta
 from workloads.random_cases import big_random_case, random_case
 
@@ -37,7 +37,8 @@ def test_struct_sizes_match_header():
 
     assert C.sizeof(_lib.TileC) == 64
     assert C.sizeof(_lib.ShardMetaC) == 8 + 16 + 3 * 64 + 16 + 8 + 16
-    assert C.sizeof(_lib.PlanOptsC) == 68
+    assert C.sizeof(_lib.PlanOptsC) == 80
+    assert C.sizeof(_lib.PlanStatsC) == 14 * 8
 
 
 # ---- decomposition (Sec. 3.2) ----------------------------------------------------------------------
@@ -86,6 +87,24 @@ def run_tiles(tiles, src, dst_sizes, poison=0xA5):
     for t in tiles:
         g = 1 << (t.flags & api.TILE_GRAN_MASK)
         assert t.dst_off % g == 0 and t.row_bytes % g == 0 and t.dst_pitch % g == 0
+        kind = (t.flags & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
+        if kind:  # converting unit: row_bytes counts target bytes, the source row holds the same elements
+            assert not t.flags & (api.TILE_ZERO | api.TILE_SMALL | api.TILE_TMA | api.TILE_TMA2D | api.TILE_FOLLOW)
+            s_isz, d_isz = (4, 2) if kind == api.CONVERT_F32_TO_BF16 else (2, 4)
+            assert t.row_bytes % d_isz == 0 and t.dst_off % d_isz == 0 and t.src_off % s_isz == 0
+            n = t.row_bytes // d_isz
+            for r in range(t.rows):
+                d0, s0 = t.dst_off + r * t.dst_pitch, t.src_off + r * t.src_pitch
+                chunk = src[t.src_buf][s0:s0 + n * s_isz]
+                assert chunk.size == n * s_isz
+                if kind == api.CONVERT_F32_TO_BF16:  # the usual integer form of round-to-nearest-even
+                    x = chunk.view(np.uint32).astype(np.uint64)
+                    y = np.where((x & 0x7FFFFFFF) > 0x7F800000, 0x7FC0, (x + 0x7FFF + ((x >> 16) & 1)) >> 16).astype(np.uint16)
+                else:
+                    y = chunk.view(np.uint16).astype(np.uint32) << 16
+                out[t.dst_buf][d0:d0 + t.row_bytes] = y.view(np.uint8)
+                count[t.dst_buf][d0:d0 + t.row_bytes] += 1
+            continue
         for r in range(t.rows):
             d0 = t.dst_off + r * t.dst_pitch
             if t.flags & api.TILE_ZERO:
@@ -102,11 +121,11 @@ def run_tiles(tiles, src, dst_sizes, poison=0xA5):
 
 def check_case(case, fill="index", **opts):
     blobs = np_bufs(fills.fill_state(case.src, case.key_ids, fill, case.seed, "cpu", poison=0x5A))
-    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts, **case.plan_opts)
     tiles = plan.tiles()
     st = plan.stats()
     got, count = run_tiles(tiles, blobs, case.dst.buf_bytes)
-    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5)
+    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, convert=case.convert)
     for g, w in zip(got, want):
         assert np.array_equal(g, w)
     # every named target byte is written exactly once, every other byte never
@@ -118,9 +137,9 @@ def check_case(case, fill="index", **opts):
     assert st["bytes_copied"] == case.dst.total_bytes
     tb = opts.get("tile_bytes", 65536)
     assert all(t.rows * t.row_bytes <= tb for t in tiles)
-    assert st["n_tiles"] + st["n_small_tiles"] == len(tiles)
-    small = [bool(t.flags & api.TILE_SMALL) for t in tiles]
-    assert small == sorted(small), "CTA-wide units come first"
+    assert st["n_tiles"] + st["n_small_tiles"] + st["n_cvt_tiles"] == len(tiles)
+    rank = [2 if t.flags & api.TILE_CVT_MASK else 1 if t.flags & api.TILE_SMALL else 0 for t in tiles]
+    assert rank == sorted(rank), "CTA-wide units come first, converting units last"
     plan.destroy()
     return st
 
@@ -412,6 +431,51 @@ def test_pack_layout_matches_closed_form():
         assert bcp.bcp_pack_layout(sizes, align) == orc.pack_layout(sizes, align)
     with pytest.raises(bcp.BcpError):
         bcp.bcp_pack_layout(sizes, 24)
+
+
+# ---- element conversion (an extension: the paper moves bytes only) -------------------------------
+@pytest.mark.parametrize("case", convert_cases(), ids=lambda c: c.name)
+@pytest.mark.parametrize("opts", [dict(), dict(tile_bytes=4096, order=2)], ids=str)
+def test_converting_plans_match_oracle(case, opts):
+    st = check_case(case, **opts)
+    assert st["n_cvt_tiles"] > 0 and st["n_tma_tiles"] == 0
+    # source bytes are counted in the saved type, target bytes in the wanted one
+    assert st["bytes_copied"] == case.dst.total_bytes and st["bytes_src_unique"] == case.src.total_bytes
+
+
+def test_conversion_is_per_tensor_and_needs_both_tags():
+    f32, bf16 = 2, 1
+    src = [_m("a", 4, f32, boff=0), _m("b", 2, bf16, boff=64)]
+    dst = [_m("a", 2, bf16, boff=0), _m("b", 2, bf16, boff=32)]
+    # without the option a tensor that changes its type is a mismatch, as before
+    assert _plan_err(src, [96], dst, [64]) == api.ERR_MISMATCH
+    plan = bcp.bcp_plan(src, [96], dst, [64], convert=api.CONVERT_F32_TO_BF16, convert_src_tag=f32, convert_dst_tag=bf16)
+    tiles = plan.tiles()
+    assert sorted((t.flags & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT for t in tiles) == [0, 1]  # "b" is copied, "a" converted
+    plan.destroy()
+    # the wrong direction, the wrong tags, or the wrong sizes are still mismatches
+    assert _plan_err(src, [96], dst, [64], convert=api.CONVERT_BF16_TO_F32, convert_src_tag=f32, convert_dst_tag=bf16) == api.ERR_MISMATCH
+    assert _plan_err(src, [96], dst, [64], convert=api.CONVERT_F32_TO_BF16, convert_src_tag=bf16, convert_dst_tag=f32) == api.ERR_MISMATCH
+    assert _plan_err([_m("a", 8, f32)], [128], [_m("a", 2, bf16)], [32], convert=1, convert_src_tag=f32, convert_dst_tag=bf16) == api.ERR_MISMATCH
+    # wanted entries of one tensor must agree among themselves
+    two = [_m("a", 2, bf16, off=(0, 0), ln=(2, 4), boff=0), _m("a", 4, f32, off=(2, 0), ln=(2, 4), boff=32)]
+    assert _plan_err(src[:1], [64], two, [64], convert=1, convert_src_tag=f32, convert_dst_tag=bf16) == api.ERR_MISMATCH
+    # option checks
+    assert _plan_err(src, [96], dst, [64], convert=3, convert_src_tag=f32, convert_dst_tag=bf16) == api.ERR_INVALID
+    assert _plan_err(src, [96], dst, [64], convert=1, convert_src_tag=f32, convert_dst_tag=f32) == api.ERR_INVALID
+    assert _plan_err(src, [96], dst, [64], convert_src_tag=f32) == api.ERR_INVALID
+
+
+def test_converting_plan_image_round_trip():
+    case = convert_cases()[2]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, tile_bytes=4096, **case.plan_opts)
+    image = plan.serialize()
+    again = bcp.Plan.deserialize(image)
+    assert again.serialize() == image and again.stats()["n_cvt_tiles"] == plan.stats()["n_cvt_tiles"] > 0
+    blobs = np_bufs(fills.fill_state(case.src, case.key_ids, "index", case.seed, "cpu"))
+    got, _ = run_tiles(again.tiles(), blobs, case.dst.buf_bytes)
+    want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, convert=case.convert)
+    assert all(np.array_equal(g, w) for g, w in zip(got, want))
 
 
 # ---- host threads --------------------------------------------------------------------------------

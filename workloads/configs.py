@@ -9,7 +9,7 @@ from __future__ import annotations
 
 from typing import Callable, Dict, List
 
-from .layouts import (ModelSpec, Parallelism, ReshardCase, StateKinds, gpt_model, llama_model,
+from .layouts import (ModelSpec, Parallelism, ReshardCase, StateKinds, build_state, gpt_model, llama_model,
                       moe_model, reshard_case)
 from .meta import DTYPE_BF16, DTYPE_F32
 
@@ -17,6 +17,7 @@ MIXED = StateKinds()  # bf16 params + fp32 master / exp_avg / exp_avg_sq
 PARAMS_ONLY = StateKinds(optim=())
 OPTIM_ONLY = StateKinds(param_dtype=None)
 MOE_KINDS = StateKinds(optim=("exp_avg",))
+F32_PARAMS = StateKinds(param_dtype=(4, DTYPE_F32), optim=())  # parameters kept in binary32 (master copy)
 
 
 def cfg1(fill: str = "uniform") -> ReshardCase:
@@ -85,7 +86,8 @@ def odd_gpt(layers: int = 12) -> ReshardCase:
                         seed=20151)
 
 
-STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows, "oddgpt": odd_gpt}
+STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows, "oddgpt": odd_gpt,
+                                                   "evalmerge": lambda layers=32: eval_merge(layers)}
 
 CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
     "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
@@ -160,3 +162,42 @@ def stacked_experts_case() -> ReshardCase:
                                   min(n, (r + 1) * cut)) for r in range(6)],
                        [(min(n, (r + 1) * cut) - r * cut) * isz for r in range(6)])
     return ReshardCase("stacked-experts-3d", src, dst, "index", 3)
+
+
+# --------------------------------------------------------------------------- element conversion
+def convert_case(name: str, model: ModelSpec, src_par: Parallelism, dst_par: Parallelism, narrow: bool = True,
+                 fill: str = "index", seed: int = 0, flat: bool = False) -> ReshardCase:
+    """Parameters saved in binary32 and wanted in bfloat16 under another parallelism (narrow),
+    or the reverse.  Not one of the paper's workloads: the paper moves bytes only."""
+    if flat:  # one optimizer state per parameter, flat-partitioned (ZeRO / FSDP), in either type
+        wide, slim = (StateKinds(param_dtype=None, optim=("master",), optim_dtype=d) for d in ((4, DTYPE_F32), (2, DTYPE_BF16)))
+    else:
+        wide, slim = F32_PARAMS, PARAMS_ONLY
+    a, b = (wide, slim) if narrow else (slim, wide)
+    tags = (1, DTYPE_F32, DTYPE_BF16) if narrow else (2, DTYPE_BF16, DTYPE_F32)
+    return ReshardCase(name, build_state(model, src_par, a, dedup=True), build_state(model, dst_par, b, dedup=False),
+                       fill, seed, convert=tags)
+
+
+def convert_cases() -> List[ReshardCase]:
+    g, l = small_gpt(), small_llama()
+    odd = gpt_model("gpt-odd", L=2, H=60, F=150, V=251, P=17)  # odd sizes: rows start at every alignment
+    f = llama_model("llama-f", 3, 96, 6, 2, 200, 777, fused=False, tied=True, fsdp_units=True)
+    return [
+        convert_case("narrow-gpt-tp1-to-tp2", g, Parallelism(tp=1, dp=2), Parallelism(tp=2, dp=2)),
+        convert_case("narrow-llama-tp8-to-tp2", l, Parallelism(tp=8), Parallelism(tp=2)),
+        convert_case("narrow-odd-tp3-to-tp2", odd, Parallelism(tp=3), Parallelism(tp=2)),
+        convert_case("widen-llama-tp2-to-tp8", l, Parallelism(tp=2), Parallelism(tp=8), narrow=False),
+        convert_case("widen-odd-tp2-to-tp3", odd, Parallelism(tp=2), Parallelism(tp=3), narrow=False),
+        convert_case("narrow-fsdp-5-to-3", f, Parallelism(dp=5, zero="fsdp"), Parallelism(dp=3, zero="fsdp"), flat=True),
+        convert_case("widen-zero1-dp3-to-dp4", g, Parallelism(tp=2, dp=3, zero="zero1"), Parallelism(tp=1, dp=4, zero="zero1"),
+                     narrow=False, flat=True),
+    ]
+
+
+def eval_merge(layers: int = 32) -> ReshardCase:
+    """Unscored: the Llama-3-8B shapes of cfg3 with binary32 parameters saved under TP8 and wanted in
+    bfloat16 under TP2 (32 GB read, 16 GB written)."""
+    m = llama_model("llama3-8b", L=layers, H=4096, nq=32, nkv=8, F=14336, V=128256, fused=True, tied=False)
+    return convert_case("eval-merge-llama3-8b-f32-to-bf16" + ("" if layers == 32 else f"-L{layers}"), m,
+                        Parallelism(tp=8), Parallelism(tp=2), True, "normal", 20150)

@@ -347,6 +347,16 @@ class ReshardCase:
     fill: str = "index"  # "index" | "uniform" | "normal"
     seed: int = 0
     note: str = ""
+    # (kind, saved dtype tag, wanted dtype tag) when tensors change their element type on the
+    # way (kind 1: binary32 -> bfloat16, kind 2: the reverse); None: bytes are moved unchanged
+    convert: Optional[Tuple[int, int, int]] = None
+
+    @property
+    def plan_opts(self) -> Dict[str, int]:
+        """Planner options this case needs (none unless it converts)."""
+        if self.convert is None:
+            return {}
+        return dict(convert=self.convert[0], convert_src_tag=self.convert[1], convert_dst_tag=self.convert[2])
 
     @property
     def key_ids(self) -> Dict[str, int]:
