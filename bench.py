@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="bcp", choices=["bcp", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg4odd", "narrow", "oddgpt"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg4odd", "narrow", "oddgpt", "evalmerge"])
     ap.add_argument("--layers", type=int, default=0, help="shrink the depth (profiler captures); 0 = full size")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
@@ -192,7 +192,7 @@ def time_oracle(case, fetch_payload, target_bytes: float, steps: int = 1, warmup
     for i in range(warmup + steps):
         t0 = time.perf_counter()
         for ss, ps, ds in inputs:
-            orc.reshard_fqn(ss, ps, ds)
+            orc.reshard_fqn(ss, ps, ds, convert=case.convert)
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     return sum(times) / len(times), src_b, dst_b, len(picked)
@@ -201,8 +201,8 @@ def time_oracle(case, fetch_payload, target_bytes: float, steps: int = 1, warmup
 def _oracle_job(i):
     from oracle import reshard_oracle as orc
 
-    ss, ps, ds = _ORACLE_INPUTS[i]
-    orc.reshard_fqn(ss, ps, ds)
+    ss, ps, ds, convert = _ORACLE_INPUTS[i]
+    orc.reshard_fqn(ss, ps, ds, convert=convert)
     return i
 
 
@@ -216,9 +216,9 @@ def time_oracle_all_cores(case, fetch_payload, target_bytes: float, passes: int 
 
     global _ORACLE_INPUTS
     picked, by_src, by_dst = oracle_sample(case, target_bytes)
-    _ORACLE_INPUTS = [(by_src[n], [fetch_payload(s) for s in by_src[n]], by_dst[n]) for n in picked]
-    src_b = sum(s.byte_length for ss, _, _ in _ORACLE_INPUTS for s in ss)
-    dst_b = sum(d.byte_length for _, _, ds in _ORACLE_INPUTS for d in ds)
+    _ORACLE_INPUTS = [(by_src[n], [fetch_payload(s) for s in by_src[n]], by_dst[n], case.convert) for n in picked]
+    src_b = sum(s.byte_length for ss, _, _, _ in _ORACLE_INPUTS for s in ss)
+    dst_b = sum(d.byte_length for _, _, ds, _ in _ORACLE_INPUTS for d in ds)
     cores = os.cpu_count() or 1
     ctx = mp.get_context("fork")
     with ctx.Pool(cores) as pool:
@@ -282,11 +282,13 @@ def main():
     keys = case.key_ids
     opts = plan_opts(a)
     t0 = time.perf_counter()
-    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts, **case.plan_opts)
     plan_ms = (time.perf_counter() - t0) * 1e3
     st = plan.stats()
     b_min = st["bytes_src_unique"] + st["bytes_copied"]
-    b_moved = 2 * st["bytes_copied"]
+    # what the unit list loads + stores (replica reads counted every time); a converting plan reads
+    # the saved type and writes the wanted one, and none of its sources is read twice
+    b_moved = b_min if case.convert else 2 * st["bytes_copied"]
     free, _ = torch.cuda.mem_get_info()
     need = sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)
     assert free > need + (2 << 30), f"{case.name} needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free"
@@ -338,19 +340,21 @@ def main():
     # register kernel (if any unit is left for it)
     n_tma = st["n_tma_tiles"]
     n_reg = st["n_tiles"] - n_tma + st["n_small_tiles"]
-    kernels_per_step = int(n_tma > 0) + int(n_reg > 0)
-    dominant = "bcp_tma_kernel" if n_tma > 0 else "bcp_copy_kernel"
+    n_cvt = st["n_cvt_tiles"]
+    kernels_per_step = int(n_tma > 0) + int(n_reg > 0) + int(n_cvt > 0)
+    dominant = "bcp_convert_kernel" if case.convert else "bcp_tma_kernel" if n_tma > 0 else "bcp_copy_kernel"
     peak, peak_kind = measured_peak()
     avg_launch_ms = sum(launch_ms) / len(launch_ms)
     achieved = b_min / (avg_launch_ms * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": a.steps, "warmup": max(a.warmup, 3),
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32->bf16" if case.convert else "u8",
         "data": "synthetic",
         "config": {"workload": case.name, "src_bytes": st["bytes_src_unique"], "dst_bytes": st["bytes_copied"],
                    "bytes_per_step": b_min, "bytes_counted": "unique source bytes read + target bytes written",
                    "src_ranks": len(case.src.buf_bytes), "dst_ranks": len(case.dst.buf_bytes),
-                   "work_units": st["n_tiles"] + st["n_small_tiles"],
+                   "work_units": st["n_tiles"] + st["n_small_tiles"] + st["n_cvt_tiles"],
                    "l2": "inputs_exceed_l2" if flush is None else "flushed_before_every_step_512MiB", "fill": case.fill,
                    "multi_gpu": "replicas only", "plan_opts": opts, "plan_ms": plan_ms},
         "gbps_b_moved": b_moved * ws / (ms_step * 1e-3) / 1e9,
@@ -539,7 +543,7 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     same = all(bool(torch.equal(h[: 1 << 20], d[: 1 << 20].cpu())) for h, d in zip(hdst, dst))
     # pinned buffers are addressed by the kernels directly: every unit's source bytes cross PCIe when
     # it is copied (replica reads cross again), every target byte crosses once on its way out
-    moved_in = plan.stats()["bytes_copied"]
+    moved_in = plan.stats()["bytes_src_unique" if case.convert else "bytes_copied"]
     return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": moved_in, "d2h_bytes_per_step": d2h,
             "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same,
             "mode": "pinned host buffers read and written in place by the kernels (no staging copy)",

@@ -383,15 +383,18 @@ def _free_gb():
 
 
 @pytest.mark.parametrize("name,max_fqn_bytes", [("cfg2", 450e6), ("cfg3", 1.2e9), ("cfg4", 0.5e9), ("cfg5", 300e6),
-                                                ("cfg4odd", 0.5e9), ("narrow", 0.6e9), ("oddgpt", 0.6e9)])
+                                                ("cfg4odd", 0.5e9), ("narrow", 0.6e9), ("oddgpt", 0.6e9), ("evalmerge", 1.2e9)])
 def test_full_size_config(cuda_device, name, max_fqn_bytes):
     case = (CONFIGS.get(name) or STRESS[name])()
     need = (sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)) / 1e9 + 8
     assert _free_gb() > need, f"{name} needs {need:.0f} GB of device memory"
     keys = case.key_ids
-    src = fills.fill_state(case.src, keys, "index", case.seed, cuda_device, poison=0x5A)
+    # closed form of the expected target bytes: the index pattern for plain copies; for a narrowing
+    # conversion the value fills, whose bfloat16 form is the rounded binary32 form of the same pool
+    fill = "normal" if case.convert else "index"
+    src = fills.fill_state(case.src, keys, fill, case.seed, cuda_device, poison=0x5A)
     dst = fills.make_buffers(case.dst, cuda_device, POISON)
-    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)  # bench defaults
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **case.plan_opts)  # bench defaults
     bcp.bcp_reshard(plan, src, dst)
     torch.cuda.synchronize()
     bcp.bcp_plan_device_status(plan)
@@ -402,7 +405,7 @@ def test_full_size_config(cuda_device, name, max_fqn_bytes):
         n = m.numel
         for lo in range(0, n, 1 << 26):
             hi = min(n, lo + (1 << 26))
-            want = fills.entry_bytes(m, keys[m.fqn], "index", case.seed, cuda_device, lo, hi)
+            want = fills.entry_bytes(m, keys[m.fqn], fill, case.seed, cuda_device, lo, hi)
             b = m.byte_offset + lo * m.itemsize
             got = dst[m.buf_index][b:b + (hi - lo) * m.itemsize]
             if not torch.equal(got, want):
@@ -426,7 +429,7 @@ def test_full_size_config(cuda_device, name, max_fqn_bytes):
         if sum(s.byte_length for s in ss) > max_fqn_bytes:
             continue
         payloads = [src[s.buf_index][s.byte_offset:s.byte_offset + s.byte_length].cpu().numpy().view(orc._UINT[s.itemsize]) for s in ss]
-        for d, w in zip(ds, orc.reshard_fqn(ss, payloads, ds)):
+        for d, w in zip(ds, orc.reshard_fqn(ss, payloads, ds, convert=case.convert)):
             got = dst[d.buf_index][d.byte_offset:d.byte_offset + d.byte_length].cpu().numpy()
             assert np.array_equal(got, w), f"{name} {fqn}: oracle mismatch on target rank {d.buf_index}"
             checked += d.byte_length
