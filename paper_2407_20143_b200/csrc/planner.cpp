@@ -500,6 +500,14 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
                       f.src[j].meta);
       }
     }
+    if (f.cvt) {  // a converting unit reads and writes whole elements at their natural alignment
+      for (const Entry& e : f.src)
+        if (e.byte_off % f.itemsize)
+          return fail(BCP_ERR_INVALID, "%s: src[%u] is converted, so its byte_offset must be a multiple of %u", f.fqn, e.meta, f.itemsize);
+      for (const Entry& e : f.dst)
+        if (e.byte_off % f.d_itemsize)
+          return fail(BCP_ERR_INVALID, "%s: dst[%u] is converted, so its byte_offset must be a multiple of %u", f.fqn, e.meta, f.d_itemsize);
+    }
     reach.resize(f.src.size());
     for (size_t i = 0; i < f.src.size(); ++i)
       reach[i] = std::max(i ? reach[i - 1] : INT64_MIN, f.src[i].off[0] + f.src[i].len[0]);

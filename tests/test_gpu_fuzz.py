@@ -9,7 +9,7 @@ import paper_2407_20143_b200 as bcp
 from oracle import reshard_oracle as orc
 from workloads import fills
 from workloads.configs import scenario_cases
-from workloads.random_cases import big_random_case, random_case
+from workloads.random_cases import big_random_case, random_case, random_convert_case
 
 pytestmark = pytest.mark.gpu
 
@@ -42,6 +42,36 @@ def test_random_problems_and_options(cuda_device, stream_seed):
         src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device, poison=0x5A)
         want = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src], case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5)
         plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+        backs = [torch.full((m + 8192,), 0xA5, dtype=torch.uint8, device=cuda_device) for m in case.dst.buf_bytes]
+        dst = [b[4096:4096 + m] for b, m in zip(backs, case.dst.buf_bytes)]
+        for _ in range(2):
+            bcp.bcp_reshard(plan, src, dst)
+        torch.cuda.synchronize()
+        bcp.bcp_plan_device_status(plan)
+        for d, w in zip(dst, want):
+            assert np.array_equal(d.cpu().numpy(), w), (case.name, opts)
+        for b, m in zip(backs, case.dst.buf_bytes):
+            assert bool((b[:4096] == 0xA5).all()) and bool((b[4096 + m:] == 0xA5).all()), (case.name, opts)
+        plan.destroy()
+
+
+@pytest.mark.parametrize("stream_seed", [11, 12])
+def test_random_converting_problems_and_options(cuda_device, stream_seed):
+    """The same for plans that convert some tensors (binary32 <-> bfloat16) and copy the others;
+    sources are random bytes, so every bit pattern (NaN, infinities, subnormals) takes part."""
+    rng = np.random.default_rng(stream_seed)
+    for it in range(30):
+        seed = int(rng.integers(0, 1 << 30))
+        case = random_convert_case(seed, narrow=bool(it % 2), big=it % 3 == 0, dst_replicas=int(rng.integers(1, 3)))
+        opts = dict(path_mask=int(rng.choice([1, 3, 7])), tile_bytes=int(rng.choice([4096, 8192, 65536])), order=int(rng.choice([1, 2])),
+                    tma_min_row_bytes=int(rng.choice([16, 512])), worker=int(rng.choice([1, 2])), small_bytes=int(rng.choice([64, 4096])))
+        g = torch.Generator(device="cpu").manual_seed(seed)
+        host = [torch.randint(0, 256, (n,), dtype=torch.uint8, generator=g) for n in case.src.buf_bytes]
+        want = orc.reshard(case.src.metas, [h.numpy() for h in host], case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5,
+                           convert=case.convert)
+        plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts, **case.plan_opts)
+        assert plan.stats()["n_cvt_tiles"] > 0
+        src = [h.to(cuda_device) for h in host]
         backs = [torch.full((m + 8192,), 0xA5, dtype=torch.uint8, device=cuda_device) for m in case.dst.buf_bytes]
         dst = [b[4096:4096 + m] for b, m in zip(backs, case.dst.buf_bytes)]
         for _ in range(2):

@@ -14,7 +14,7 @@ from oracle import reshard_oracle as orc
 from workloads import fills
 from workloads.configs import CONFIGS, EXPECTED_TOTALS, convert_cases, scenario_cases
 from workloads.meta import BOX, FLAT_SLICE, ShardMeta
-from workloads.random_cases import big_random_case, random_case
+from workloads.random_cases import big_random_case, random_case, random_convert_case
 
 from helpers import np_bufs, read_irregular_example
 
@@ -368,6 +368,55 @@ def test_plan_image_is_verified():
     assert "checksum" in str(e.value)
 
 
+def _reseal(image: bytearray) -> bytes:
+    """Recompute the trailing FNV-1a checksum after editing an image (what a careless or hostile
+    writer of plan files could do)."""
+    h = 1469598103934665603
+    for b in image[:-8]:
+        h = ((h ^ b) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
+    return bytes(image[:-8]) + h.to_bytes(8, "little")
+
+
+def test_plan_image_units_are_checked_against_the_buffers():
+    """A unit drives device copies, so a well-formed image with a wrong unit must be refused:
+    plain and converting units are edited in place and the image is resealed."""
+    import ctypes as C
+    import struct
+
+    case = convert_cases()[2]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, tile_bytes=4096, **case.plan_opts)
+    tiles = plan.tiles()
+    image = bytearray(plan.serialize())
+    first = image.find(bytes(tiles[0]))  # the first unit record inside the image
+    assert first > 0 and bcp.Plan.deserialize(_reseal(bytearray(image))).stats() == plan.stats()
+    cvt = next(i for i, t in enumerate(tiles) if t.flags & api.TILE_CVT_MASK)
+    F = {n: getattr(_lib.TileC, n).offset for n, _ in _lib.TileC._fields_}
+
+    def edited(i, field, fn):
+        out = bytearray(image)
+        at = first + i * C.sizeof(_lib.TileC) + F[field]
+        width = 8 if field.endswith("off") or field.endswith("pitch") else 4
+        v = int.from_bytes(out[at:at + width], "little")
+        out[at:at + width] = fn(v).to_bytes(width, "little")
+        return _reseal(out)
+
+    bad = [
+        edited(cvt, "row_bytes", lambda v: v + (1 << 24)),        # runs past both buffers
+        edited(cvt, "src_off", lambda v: v + 2),                   # binary32 source not 4-byte aligned
+        edited(cvt, "dst_off", lambda v: v + 1),                   # bfloat16 target not 2-byte aligned
+        edited(cvt, "flags", lambda v: v | api.TILE_SMALL),        # a converting unit has no other class
+        edited(cvt, "flags", lambda v: v | api.TILE_CVT_MASK),     # unknown conversion kind
+        edited(cvt, "flags", lambda v: v & ~api.TILE_CVT_MASK),    # plain unit in the converting class
+        edited(cvt, "src_buf", lambda v: v + 1000),
+        edited(0, "dst_off", lambda v: v + (1 << 40)),
+    ]
+    for im in bad:
+        with pytest.raises(bcp.BcpError) as e:
+            bcp.Plan.deserialize(im)
+        assert "work unit" in str(e.value) or "inconsistent" in str(e.value)
+    plan.destroy()
+
+
 # ---- full-size configurations: planning is host-only, so their work lists are checked here ---------
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
 def test_full_config_plans(name):
@@ -441,6 +490,27 @@ def test_converting_plans_match_oracle(case, opts):
     assert st["n_cvt_tiles"] > 0 and st["n_tma_tiles"] == 0
     # source bytes are counted in the saved type, target bytes in the wanted one
     assert st["bytes_copied"] == case.dst.total_bytes and st["bytes_src_unique"] == case.src.total_bytes
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_converting_cases(seed):
+    """Converted and unchanged tensors in one plan, flat slices, odd offsets, replicas on the wanted side."""
+    check_case(random_convert_case(seed, narrow=seed % 2 == 0, dst_replicas=1 + seed % 3 // 2), tile_bytes=4096)
+
+
+@pytest.mark.parametrize("seed,narrow", [(1, True), (2, False)])
+def test_big_random_converting_cases(seed, narrow):
+    st = check_case(random_convert_case(seed, narrow=narrow, big=True, dst_replicas=2), tile_bytes=8192)
+    assert st["n_cvt_tiles"] > 100 and st["n_tiles"] + st["n_small_tiles"] > 0
+
+
+def test_converting_entries_must_be_element_aligned():
+    """A plain copy may start at any byte; a conversion reads and writes whole elements."""
+    f32, bf16 = 2, 1
+    opts = dict(convert=api.CONVERT_F32_TO_BF16, convert_src_tag=f32, convert_dst_tag=bf16)
+    assert _plan_err([_m("a", 4, f32, boff=2)], [96], [_m("a", 2, bf16)], [64], **opts) == api.ERR_INVALID
+    assert _plan_err([_m("a", 4, f32)], [96], [_m("a", 2, bf16, boff=1)], [64], **opts) == api.ERR_INVALID
+    bcp.bcp_plan([_m("a", 4, f32, boff=4)], [96], [_m("a", 2, bf16, boff=6)], [64], **opts).destroy()
 
 
 def test_conversion_is_per_tensor_and_needs_both_tags():

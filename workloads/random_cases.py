@@ -24,9 +24,11 @@ def _cuts(rng: np.random.Generator, n: int, max_parts: int) -> List[int]:
 
 def random_side(rng: np.random.Generator, tensors: Sequence[Tuple[str, Tuple[int, ...], int]], n_bufs: int,
                 *, max_parts: int = 3, flat_prob: float = 0.5, replicas: int = 1, gap_mod: int = 0,
-                shuffle: bool = True) -> ShardedState:
+                shuffle: bool = True, element_aligned: bool = False) -> ShardedState:
     """tensors: (fqn, global shape, itemsize).  gap_mod > 0 inserts random gaps of
-    0..gap_mod-1 elements between entries so that offsets are not 16-byte aligned."""
+    0..gap_mod-1 elements between entries so that offsets are not 16-byte aligned.
+    element_aligned: every entry starts on a multiple of its item size (entries of different
+    item sizes share buffers, so this does not follow from the gaps)."""
     entries: List[ShardMeta] = []
     for rep in range(replicas):
         for fqn, shape, isz in tensors:
@@ -48,7 +50,10 @@ def random_side(rng: np.random.Generator, tensors: Sequence[Tuple[str, Tuple[int
         e = entries[int(i)]
         b = int(rng.integers(0, n_bufs))
         gap = int(rng.integers(0, gap_mod)) * e.itemsize if gap_mod else 0
-        e.buf_index, e.byte_offset = b, fill[b] + gap
+        start = fill[b] + gap
+        if element_aligned:
+            start = -(-start // e.itemsize) * e.itemsize
+        e.buf_index, e.byte_offset = b, start
         fill[b] = e.byte_offset + e.byte_length
     return ShardedState(entries, [f + int(rng.integers(0, 64)) for f in fill])
 
@@ -100,3 +105,29 @@ def many_tiny_case(n_tensors: int = 100_000, seed: int = 7) -> ReshardCase:
                     st.metas.append(ShardMeta(name, w, w, (n,), (a,), (b - a,), r, st.buf_bytes[r]))
                     st.buf_bytes[r] += (b - a) * w
     return ReshardCase(f"many-tiny-{n_tensors}", src, dst, "index", seed)
+
+
+def random_convert_case(seed: int, *, narrow: bool = True, big: bool = False, dst_replicas: int = 1) -> ReshardCase:
+    """Random problem in which about half of the tensors change their element type on the way
+    (4-byte saved, 2-byte wanted when `narrow`, else the reverse; dtype tag = item size) and the
+    rest are moved unchanged.  Fill them with bit patterns, not values: every pattern is legal."""
+    rng = np.random.default_rng(seed)
+    a, b = (4, 2) if narrow else (2, 4)
+    if big:
+        shapes = [(1000, 517), (50257, 6), (9, 130, 67), (300_001,), (4, 3, 33, 65), ()]
+    else:
+        shapes = [tuple(int(rng.integers(1, 8)) for _ in range(int(rng.integers(0, 4)))) for _ in range(5)]
+    saved, wanted = [], []
+    for t, shape in enumerate(shapes):
+        if t % 2 == 0 or rng.random() < 0.3:
+            saved.append((f"c{t}.w", shape, a))
+            wanted.append((f"c{t}.w", shape, b))
+        else:
+            isz = int(rng.choice([1, 2, 4, 8]))
+            saved.append((f"c{t}.w", shape, isz))
+            wanted.append((f"c{t}.w", shape, isz))
+    parts = 4 if big else 3
+    src = random_side(rng, saved, int(rng.integers(1, 4)), max_parts=parts, gap_mod=7, element_aligned=True)
+    dst = random_side(rng, wanted, int(rng.integers(1, 4)), max_parts=3, gap_mod=7, replicas=dst_replicas, element_aligned=True)
+    return ReshardCase(f"random-convert-{seed}-{'narrow' if narrow else 'widen'}{'-big' if big else ''}", src, dst, "index", seed,
+                       convert=(1 if narrow else 2, a, b))
