@@ -1,0 +1,197 @@
+"""Resharding across several GPUs: saved blobs and target buffers are spread over the ranks of
+a process group (one process per GPU), and every rank materialises its own target buffers.
+
+The paper's load pipeline has exactly one exchange step: every saved shard is read by one
+rank and the pieces other ranks need travel in an all-to-all (Sec. 4.1, "Eliminating redundant
+loading", and the load pipeline of Sec. 4.2).  Here the saved blobs already sit in the HBM of
+their owners, so the same step becomes:
+
+  1. every rank plans its own targets against the GLOBAL saved metadata (host only) and reads
+     off the plan which saved entries it touches;
+  2. the lists of needed entries are gathered, so every owner knows what to send to whom;
+  3. every owner packs, per receiver, the needed entries of its blobs into one send buffer
+     (`bcp_pack`, on the GPU), and one `all_to_all_single` moves the segments (NCCL over NVLink);
+  4. every rank re-plans its targets against the entries as they now lie in its memory (its
+     own blobs plus one received segment per peer) and executes that plan (`bcp_reshard`).
+
+Steps 1, 2 and 4's planning are metadata work; all bytes move in library kernels and in the
+collective.  Everything here is argument marshalling around the C ABI and `torch.distributed`.
+"""
+from __future__ import annotations
+
+import copy
+from bisect import bisect_right
+from dataclasses import dataclass, field
+from typing import Callable, Dict, List, Optional, Sequence, Tuple
+
+from . import api
+
+SEGMENT_ALIGN = 256  # entries inside a send segment, and segments inside the buffers
+
+
+@dataclass
+class Exchange:
+    """What one rank sends, receives and finally executes."""
+
+    rank: int
+    world: int
+    local_src: List[int]                 # global indices of the saved blobs this rank owns, in local order
+    local_dst: List[int]                 # global indices of the target buffers this rank fills, in local order
+    send_entries: List[List[int]]        # per receiver: indices into the global saved metas, in pack order
+    send_offsets: List[List[int]]        # per receiver: byte offset of every such entry inside the segment
+    send_bytes: List[int]                # per receiver: segment size (multiple of SEGMENT_ALIGN; 0 for none / self)
+    recv_bytes: List[int]                # per sender
+    plan: Optional[api.Plan] = None      # final plan: sources = own blobs, then one segment per sender with recv_bytes > 0
+    src_buf_bytes: List[int] = field(default_factory=list)
+    dst_buf_bytes: List[int] = field(default_factory=list)
+
+    def destroy(self) -> None:
+        if self.plan is not None:
+            self.plan.destroy()
+            self.plan = None
+
+
+def _local_targets(dst_metas: Sequence, dst_buf_bytes: Sequence[int], dst_owner: Sequence[int], rank: int):
+    """This rank's target entries with buffer indices renumbered densely."""
+    mine = [b for b, o in enumerate(dst_owner) if o == rank]
+    local = {b: i for i, b in enumerate(mine)}
+    metas = []
+    for m in dst_metas:
+        if m.buf_index in local:
+            k = copy.copy(m)
+            k.buf_index = local[m.buf_index]
+            metas.append(k)
+    return mine, metas, [dst_buf_bytes[b] for b in mine]
+
+
+def needed_entries(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas: Sequence, dst_buf_bytes: Sequence[int],
+                   dst_owner: Sequence[int], rank: int, **opts) -> List[int]:
+    """Indices of the saved entries whose bytes this rank's targets read.  The planner does the
+    matching; this only maps the source ranges of its work units back to entries."""
+    _, mine, mine_bytes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
+    probe = api.bcp_plan(src_metas, src_buf_bytes, mine, mine_bytes, **opts)
+    try:
+        starts: Dict[int, List[int]] = {}
+        index: Dict[int, List[int]] = {}
+        order = sorted((i for i, m in enumerate(src_metas) if m.byte_length), key=lambda i: (src_metas[i].buf_index, src_metas[i].byte_offset))
+        for i in order:
+            starts.setdefault(src_metas[i].buf_index, []).append(src_metas[i].byte_offset)
+            index.setdefault(src_metas[i].buf_index, []).append(i)
+        used = set()
+        for t in probe.tiles():
+            if t.flags & api.TILE_ZERO:
+                continue
+            kind = (t.flags & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
+            row = t.row_bytes * 2 if kind == api.CONVERT_F32_TO_BF16 else t.row_bytes // 2 if kind else t.row_bytes
+            s, ix = starts[t.src_buf], index[t.src_buf]
+            lo, hi = t.src_off, t.src_off + (t.rows - 1) * t.src_pitch + row
+            k = bisect_right(s, lo) - 1
+            while k < len(s) and s[k] < hi:  # a coalesced unit may span several adjacent entries
+                m = src_metas[ix[k]]
+                if m.byte_offset + m.byte_length > lo:
+                    used.add(ix[k])
+                k += 1
+    finally:
+        probe.destroy()
+    return sorted(used)
+
+
+def build_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: Sequence[int], dst_metas: Sequence,
+                   dst_buf_bytes: Sequence[int], dst_owner: Sequence[int], rank: int, world: int,
+                   all_needs: Sequence[Sequence[int]], **opts) -> Exchange:
+    """all_needs[r] = needed_entries(...) of rank r, for every rank (gathered by the caller)."""
+    owner_of = lambda i: src_owner[src_metas[i].buf_index]  # noqa: E731
+    send_entries, send_offsets, send_bytes = [], [], []
+    for q in range(world):
+        ents = [i for i in all_needs[q] if owner_of(i) == rank] if q != rank else []
+        offs, total = api.bcp_pack_layout([src_metas[i].byte_length for i in ents], SEGMENT_ALIGN) if ents else ([], 0)
+        send_entries.append(ents)
+        send_offsets.append(offs)
+        send_bytes.append(total)
+    # what arrives, and where every needed entry will lie in this rank's memory
+    local_src = [b for b, o in enumerate(src_owner) if o == rank]
+    local_id = {b: i for i, b in enumerate(local_src)}
+    metas, sizes = [], [src_buf_bytes[b] for b in local_src]
+    recv_bytes = [0] * world
+    by_sender: Dict[int, List[int]] = {}
+    for i in all_needs[rank]:
+        by_sender.setdefault(owner_of(i), []).append(i)
+    for s in range(world):
+        ents = by_sender.get(s, [])
+        if s == rank:
+            for i in ents:
+                k = copy.copy(src_metas[i])
+                k.buf_index = local_id[k.buf_index]
+                metas.append(k)
+            continue
+        if not ents:
+            continue
+        offs, total = api.bcp_pack_layout([src_metas[i].byte_length for i in ents], SEGMENT_ALIGN)
+        recv_bytes[s] = total
+        for i, o in zip(ents, offs):
+            k = copy.copy(src_metas[i])
+            k.buf_index, k.byte_offset = len(sizes), o
+            metas.append(k)
+        sizes.append(total)
+    local_dst, mine, mine_bytes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
+    plan = api.bcp_plan(metas, sizes, mine, mine_bytes, **opts)
+    return Exchange(rank, world, local_src, local_dst, send_entries, send_offsets, send_bytes, recv_bytes, plan, sizes, mine_bytes)
+
+
+def plan_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: Sequence[int], dst_metas: Sequence,
+                  dst_buf_bytes: Sequence[int], dst_owner: Sequence[int], **opts) -> Exchange:
+    """Collective: every rank of the default process group calls this with the same metadata."""
+    import torch.distributed as dist
+
+    rank, world = (dist.get_rank(), dist.get_world_size()) if dist.is_initialized() else (0, 1)
+    mine = needed_entries(src_metas, src_buf_bytes, dst_metas, dst_buf_bytes, dst_owner, rank, **opts)
+    all_needs: List = [None] * world
+    if world > 1:
+        dist.all_gather_object(all_needs, mine)
+    else:
+        all_needs[0] = mine
+    return build_exchange(src_metas, src_buf_bytes, src_owner, dst_metas, dst_buf_bytes, dst_owner, rank, world, all_needs, **opts)
+
+
+def pack_sends(x: Exchange, src_metas: Sequence, local_blobs: Sequence, send_buf, stream=None) -> None:
+    """Step 3, sender side: the needed entries of this rank's blobs, one segment per receiver,
+    into `send_buf` (device, sum(send_bytes) bytes) with one multi-tensor pack."""
+    local_id = {b: i for i, b in enumerate(x.local_src)}
+    ptrs, metas, base = [], [], 0
+    for q in range(x.world):
+        for i, o in zip(x.send_entries[q], x.send_offsets[q]):
+            m = src_metas[i]
+            ptrs.append(local_blobs[local_id[m.buf_index]].data_ptr() + m.byte_offset)
+            metas.append((base + o, m.byte_length))
+        base += x.send_bytes[q]
+    if base:
+        api.bcp_pack(ptrs, metas, send_buf, base, stream=stream)
+
+
+def run_exchange(x: Exchange, src_metas: Sequence, local_blobs: Sequence, dst_bufs: Sequence, stream=None,
+                 all_to_all: Optional[Callable] = None):
+    """Steps 3 and 4 on the current device.  `all_to_all(recv, send, recv_splits, send_splits)`
+    defaults to `torch.distributed.all_to_all_single`; returns the buffers that must stay alive
+    until the stream has run (send buffer, receive buffer)."""
+    import torch
+
+    dev = local_blobs[0].device if local_blobs else dst_bufs[0].device
+    send = torch.empty(max(1, sum(x.send_bytes)), dtype=torch.uint8, device=dev)
+    recv = torch.empty(max(1, sum(x.recv_bytes)), dtype=torch.uint8, device=dev)
+    pack_sends(x, src_metas, local_blobs, send, stream)
+    if x.world > 1:
+        if all_to_all is None:
+            import torch.distributed as dist
+
+            s = torch.cuda.current_stream() if stream is None else stream
+            with torch.cuda.stream(s):
+                dist.all_to_all_single(recv[: sum(x.recv_bytes)], send[: sum(x.send_bytes)], list(x.recv_bytes), list(x.send_bytes))
+        else:
+            all_to_all(recv, send, list(x.recv_bytes), list(x.send_bytes))
+    srcs, at = list(local_blobs), 0
+    for s in range(x.world):
+        if x.recv_bytes[s]:
+            srcs.append(recv[at:at + x.recv_bytes[s]])
+            at += x.recv_bytes[s]
+    api.bcp_reshard(x.plan, srcs, dst_bufs, stream=stream)
+    return send, recv

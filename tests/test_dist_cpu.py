@@ -51,3 +51,70 @@ def test_single_process_is_a_no_op():
     finally:
         if env_ws is not None:
             os.environ["WORLD_SIZE"] = env_ws
+
+
+# ---- cross-rank resharding: the exchange schedule on two gloo ranks ------------------------------
+EXCHANGE_WORKER = textwrap.dedent("""
+    import os, sys
+    sys.path.insert(0, %r)
+    sys.path.insert(0, os.path.join(%r, "tests"))
+    import numpy as np, torch, torch.distributed as tdist
+    from paper_2407_20143_b200 import dist, multi
+    from oracle import reshard_oracle as orc
+    from workloads import fills
+    from workloads.configs import scenario_cases, convert_cases
+    from test_planner import run_tiles
+    assert dist.init("gloo")
+    rank, _, ws = dist.world()
+    for case in [c for c in scenario_cases() if c.name in ("hybrid", "llama-tp8-to-tp2", "dp4-to-dp8")] + convert_cases()[:1]:
+        opts = case.plan_opts
+        src_owner = [b %% ws for b in range(len(case.src.buf_bytes))]            # saved blobs round-robin over the ranks
+        nd = len(case.dst.buf_bytes)
+        dst_owner = [((b // 2) if nd >= 4 else b) %% ws for b in range(nd)]      # target buffers in pairs (singly when there are two)
+        x = multi.plan_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, **opts)
+        blobs = [t.numpy() for t in fills.fill_state(case.src, case.key_ids, "index", case.seed, "cpu")]
+        # stand-in for the device pack: the schedule's entries at the schedule's offsets
+        send = np.zeros(max(1, sum(x.send_bytes)), dtype=np.uint8)
+        base = 0
+        for q in range(ws):
+            for i, o in zip(x.send_entries[q], x.send_offsets[q]):
+                m = case.src.metas[i]
+                assert src_owner[m.buf_index] == rank and q != rank
+                send[base + o:base + o + m.byte_length] = blobs[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length]
+            base += x.send_bytes[q]
+        recv = torch.zeros(max(1, sum(x.recv_bytes)), dtype=torch.uint8)
+        tdist.all_to_all_single(recv[:sum(x.recv_bytes)], torch.from_numpy(send)[:sum(x.send_bytes)], list(x.recv_bytes), list(x.send_bytes))
+        srcs, at = [blobs[b] for b in x.local_src], 0
+        for s in range(ws):
+            if x.recv_bytes[s]:
+                srcs.append(recv[at:at + x.recv_bytes[s]].numpy())
+                at += x.recv_bytes[s]
+        assert [len(s) for s in srcs] == x.src_buf_bytes
+        got, _ = run_tiles(x.plan.tiles(), srcs, x.dst_buf_bytes)
+        want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, convert=case.convert)
+        assert len(x.local_dst) > 0 and sum(x.recv_bytes) > 0 and sum(x.send_bytes) > 0, case.name
+        for g, b in zip(got, x.local_dst):
+            assert np.array_equal(g, want[b]), (case.name, rank, b)
+        # nothing is sent that the receiver does not read, and nothing twice
+        assert all(len(set(e)) == len(e) for e in x.send_entries)
+        x.destroy()
+    dist.barrier()
+    print("exchange ok", rank)
+    dist.shutdown()
+""") % (ROOT, ROOT)
+
+
+def test_two_rank_exchange_schedule(tmp_path):
+    """Every rank plans its targets against the global metadata, the needed saved entries travel in
+    one all-to-all with the schedule's split sizes, and the final per-rank plan, run by the numpy
+    unit simulator on the bytes as they arrived, equals the oracle on that rank's targets."""
+    script = tmp_path / "exchange_worker.py"
+    script.write_text(EXCHANGE_WORKER)
+    port = 29900 + os.getpid() % 90
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=300) for p in procs]
+    assert all(p.returncode == 0 for p in procs), outs
+    assert all("exchange ok" in o[0] for o in outs)

@@ -1,0 +1,63 @@
+"""Cross-rank resharding on one GPU: the ranks of a 2- and 3-rank job are emulated one after the
+other in one process (pack of all ranks, then the segment swap an all-to-all would do, then every
+rank's reshard), so every device step of the exchange runs through the library; only the
+collective itself is replaced by tensor copies.  No kernel waits for another."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2407_20143_b200 import multi
+from oracle import reshard_oracle as orc
+from workloads import fills
+from workloads.configs import convert_cases, scenario_cases
+from workloads.random_cases import big_random_case
+
+pytestmark = pytest.mark.gpu
+POISON = 0xA5
+
+CASES = [c for c in scenario_cases() if c.name in ("hybrid", "dp150-to-dp75", "llama-tp8-to-tp2")] + [big_random_case(4, itemsize=2), convert_cases()[1]]
+
+
+@pytest.mark.parametrize("world", [1, 2, 3])
+@pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
+def test_emulated_ranks_exchange_and_reshard(cuda_device, case, world):
+    ns, nd = len(case.src.buf_bytes), len(case.dst.buf_bytes)
+    src_owner = [b % world for b in range(ns)]
+    dst_owner = [(b * world) // nd for b in range(nd)]  # contiguous blocks of target buffers
+    opts = case.plan_opts
+    blobs = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device, poison=0x5A)
+    want = orc.reshard(case.src.metas, [b.cpu().numpy() for b in blobs], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON,
+                       convert=case.convert)
+    needs = [multi.needed_entries(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, dst_owner, r, **opts)
+             for r in range(world)]
+    xs = [multi.build_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, r, world,
+                               needs, **opts) for r in range(world)]
+    # sender side of every rank
+    sends = []
+    for x in xs:
+        buf = torch.full((max(1, sum(x.send_bytes)),), 0xEE, dtype=torch.uint8, device=cuda_device)
+        multi.pack_sends(x, case.src.metas, [blobs[b] for b in x.local_src], buf)
+        sends.append(buf)
+    torch.cuda.synchronize()
+    for r, x in enumerate(xs):
+        assert x.recv_bytes == [xs[s].send_bytes[r] for s in range(world)]
+
+        def swap(recv, send, recv_splits, send_splits, r=r):  # what all_to_all_single does, from the emulated peers' buffers
+            at = 0
+            for s in range(world):
+                off = sum(xs[s].send_bytes[:r])
+                recv[at:at + recv_splits[s]].copy_(sends[s][off:off + recv_splits[s]])
+                at += recv_splits[s]
+
+        dst = [torch.full((n,), POISON, dtype=torch.uint8, device=cuda_device) for n in x.dst_buf_bytes]
+        keep = multi.run_exchange(x, case.src.metas, [blobs[b] for b in x.local_src], dst, all_to_all=swap)
+        torch.cuda.synchronize()
+        for d, b in zip(dst, x.local_dst):
+            assert np.array_equal(d.cpu().numpy(), want[b]), (case.name, world, r, b)
+        del keep
+    # every target buffer has exactly one owner
+    assert sorted(b for x in xs for b in x.local_dst) == list(range(nd))
+    if world > 1:  # bytes that crossed ranks: at most what the targets read, and none for a rank's own blobs
+        assert all(x.send_bytes[x.rank] == 0 for x in xs) and sum(sum(x.send_bytes) for x in xs) > 0
+    for x in xs:
+        x.destroy()
