@@ -87,6 +87,19 @@ class Plan:
         _check(L.lib().bcp_plan_tiles(self.handle, arr, n.value, C.byref(n)))
         return list(arr[: n.value])
 
+    def tiles_array(self):
+        """The same records as one numpy structured array (fields as in bcp_tile), for long lists."""
+        import numpy as np
+
+        n = C.c_size_t()
+        _check(L.lib().bcp_plan_tiles(self.handle, None, 0, C.byref(n)))
+        arr = (L.TileC * max(1, n.value))()
+        _check(L.lib().bcp_plan_tiles(self.handle, arr, n.value, C.byref(n)))
+        dt = np.dtype([("src_off", "<u8"), ("dst_off", "<u8"), ("src_pitch", "<u8"), ("dst_pitch", "<u8"), ("row_bytes", "<u4"),
+                       ("rows", "<u4"), ("src_buf", "<u4"), ("dst_buf", "<u4"), ("flags", "<u4"), ("reserved", "<u4", (3,))])
+        assert dt.itemsize == C.sizeof(L.TileC)
+        return np.frombuffer(arr, dtype=dt, count=n.value)
+
     def serialize(self) -> bytes:
         """Self-contained image of the plan (bcp_plan_serialize) for reuse in another process."""
         n = C.c_size_t()

@@ -20,7 +20,6 @@ collective.  Everything here is argument marshalling around the C ABI and `torch
 from __future__ import annotations
 
 import copy
-from bisect import bisect_right
 from dataclasses import dataclass, field
 from typing import Callable, Dict, List, Optional, Sequence, Tuple
 
@@ -71,26 +70,30 @@ def needed_entries(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas:
     _, mine, mine_bytes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
     probe = api.bcp_plan(src_metas, src_buf_bytes, mine, mine_bytes, **opts)
     try:
-        starts: Dict[int, List[int]] = {}
-        index: Dict[int, List[int]] = {}
-        order = sorted((i for i, m in enumerate(src_metas) if m.byte_length), key=lambda i: (src_metas[i].buf_index, src_metas[i].byte_offset))
-        for i in order:
-            starts.setdefault(src_metas[i].buf_index, []).append(src_metas[i].byte_offset)
-            index.setdefault(src_metas[i].buf_index, []).append(i)
-        used = set()
-        for t in probe.tiles():
-            if t.flags & api.TILE_ZERO:
-                continue
-            kind = (t.flags & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
-            row = t.row_bytes * 2 if kind == api.CONVERT_F32_TO_BF16 else t.row_bytes // 2 if kind else t.row_bytes
-            s, ix = starts[t.src_buf], index[t.src_buf]
-            lo, hi = t.src_off, t.src_off + (t.rows - 1) * t.src_pitch + row
-            k = bisect_right(s, lo) - 1
-            while k < len(s) and s[k] < hi:  # a coalesced unit may span several adjacent entries
-                m = src_metas[ix[k]]
-                if m.byte_offset + m.byte_length > lo:
-                    used.add(ix[k])
-                k += 1
+        import numpy as np
+
+        tiles = probe.tiles_array()
+        tiles = tiles[(tiles["flags"] & api.TILE_ZERO) == 0]
+        kind = (tiles["flags"] & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
+        row = tiles["row_bytes"].astype(np.uint64)
+        row = np.where(kind == api.CONVERT_F32_TO_BF16, row * 2, np.where(kind == api.CONVERT_BF16_TO_F32, row // 2, row))
+        lo = tiles["src_off"]
+        hi = lo + (tiles["rows"].astype(np.uint64) - 1) * tiles["src_pitch"] + row  # a rectangle lies inside one entry
+        named = np.array([i for i, m in enumerate(src_metas) if m.byte_length], dtype=np.int64)
+        bufs = np.array([src_metas[i].buf_index for i in named], dtype=np.int64)
+        offs = np.array([src_metas[i].byte_offset for i in named], dtype=np.uint64)
+        used: List[int] = []
+        for b in np.unique(tiles["src_buf"]):
+            sel = named[bufs == b]
+            sel = sel[np.argsort(offs[bufs == b], kind="stable")]
+            starts = np.array([src_metas[i].byte_offset for i in sel], dtype=np.uint64)
+            of_buf = tiles["src_buf"] == b
+            first = np.searchsorted(starts, lo[of_buf], side="right") - 1   # entry that holds the unit's first byte
+            last = np.searchsorted(starts, hi[of_buf], side="left")          # a coalesced run may span adjacent entries
+            mark = np.zeros(len(sel) + 1, dtype=np.int64)
+            np.add.at(mark, first, 1)
+            np.add.at(mark, last, -1)
+            used.extend(int(i) for i in sel[np.cumsum(mark[:-1]) > 0])
     finally:
         probe.destroy()
     return sorted(used)
