@@ -154,6 +154,8 @@ typedef struct {
                                whose saved entries have dtype_tag convert_src_tag and whose wanted entries have
                                dtype_tag convert_dst_tag (itemsizes 4 and 2, resp. 2 and 4) is converted
                                element by element while it is resharded; every other FQN is moved unchanged.
+                               Entries of a converted FQN must start on a multiple of their item size
+                               (BCP_ERR_INVALID otherwise; plain copies may start at any byte).
                                The paper moves bytes only; this serves the hand-over of fp32 master weights
                                to a bf16 evaluation job (and back).                                       */
   uint32_t convert_src_tag; /* see convert */

@@ -118,3 +118,38 @@ def test_two_rank_exchange_schedule(tmp_path):
     outs = [p.communicate(timeout=300) for p in procs]
     assert all(p.returncode == 0 for p in procs), outs
     assert all("exchange ok" in o[0] for o in outs)
+
+
+def test_exchange_schedule_properties_without_a_process_group():
+    """Host logic of the exchange on emulated ranks: what one rank sends is what the other expects,
+    only needed entries travel, a rank's own blobs are never sent, and with one rank nothing moves."""
+    from paper_2407_20143_b200 import multi
+    from workloads.configs import scenario_cases
+
+    case = [c for c in scenario_cases() if c.name == "hybrid"][0]
+    ns, nd = len(case.src.buf_bytes), len(case.dst.buf_bytes)
+    for world in (1, 2, 4):
+        src_owner = [b % world for b in range(ns)]
+        dst_owner = [(b * world) // nd for b in range(nd)]
+        needs = [multi.needed_entries(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, dst_owner, r)
+                 for r in range(world)]
+        xs = [multi.build_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner,
+                                   r, world, needs) for r in range(world)]
+        for r, x in enumerate(xs):
+            assert x.recv_bytes == [xs[s].send_bytes[r] for s in range(world)]
+            assert x.send_bytes[r] == 0 and x.send_entries[r] == []
+            for q in range(world):
+                assert set(x.send_entries[q]) <= set(needs[q])
+                assert all(src_owner[case.src.metas[i].buf_index] == r for i in x.send_entries[q])
+                assert x.send_bytes[q] % multi.SEGMENT_ALIGN == 0
+            # the final plan writes exactly this rank's target bytes
+            mine = sum(m.byte_length for m in case.dst.metas if dst_owner[m.buf_index] == r)
+            assert x.plan.stats()["bytes_copied"] == mine
+        # every needed entry is either local or sent by its owner, once
+        for q in range(world):
+            got = sorted(i for x in xs for i in x.send_entries[q]) + [i for i in needs[q] if src_owner[case.src.metas[i].buf_index] == q]
+            assert sorted(got) == sorted(needs[q])
+        if world == 1:
+            assert xs[0].send_bytes == [0] and xs[0].recv_bytes == [0] and xs[0].local_dst == list(range(nd))
+        for x in xs:
+            x.destroy()
