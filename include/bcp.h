@@ -323,8 +323,11 @@ BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, si
  * sources and targets not overlapping; counts must equal the planned ones.  The call uploads the
  * work list on first use, enqueues the pointer tables and the copy kernel on `stream`
  * and returns without waiting; buffers must stay valid until the stream reaches that
- * point.  Executions of one plan must be ordered (same stream, or externally
- * synchronised): they share the plan's device-side pointer tables and ticket counter.
+ * point.  Executions of one plan share its device-side pointer tables and ticket counters,
+ * so they are ordered: on one stream by the stream; when the stream differs from that of the
+ * previous execution, the new stream is made to wait (on the device) for what is queued on the
+ * previous one.  Calls on one plan from several host threads must not overlap, and inside a
+ * stream capture the caller orders the executions.
  * Target bytes not named by any target entry are left untouched.
  * Once a plan has run on a set of buffer addresses, running it again on the same addresses
  * enqueues kernel launches only (no allocation, no copy, no synchronisation), so the call
@@ -377,7 +380,8 @@ BCP_API int bcp_pack_layout(const uint64_t* tensor_bytes, size_t n, uint64_t ali
  * by byte_offset and non-overlapping, inside blob_bytes.  tensors and metas are host
  * arrays.  Tensor and blob addresses need no particular alignment (16-byte aligned ones
  * copy fastest).  Asynchronous on `stream`.  Work lists are cached inside the library per
- * (metas, blob_bytes), so repeated packs of the same layout only upload pointers.
+ * (metas, blob_bytes), so repeated packs of the same layout only upload pointers; packs of one
+ * layout issued on different streams run one after the other (see bcp_reshard).
  */
 BCP_API int bcp_pack(const void* const* tensors, const bcp_pack_meta* metas, size_t n, void* blob,
              uint64_t blob_bytes, void* stream);

@@ -31,6 +31,7 @@ struct bcp_plan_s {
   Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel, [2] converting kernel
   uint32_t grid = 0, tma_grid = 0, cvt_grid = 0;
   cudaStream_t last_stream = nullptr;
+  cudaEvent_t ev_switch = nullptr;  // orders an execution after the previous one when the stream changes
   bool ran = false;
   std::vector<void*> h_ptrs;
   bool table_current = false;  // the device pointer table already holds h_ptrs
@@ -229,6 +230,23 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
     if (reinterpret_cast<uintptr_t>(dst[i]) & 15) return fail(BCP_ERR_INVALID, "target buffer %zu is not 16-byte aligned", i);
   if (int rc = bind_device(p)) return rc;
   if (p->tiles.empty()) return BCP_OK;
+  // Executions of a plan share its pointer tables and ticket counters.  On the same stream they
+  // are ordered anyway; when the stream changes (two users of one cached pack layout, say) the
+  // new stream is made to wait for everything queued on the previous one.  Not during a stream
+  // capture, which must not depend on outside work: there the caller orders the executions.
+  if (p->ran && p->last_stream != stream) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+      if (!p->ev_switch) BCP_CUDA(cudaEventCreateWithFlags(&p->ev_switch, cudaEventDisableTiming));
+      if (cudaEventRecord(p->ev_switch, p->last_stream) == cudaSuccess) {
+        BCP_CUDA(cudaStreamWaitEvent(stream, p->ev_switch, 0));
+      } else {
+        cudaGetLastError();  // the previous stream no longer exists (then its work is done) or is being captured
+      }
+    } else {
+      cudaGetLastError();
+    }
+  }
   // The device pointer table is refreshed only when a base address changed since the last
   // execution (executions of a plan are ordered, so the previous upload has been consumed).
   bool same = p->table_current;
@@ -867,6 +885,7 @@ int bcp_plan_destroy(bcp_plan_t* plan) {
     }
     if (plan->s_h2d) cudaStreamSynchronize(plan->s_h2d);
     if (plan->s_d2h) cudaStreamSynchronize(plan->s_d2h);
+    if (plan->ev_switch) cudaEventDestroy(plan->ev_switch);
     for (cudaEvent_t e : plan->ev_src)
       if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : plan->ev_dst)

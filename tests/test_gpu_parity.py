@@ -601,3 +601,44 @@ def test_converting_reshard_from_host_buffers(cuda_device):
         bcp.bcp_reshard_host(plan, a, dst)
         assert all(np.array_equal(d.numpy(), w) for d, w in zip(dst, want))
     plan.destroy()
+
+
+# ---- one plan, two streams -----------------------------------------------------------------------
+def test_same_layout_on_two_streams_is_ordered(cuda_device):
+    """Packs of one layout share a cached work list (pointer table, ticket counters); issued on two
+    streams back to back, the second must wait for the first instead of racing it.  Same for a plan
+    the caller executes on two streams."""
+    n, parts = 96 << 20, 6
+    sizes = [n // parts] * parts
+    offs, total = bcp.bcp_pack_layout(sizes, 256)
+    metas = list(zip(offs, sizes))
+    s1, s2 = torch.cuda.Stream(device=cuda_device), torch.cuda.Stream(device=cuda_device)
+    a = [torch.full((m,), 1 + i, dtype=torch.uint8, device=cuda_device) for i, m in enumerate(sizes)]
+    b = [torch.full((m,), 101 + i, dtype=torch.uint8, device=cuda_device) for i, m in enumerate(sizes)]
+    blob_a = torch.full((total,), POISON, dtype=torch.uint8, device=cuda_device)
+    blob_b = torch.full((total,), POISON, dtype=torch.uint8, device=cuda_device)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        bcp.bcp_pack(a, metas, blob_a, stream=s1)
+        bcp.bcp_pack(b, metas, blob_b, stream=s2)  # no host synchronisation in between
+    torch.cuda.synchronize()
+    for i, (o, m) in enumerate(metas):
+        assert bool((blob_a[o:o + m] == 1 + i).all()) and bool((blob_b[o:o + m] == 101 + i).all())
+    # a plan executed alternately on two streams, with different buffers
+    case = big_random_case(2, itemsize=4)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, path_mask=3, tile_bytes=8192)
+    src1 = fills.fill_state(case.src, case.key_ids, "index", 1, cuda_device)
+    src2 = fills.fill_state(case.src, case.key_ids, "index", 2, cuda_device)
+    want1 = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src1], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    want2 = orc.reshard(case.src.metas, [s.cpu().numpy() for s in src2], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    dst1 = [torch.full((m,), POISON, dtype=torch.uint8, device=cuda_device) for m in case.dst.buf_bytes]
+    dst2 = [torch.full((m,), POISON, dtype=torch.uint8, device=cuda_device) for m in case.dst.buf_bytes]
+    torch.cuda.synchronize()
+    for _ in range(4):
+        bcp.bcp_reshard(plan, src1, dst1, stream=s1)
+        bcp.bcp_reshard(plan, src2, dst2, stream=s2)
+    torch.cuda.synchronize()
+    bcp.bcp_plan_device_status(plan)
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst1, want1))
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst2, want2))
+    plan.destroy()
