@@ -39,8 +39,9 @@ METRIC = "reshard GB/s (bytes read+written, device-timed)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes moved per algorithmic byte by the dominant kernel, from ncu captures summarised
-# under profiles/ (bcp_tma_kernel_*.md): (dram__bytes_read.sum + dram__bytes_write.sum) / B_min.
-NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.9994, ("cfg3", "bcp_tma_kernel"): 0.9990}
+# under profiles/ (bcp_tma_kernel_*.md, bcp_convert_kernel_*.md): (dram__bytes_read.sum + dram__bytes_write.sum) / B_min.
+NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.9994, ("cfg3", "bcp_tma_kernel"): 0.9990,
+                                       ("cfg4", "bcp_tma_kernel"): 0.9998, ("evalmerge", "bcp_convert_kernel"): 0.9994}
 
 
 def parse_args():
@@ -374,7 +375,8 @@ def main():
     if ratio is not None:
         out["roofline"]["traffic"] = ratio * b_min
         out["roofline"]["traffic_note"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch " \
-                                          "(profiles/bcp_tma_kernel_full_size_dram_bytes.md)"
+                                          "(profiles/" + ("bcp_convert_kernel_evalmerge-L2_ncu_full.md" if case.convert else
+                                                          "bcp_tma_kernel_full_size_dram_bytes.md") + ")"
         if a.layers:
             out["roofline"]["traffic_note"] += ", scaled by algorithmic bytes to this shallower model"
 
