@@ -213,7 +213,7 @@ typedef struct {
 #define BCP_TILE_CVT_MASK (3u << BCP_TILE_CVT_SHIFT)
 
 typedef struct {
-  uint64_t n_src_entries;    /* after decomposing flat slices                        */
+  uint64_t n_src_entries;    /* after decomposing flat slices; tensors no wanted entry names are left out */
   uint64_t n_dst_entries;
   uint64_t n_fqns;
   uint64_t n_intersections;  /* non-empty source x target box intersections          */

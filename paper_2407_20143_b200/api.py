@@ -7,6 +7,7 @@ tensors to device pointers.
 from __future__ import annotations
 
 import ctypes as C
+import struct
 from typing import List, Optional, Sequence, Tuple
 
 from . import _lib as L
@@ -30,8 +31,11 @@ def _check(rc: int) -> None:
         raise BcpError(rc, L.lib().bcp_last_error().decode("utf-8", "replace"))
 
 
-def _metas_to_c(metas: Sequence) -> Tuple[C.Array, list]:
-    """Objects with the attributes of workloads.meta.ShardMeta -> array of bcp_shard_meta."""
+_META_FMT = struct.Struct("<Q4I%dq2q2I2Q" % (3 * L.BCP_MAX_NDIM))  # field for field bcp_shard_meta (little endian, no padding needed)
+_PAD = [(0,) * k for k in range(L.BCP_MAX_NDIM + 1)]
+
+
+def _metas_to_c_loop(metas: Sequence) -> Tuple[C.Array, list]:
     arr = (L.ShardMetaC * max(1, len(metas)))()
     keep = []
     for c, m in zip(arr, metas):
@@ -44,6 +48,37 @@ def _metas_to_c(metas: Sequence) -> Tuple[C.Array, list]:
         c.flat_begin, c.flat_end = m.flat_begin, m.flat_end
         c.buf_index, c.byte_offset, c.byte_length = m.buf_index, m.byte_offset, m.byte_length
     return arr, keep
+
+
+def _metas_to_c(metas: Sequence) -> Tuple[C.Array, list]:
+    """Objects with the attributes of workloads.meta.ShardMeta -> array of bcp_shard_meta (plus what
+    must stay alive with it).  Records are packed whole, names go into one NUL-separated buffer;
+    anything irregular (values a C field cannot hold, ragged shapes, NUL inside a name) goes
+    through the field-by-field loop, which passes it on for the library to judge."""
+    n = len(metas)
+    if _META_FMT.size != C.sizeof(L.ShardMetaC) or n == 0:
+        return _metas_to_c_loop(metas)
+    try:
+        names = [m.fqn.encode() for m in metas]
+        blob = b"\0".join(names) + b"\0"
+        if blob.count(b"\0") != n:
+            return _metas_to_c_loop(metas)
+        text = C.create_string_buffer(blob, len(blob))
+        at = C.addressof(text)
+        arr = (L.ShardMetaC * n)()
+        raw = (C.c_char * (n * _META_FMT.size)).from_buffer(arr)
+        pack, size, pad = _META_FMT.pack_into, _META_FMT.size, _PAD
+        for i, m in enumerate(metas):
+            g = m.global_shape
+            k = L.BCP_MAX_NDIM - len(g)
+            if len(m.offsets) != len(g) or len(m.lengths) != len(g):
+                return _metas_to_c_loop(metas)
+            pack(raw, i * size, at, m.itemsize, m.dtype_tag, len(g), m.kind, *g, *pad[k], *m.offsets, *pad[k], *m.lengths, *pad[k],
+                 m.flat_begin, m.flat_end, m.buf_index, 0, m.byte_offset, m.byte_length)
+            at += len(names[i]) + 1
+        return arr, [text]
+    except (struct.error, IndexError, TypeError, OverflowError):
+        return _metas_to_c_loop(metas)
 
 
 def _u64(xs: Sequence[int]) -> C.Array:

@@ -17,6 +17,7 @@
 #include <string>
 #include <string_view>
 #include <unordered_map>
+#include <unordered_set>
 
 #include "plan.hpp"
 
@@ -422,11 +423,18 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
     }
     return fail(BCP_ERR_MISMATCH, kDiffers, side, i, m.fqn);
   };
+  // A plan may cover a few target ranks against the saved metadata of a whole job (partial loads):
+  // saved entries of tensors that no wanted entry names are validated but take no further part.
+  std::unordered_set<std::string_view> wanted;
+  wanted.reserve(n_dst);
+  for (size_t i = 0; i < n_dst; ++i)
+    if (dst[i].fqn) wanted.emplace(dst[i].fqn);
   std::vector<RelBox> scratch;
   for (size_t i = 0; i < n_src; ++i) {
     int64_t n;
     uint32_t f;
     if (int rc = check_meta(src[i], "src", i, src_buf_bytes, n_src_bufs, &n)) return rc;
+    if (!wanted.count(src[i].fqn)) continue;
     if (int rc = family_of(src[i], "src", i, false, &f)) return rc;
     expand(src[i], uint32_t(i), n, &fams[f].src, &scratch);
   }
