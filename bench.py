@@ -531,10 +531,17 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     if not ok:
         return {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "skipped": reason or "another rank could not allocate"}
-    hsrc = [torch.empty(n, dtype=torch.uint8, pin_memory=True) for n in case.src.buf_bytes]
+    def host_buffers(sizes):  # pinned if the host allows it (memlock limits), else pageable
+        try:
+            return [torch.empty(n, dtype=torch.uint8, pin_memory=True) for n in sizes], True
+        except RuntimeError:
+            return [torch.empty(n, dtype=torch.uint8) for n in sizes], False
+
+    hsrc, pin_s = host_buffers(case.src.buf_bytes)
     for h, s in zip(hsrc, src):
         h.copy_(s)
-    hdst = [torch.empty(n, dtype=torch.uint8, pin_memory=True) for n in case.dst.buf_bytes]
+    hdst, pin_d = host_buffers(case.dst.buf_bytes)
+    pinned = pin_s and pin_d
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
     bcp.bcp_reshard_host(plan, hsrc, hdst, stream)  # warm-up: allocates the staging buffers
@@ -553,7 +560,8 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     moved_in = plan.stats()["bytes_src_unique" if case.convert else "bytes_copied"]
     return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": moved_in, "d2h_bytes_per_step": d2h,
             "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same,
-            "mode": "pinned host buffers read and written in place by the kernels (no staging copy)",
+            "mode": "pinned host buffers read and written in place by the kernels (no staging copy)" if pinned else
+                    "pageable host buffers (pinning failed) through device staging, uploads / kernels / downloads pipelined",
             "host_buffer_bytes": {"sources": h2d, "targets": d2h}}
 
 
