@@ -87,7 +87,7 @@ def odd_gpt(layers: int = 12) -> ReshardCase:
 
 
 STRESS: Dict[str, Callable[..., ReshardCase]] = {"cfg4odd": cfg4_odd, "narrow": narrow_rows, "oddgpt": odd_gpt,
-                                                   "evalmerge": lambda layers=32: eval_merge(layers)}
+                                                   "evalmerge": lambda layers=32: eval_merge(layers)}  # defined below
 
 CONFIGS: Dict[str, Callable[..., ReshardCase]] = {
     "cfg1": cfg1, "cfg2": cfg2, "cfg3": cfg3, "cfg4": cfg4, "cfg5": cfg5}
