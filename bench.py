@@ -515,6 +515,7 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     import torch
 
     import paper_2407_20143_b200 as bcp
+    from paper_2407_20143_b200 import api
     from paper_2407_20143_b200 import dist as D
 
     h2d, d2h = sum(case.src.buf_bytes), sum(case.dst.buf_bytes)
@@ -555,9 +556,17 @@ def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
     D.barrier()
     ms = D.max_over_ranks(e0.elapsed_time(e1) / a.e2e_steps, dev)
     same = all(bool(torch.equal(h[: 1 << 20], d[: 1 << 20].cpu())) for h, d in zip(hdst, dst))
-    # pinned buffers are addressed by the kernels directly: every unit's source bytes cross PCIe when
-    # it is copied (replica reads cross again), every target byte crosses once on its way out
-    moved_in = plan.stats()["bytes_src_unique" if case.convert else "bytes_copied"]
+    # pinned buffers are addressed by the kernels directly: the source bytes of every unit cross PCIe when
+    # it is staged (a group of replica units stages its source once; units of the register kernel read
+    # theirs every time), every target byte crosses once on its way out.  Counted from the work list.
+    if pinned:
+        u = plan.tiles_array()
+        reads = (u["flags"] & (api.TILE_FOLLOW | api.TILE_ZERO)) == 0
+        kind = (u["flags"] & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
+        per_row = u["row_bytes"].astype("int64") * (1 + (kind == 1)) // (1 + (kind == 2))
+        moved_in = int((u["rows"].astype("int64") * per_row)[reads].sum())
+    else:
+        moved_in = h2d  # staging uploads every source buffer once
     return {"value": b_min * ws / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": moved_in, "d2h_bytes_per_step": d2h,
             "ms_per_step": ms, "steps": a.e2e_steps, "matches_device_path": same,
             "mode": "pinned host buffers read and written in place by the kernels (no staging copy)" if pinned else
