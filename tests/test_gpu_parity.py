@@ -642,3 +642,30 @@ def test_same_layout_on_two_streams_is_ordered(cuda_device):
     assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst1, want1))
     assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst2, want2))
     plan.destroy()
+
+
+# ---- tracing -------------------------------------------------------------------------------------
+def test_trace_spans_time_stream_work(cuda_device, tmp_path):
+    from paper_2407_20143_b200.trace import Trace
+
+    case = CONFIGS["cfg1"]("index")
+    src = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device)
+    dst = fills.make_buffers(case.dst, cuda_device, POISON)
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    st = plan.stats()
+    moved = st["bytes_src_unique"] + st["bytes_copied"]
+    tr = Trace(rank=3)
+    for step in range(4):
+        with tr.span("reshard", nbytes=moved, step=step):
+            bcp.bcp_reshard(plan, src, dst)
+    with tr.span("idle"):
+        pass
+    rows = tr.rows()
+    assert [r["name"] for r in rows] == ["reshard"] * 4 + ["idle"] and all(r["rank"] == 3 for r in rows)
+    assert [r["step"] for r in rows[:4]] == [0, 1, 2, 3]
+    assert all(0.001 < r["ms"] < 50 and r["gbps"] > 1 for r in rows[:4]) and rows[4]["gbps"] is None
+    tot = tr.totals()
+    assert tot["reshard"]["calls"] == 4 and tot["reshard"]["bytes"] == 4 * moved
+    tr.dump(str(tmp_path / "trace.jsonl"))
+    assert len(open(tmp_path / "trace.jsonl").read().splitlines()) == 5
+    plan.destroy()
