@@ -326,8 +326,9 @@ BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, si
  * point.  Executions of one plan share its device-side pointer tables and ticket counters,
  * so they are ordered: on one stream by the stream; when the stream differs from that of the
  * previous execution, the new stream is made to wait (on the device) for what is queued on the
- * previous one.  Calls on one plan from several host threads must not overlap, and inside a
- * stream capture the caller orders the executions.
+ * previous one (so that stream must still exist then, and when the plan is destroyed).  Calls on
+ * one plan from several host threads must not overlap, and inside a stream capture the caller
+ * orders the executions.
  * Target bytes not named by any target entry are left untouched.
  * Once a plan has run on a set of buffer addresses, running it again on the same addresses
  * enqueues kernel launches only (no allocation, no copy, no synchronisation), so the call
