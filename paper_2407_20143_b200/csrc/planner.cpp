@@ -187,6 +187,7 @@ struct Family {
   bool has_src, has_dst;
   int64_t shape[BCP_MAX_NDIM];
   std::vector<Entry> src, dst;
+  std::vector<uint32_t> src_metas, dst_metas;  // input entries of this tensor, expanded into src / dst when it is matched
 };
 
 const int64_t kMaxElems = int64_t(1) << 60;
@@ -374,6 +375,39 @@ struct SegKey {
 
 }  // namespace
 
+namespace {
+
+// Host threads for large work lists.  The result never depends on the count.
+unsigned plan_threads(size_t n_units) {
+  if (n_units < 32768) return 1;
+  unsigned n = 0;
+  if (const char* e = getenv("BCP_PLAN_THREADS")) n = unsigned(strtoul(e, nullptr, 10));
+  if (!n) n = std::min(8u, std::thread::hardware_concurrency());
+  return std::max(1u, std::min(n, 64u));
+}
+
+// job(0) .. job(n_jobs - 1), handed out by a counter to the caller and up to threads - 1 helpers.
+// Jobs must not throw; if helpers cannot be started the caller does all the work.
+template <class F>
+void parallel_jobs(size_t n_jobs, unsigned threads, F&& job) {
+  std::atomic<size_t> next{0};
+  auto worker = [&] {
+    for (size_t j; (j = next.fetch_add(1)) < n_jobs;) job(j);
+  };
+  std::vector<std::thread> pool;
+  if (threads > 1 && n_jobs > 1) {
+    try {
+      pool.reserve(threads - 1);
+      for (unsigned t = 1; t < threads && t < n_jobs; ++t) pool.emplace_back(worker);
+    } catch (...) {
+    }
+  }
+  worker();
+  for (std::thread& t : pool) t.join();
+}
+
+}  // namespace
+
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
                     const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
@@ -429,14 +463,13 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
   wanted.reserve(n_dst);
   for (size_t i = 0; i < n_dst; ++i)
     if (dst[i].fqn) wanted.emplace(dst[i].fqn);
-  std::vector<RelBox> scratch;
+  std::vector<int64_t> src_count(n_src), dst_count(n_dst);  // elements of every input entry
   for (size_t i = 0; i < n_src; ++i) {
-    int64_t n;
     uint32_t f;
-    if (int rc = check_meta(src[i], "src", i, src_buf_bytes, n_src_bufs, &n)) return rc;
+    if (int rc = check_meta(src[i], "src", i, src_buf_bytes, n_src_bufs, &src_count[i])) return rc;
     if (!wanted.count(src[i].fqn)) continue;
     if (int rc = family_of(src[i], "src", i, false, &f)) return rc;
-    expand(src[i], uint32_t(i), n, &fams[f].src, &scratch);
+    fams[f].src_metas.push_back(uint32_t(i));
   }
   // target byte ranges must not overlap inside a buffer
   {
@@ -447,11 +480,11 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
     std::vector<Range> rs;
     rs.reserve(n_dst);
     for (size_t i = 0; i < n_dst; ++i) {
-      int64_t n;
       uint32_t f;
-      if (int rc = check_meta(dst[i], "dst", i, dst_buf_bytes, n_dst_bufs, &n)) return rc;
+      if (int rc = check_meta(dst[i], "dst", i, dst_buf_bytes, n_dst_bufs, &dst_count[i])) return rc;
       if (int rc = family_of(dst[i], "dst", i, true, &f)) return rc;
-      expand(dst[i], uint32_t(i), n, &fams[f].dst, &scratch);
+      fams[f].dst_metas.push_back(uint32_t(i));
+      const int64_t n = dst_count[i];
       if (n > 0) rs.push_back(Range{dst[i].byte_offset, dst[i].byte_offset + dst[i].byte_length, dst[i].buf_index, uint32_t(i)});
     }
     std::sort(rs.begin(), rs.end(), [](const Range& a, const Range& b) { return a.buf != b.buf ? a.buf < b.buf : a.lo < b.lo; });
@@ -471,14 +504,23 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       }
     }
   }
-  std::vector<SegKey> segs;      // matched segments of the family at hand
-  std::vector<int64_t> reach;    // reach[i] = largest end (along dim 0) among the family's saved boxes 0..i
-  uint64_t n_inter = 0, n_se = 0, n_de = 0, uniq = 0;
-  for (uint32_t fi = 0; fi < fams.size(); ++fi) {
-    Family& f = fams[fi];
-    n_se += f.src.size();
-    n_de += f.dst.size();
+  struct Scratch {
+    std::vector<SegKey> segs;    // matched segments of the family at hand
+    std::vector<int64_t> reach;  // reach[i] = largest end (along dim 0) among the family's saved boxes 0..i
+    std::vector<RelBox> boxes;   // decomposition of one flat slice
+    uint64_t n_se = 0, n_de = 0; // boxes after decomposition
+  };
+  // One tensor: check its saved boxes, match every wanted box, lower the matches.  Families are
+  // independent, so large jobs hand blocks of them to several threads.
+  auto match_family = [&](Family& f, Scratch& sc, std::vector<Item>* items, uint64_t* n_inter_out, uint64_t* uniq_out) -> int {
+    std::vector<SegKey>& segs = sc.segs;
+    std::vector<int64_t>& reach = sc.reach;
+    uint64_t n_inter = 0, uniq = 0;
     const uint32_t nd = f.ndim;
+    for (uint32_t i : f.src_metas) expand(src[i], i, src_count[i], &f.src, &sc.boxes);
+    for (uint32_t i : f.dst_metas) expand(dst[i], i, dst_count[i], &f.dst, &sc.boxes);
+    sc.n_se += f.src.size();
+    sc.n_de += f.dst.size();
     if (allow_replicas && f.src.size() > 1) {
       // identical boxes are replicas of one shard: keep the one that came first in the input
       std::sort(f.src.begin(), f.src.end(), [nd](const Entry& a, const Entry& b) {
@@ -548,6 +590,68 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
     std::sort(segs.begin(), segs.end());
     segs.erase(std::unique(segs.begin(), segs.end()), segs.end());
     for (const SegKey& k : segs) uniq += k.bytes;
+    *n_inter_out += n_inter;
+    *uniq_out += uniq;
+    return BCP_OK;
+  };
+  uint64_t n_inter = 0, uniq = 0, n_se = 0, n_de = 0;
+  const unsigned threads = plan_threads(n_src + n_dst);
+  if (threads == 1) {
+    Scratch sc;
+    for (Family& f : fams)
+      if (int rc = match_family(f, sc, items, &n_inter, &uniq)) return rc;
+    n_se = sc.n_se, n_de = sc.n_de;
+  } else {
+    // blocks of consecutive families with about the same number of entries; a block stops at its
+    // first error, and the error of the earliest family wins, as in the serial order
+    struct Block {
+      size_t begin, end;
+      std::vector<Item> items;
+      uint64_t n_inter = 0, uniq = 0, n_se = 0, n_de = 0;
+      int rc = BCP_OK;
+      std::string err;
+    };
+    std::vector<Block> blocks;
+    const uint64_t per_block = uint64_t(n_src + n_dst) / (uint64_t(threads) * 8) + 1;
+    uint64_t acc = 0;
+    size_t begin = 0;
+    for (size_t fi = 0; fi < fams.size(); ++fi) {
+      acc += fams[fi].src_metas.size() + fams[fi].dst_metas.size();
+      if (acc >= per_block || fi + 1 == fams.size()) {
+        Block b;
+        b.begin = begin, b.end = fi + 1;
+        blocks.push_back(std::move(b));
+        begin = fi + 1, acc = 0;
+      }
+    }
+    parallel_jobs(blocks.size(), threads, [&](size_t j) {
+      Block& b = blocks[j];
+      try {
+        Scratch sc;
+        for (size_t fi = b.begin; fi < b.end && b.rc == BCP_OK; ++fi) {
+          b.rc = match_family(fams[fi], sc, &b.items, &b.n_inter, &b.uniq);
+          if (b.rc) b.err = last_error();  // the message lives in this thread
+        }
+        b.n_se = sc.n_se, b.n_de = sc.n_de;
+      } catch (const std::bad_alloc&) {
+        b.rc = BCP_ERR_NOMEM, b.err = "out of host memory";
+      }
+    });
+    for (const Block& b : blocks)  // blocks are in family order
+      if (b.rc) {
+        last_error() = b.err;
+        return b.rc;
+      }
+    size_t total = items->size();
+    for (const Block& b : blocks) total += b.items.size();
+    items->reserve(total);
+    for (Block& b : blocks) {
+      items->insert(items->end(), b.items.begin(), b.items.end());
+      n_inter += b.n_inter;
+      uniq += b.uniq;
+      n_se += b.n_se;
+      n_de += b.n_de;
+    }
   }
   stats->n_src_entries = n_se;
   stats->n_dst_entries = n_de;
@@ -564,35 +668,6 @@ inline uint32_t gran_log2(uint64_t bits) {
   uint32_t g = 0;
   while (g < 4 && !((bits >> g) & 1)) ++g;
   return g;  // 0..4 -> 1..16 bytes
-}
-
-// Host threads for large work lists.  The result never depends on the count.
-unsigned plan_threads(size_t n_units) {
-  if (n_units < 32768) return 1;
-  unsigned n = 0;
-  if (const char* e = getenv("BCP_PLAN_THREADS")) n = unsigned(strtoul(e, nullptr, 10));
-  if (!n) n = std::min(8u, std::thread::hardware_concurrency());
-  return std::max(1u, std::min(n, 64u));
-}
-
-// job(0) .. job(n_jobs - 1), handed out by a counter to the caller and up to threads - 1 helpers.
-// Jobs must not throw; if helpers cannot be started the caller does all the work.
-template <class F>
-void parallel_jobs(size_t n_jobs, unsigned threads, F&& job) {
-  std::atomic<size_t> next{0};
-  auto worker = [&] {
-    for (size_t j; (j = next.fetch_add(1)) < n_jobs;) job(j);
-  };
-  std::vector<std::thread> pool;
-  if (threads > 1 && n_jobs > 1) {
-    try {
-      pool.reserve(threads - 1);
-      for (unsigned t = 1; t < threads && t < n_jobs; ++t) pool.emplace_back(worker);
-    } catch (...) {
-    }
-  }
-  worker();
-  for (std::thread& t : pool) t.join();
 }
 
 enum { kTma = 0, kBig = 1, kSmall = 2, kCvt = 3, kClasses = 4 };  // unit classes, in the order of the final list
@@ -856,23 +931,24 @@ inline bool key_less(const Key& x, const Key& y) {
 // Merge sort over `threads` chunks; returns whichever of the two arrays holds the result.
 // Every merge of two runs is itself split into parts (cut one run evenly, find the matching
 // cut of the other by binary search), so that all rounds keep every thread busy.
-Key* sort_keys(Key* k, Key* tmp, size_t n, unsigned threads) {
+template <class T, class Less>
+T* parallel_sort(T* k, T* tmp, size_t n, unsigned threads, Less less) {
   const size_t chunks = std::max<size_t>(1, std::min<size_t>(threads, n / 8192));
   auto bound = [&](size_t i) { return n * std::min(i, chunks) / chunks; };
-  parallel_jobs(chunks, threads, [&](size_t c) { std::sort(k + bound(c), k + bound(c + 1), key_less); });
-  Key *from = k, *to = tmp;
+  parallel_jobs(chunks, threads, [&](size_t c) { std::sort(k + bound(c), k + bound(c + 1), less); });
+  T *from = k, *to = tmp;
   for (size_t w = 1; w < chunks; w *= 2) {
     const size_t pairs = (chunks + 2 * w - 1) / (2 * w);
     const size_t parts = std::max<size_t>(1, (threads + pairs - 1) / pairs);
     parallel_jobs(pairs * parts, threads, [&](size_t job) {
       const size_t j = job / parts, part = job % parts;
       const size_t lo = bound(2 * j * w), mid = bound(2 * j * w + w), hi = bound(2 * j * w + 2 * w);
-      const Key *a = from + lo, *b = from + mid;
+      const T *a = from + lo, *b = from + mid;
       const size_t na = mid - lo, nb = hi - mid;
-      auto cut_b = [&](size_t ia) { return ia >= na ? nb : size_t(std::lower_bound(b, b + nb, a[ia], key_less) - b); };
+      auto cut_b = [&](size_t ia) { return ia >= na ? nb : size_t(std::lower_bound(b, b + nb, a[ia], less) - b); };
       const size_t a0 = na * part / parts, a1 = na * (part + 1) / parts;
       const size_t b0 = part == 0 ? 0 : cut_b(a0), b1 = part + 1 == parts ? nb : cut_b(a1);
-      std::merge(a + a0, a + a1, b + b0, b + b1, to + lo + a0 + b0, key_less);
+      std::merge(a + a0, a + a1, b + b0, b + b1, to + lo + a0 + b0, less);
     });
     std::swap(from, to);
   }
@@ -884,12 +960,19 @@ Key* sort_keys(Key* k, Key* tmp, size_t n, unsigned threads) {
 void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint64_t>* src_bytes, TileVec* tiles,
                  size_t* n_tma, size_t* n_big, size_t* n_cvt, std::vector<Rect>* rects, bcp_plan_stats_t* stats) {
   // coalesce runs that are adjacent on both sides (e.g. the sub-boxes of one flat slice)
-  std::sort(items.begin(), items.end(), [](const Item& a, const Item& b) {
-    return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off;
-  });
+  auto by_target = [](const Item& a, const Item& b) { return a.dst_buf != b.dst_buf ? a.dst_buf < b.dst_buf : a.dst_off < b.dst_off; };
+  const Item* sorted_items = items.data();
+  std::vector<Item> item_tmp;
+  if (const unsigned st = plan_threads(items.size()); st > 1) {
+    item_tmp.resize(items.size());
+    sorted_items = parallel_sort(items.data(), item_tmp.data(), items.size(), st, by_target);
+  } else {
+    std::sort(items.begin(), items.end(), by_target);
+  }
   std::vector<Item> merged;
   merged.reserve(items.size());
-  for (const Item& it : items) {
+  for (size_t ii = 0; ii < items.size(); ++ii) {
+    const Item& it = sorted_items[ii];
     if (it.rows * it.row_bytes == 0) continue;
     if (!merged.empty()) {
       Item& p = merged.back();
@@ -1005,7 +1088,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   size_t base = 0;
   for (int k = 0; k < kClasses; ++k) {
     const size_t n = run.n[k];
-    const Key* sorted = sort_keys(keys.get() + base, spare.get() + base, n, threads);
+    const Key* sorted = parallel_sort(keys.get() + base, spare.get() + base, n, threads, key_less);
     bcp_tile* dst = tiles->data() + base;
     const bcp_tile* src = cls[k];
     parallel_jobs((n + kChunk - 1) / kChunk, threads, [&](size_t j) {

@@ -354,6 +354,32 @@ def test_work_list_does_not_depend_on_the_number_of_planner_threads(opts, monkey
     assert images[0] == images[1] == images[2]
 
 
+def test_matching_does_not_depend_on_the_number_of_planner_threads(monkeypatch):
+    """Above 32k input entries tensors are expanded and matched by several threads; the plan, its
+    statistics and the error that is reported (the earliest tensor's, as in serial order) stay the same."""
+    import copy
+
+    from workloads.configs import OPTIM_ONLY
+    from workloads.layouts import Parallelism, llama_model, reshard_case
+
+    m = llama_model("llama-3b-fsdp", L=28, H=3072, nq=24, nkv=8, F=8192, V=128256, fused=False, tied=True, fsdp_units=True)
+    case = reshard_case("dp256-to-dp192", m, Parallelism(dp=256, zero="fsdp"), Parallelism(dp=192, zero="fsdp"), OPTIM_ONLY)
+    assert len(case.src.metas) + len(case.dst.metas) > 32768
+    twice = list(case.src.metas) + [copy.copy(case.src.metas[len(case.src.metas) // 2]), copy.copy(case.src.metas[len(case.src.metas) // 5])]
+    images, errors = [], []
+    for threads in ("1", "8", "3"):
+        monkeypatch.setenv("BCP_PLAN_THREADS", threads)
+        plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+        images.append(_image_without_clock(plan))
+        plan.destroy()
+        with pytest.raises(bcp.BcpError) as e:  # two tensors hold an element twice
+            bcp.bcp_plan(twice, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+        assert e.value.code == api.ERR_OVERLAP
+        errors.append(str(e.value))
+    assert images[0] == images[1] == images[2]
+    assert errors[0] == errors[1] == errors[2]
+
+
 def test_plan_image_is_verified():
     case = scenario_cases()[0]
     plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
