@@ -1,61 +1,14 @@
 // C ABI of the resharding engine: plan objects, execution, pack / unpack.
+// (Plan images are in plan_image.cu, the host-buffer call in host_path.cu.)
 #include <chrono>
-#include <cstring>
 #include <mutex>
 #include <new>
-#include <vector>
 
-#include <cuda.h>
-
-#include "kernels.cuh"
-#include "plan.hpp"
+#include "plan_object.hpp"
 
 using namespace bcp;
 
-struct bcp_plan_s {
-  Options opt;
-  bcp_plan_stats_t stats;
-  TileVec tiles;  // TMA units, then other CTA-wide units, then warp units, then converting units
-  size_t n_tma = 0, n_big = 0, n_cvt = 0;
-  size_t n_small() const { return tiles.size() - n_tma - n_big - n_cvt; }
-  std::vector<uint64_t> src_bytes, dst_bytes;
-  std::vector<Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
-  std::vector<Gap> gaps;    // target bytes no entry names (zeroed by the host-buffer call)
-  std::vector<CUtensorMap> h_maps;
-  CUtensorMap* d_maps = nullptr;
-  // device side, created by the first execution
-  int device = -1;
-  bcp_tile* d_tiles = nullptr;
-  bcp_tile* d_fan_tiles = nullptr;  // the same list with replica groups marked (in-place host path)
-  void** d_ptrs = nullptr;  // source table followed by target table
-  Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel, [2] converting kernel
-  uint32_t grid = 0, tma_grid = 0, cvt_grid = 0;
-  cudaStream_t last_stream = nullptr;
-  cudaEvent_t ev_switch = nullptr;  // orders an execution after the previous one when the stream changes
-  bool ran = false;
-  std::vector<void*> h_ptrs;
-  bool table_current = false;  // the device pointer table already holds h_ptrs
-  // bcp_reshard_host: device staging plus a second copy of the work list grouped by target
-  // buffer, so that uploads, kernels and downloads of different target buffers overlap
-  struct Group {  // units of one target buffer inside d_host_tiles
-    size_t first = 0, n_tma = 0, n_big = 0, n_small = 0, n_cvt = 0;
-    std::vector<uint32_t> needs;  // source buffers its units read
-  };
-  std::vector<void*> stage_src, stage_dst;
-  bcp_tile* d_host_tiles = nullptr;
-  std::vector<Group> groups;     // one per target buffer
-  std::vector<uint32_t> order;   // target buffers in processing order
-  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
-  std::vector<cudaEvent_t> ev_src, ev_dst;
-};
-
-namespace {
-
-#define BCP_CUDA(call)                                                                       \
-  do {                                                                                       \
-    cudaError_t e_ = (call);                                                                 \
-    if (e_ != cudaSuccess) return fail(BCP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
-  } while (0)
+namespace bcp {
 
 int bind_device_alloc(bcp_plan_t* p) {
   const size_t n_ptrs = p->src_bytes.size() + p->dst_bytes.size();
@@ -213,7 +166,7 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
 }
 
 int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, size_t nd, cudaStream_t stream,
-            const bcp_tile* list = nullptr) {
+            const bcp_tile* list) {
   if (!p) return fail(BCP_ERR_INVALID, "plan is NULL");
   if (ns != p->src_bytes.size() || nd != p->dst_bytes.size())
     return fail(BCP_ERR_INVALID, "buffer counts (%zu, %zu) differ from the planned (%zu, %zu)", ns, nd, p->src_bytes.size(),
@@ -262,6 +215,10 @@ int execute(bcp_plan_t* p, const void* const* src, size_t ns, void* const* dst, 
   p->ran = true;
   return BCP_OK;
 }
+
+}  // namespace bcp
+
+namespace {
 
 bcp_plan_t* finish_plan(std::vector<Item>& items, const Options& opt, bcp_plan_stats_t stats,
                       std::vector<uint64_t> src_bytes, std::vector<uint64_t> dst_bytes) {
@@ -378,74 +335,6 @@ int pack_plan(bool unpack, const bcp_pack_meta* metas, size_t n, uint64_t blob_b
   return BCP_OK;
 }
 
-// One-time set-up of the host-buffer path: staging buffers, streams, events, and the work list
-// regrouped by target buffer.
-int prepare_host_path(bcp_plan_t* p) {
-  if (p->s_h2d) return BCP_OK;
-  const size_t ns = p->src_bytes.size(), nd = p->dst_bytes.size();
-  p->groups.assign(nd, bcp_plan_s::Group());
-  std::vector<std::vector<bcp_tile>> tma(nd), big(nd), small(nd), cvt(nd);
-  std::vector<std::vector<char>> need(nd, std::vector<char>(ns, 0));
-  for (const bcp_tile& t : p->tiles) {
-    const uint32_t d = t.dst_buf;
-    if (!(t.flags & BCP_TILE_ZERO)) need[d][t.src_buf] = 1;
-    bcp_tile u = t;
-    u.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));  // groups are per target buffer here: every unit is staged on its own
-    ((u.flags & BCP_TILE_CVT_MASK) ? cvt : (u.flags & BCP_TILE_TMA) ? tma : (u.flags & BCP_TILE_SMALL) ? small : big)[d].push_back(u);
-  }
-  std::vector<bcp_tile> flat;
-  flat.reserve(p->tiles.size());
-  for (size_t d = 0; d < nd; ++d) {
-    bcp_plan_s::Group& g = p->groups[d];
-    g.first = flat.size();
-    g.n_tma = tma[d].size();
-    g.n_big = big[d].size();
-    g.n_small = small[d].size();
-    g.n_cvt = cvt[d].size();
-    flat.insert(flat.end(), tma[d].begin(), tma[d].end());
-    flat.insert(flat.end(), big[d].begin(), big[d].end());
-    flat.insert(flat.end(), small[d].begin(), small[d].end());
-    flat.insert(flat.end(), cvt[d].begin(), cvt[d].end());
-    for (uint32_t sb = 0; sb < ns; ++sb)
-      if (need[d][sb]) g.needs.push_back(sb);
-  }
-  // order: always take the target buffer that needs the fewest bytes not yet uploaded, so that
-  // the first download starts early and uploads keep running under the downloads
-  std::vector<char> have(ns, 0), done(nd, 0);
-  for (size_t k = 0; k < nd; ++k) {
-    size_t best = nd;
-    uint64_t best_cost = ~uint64_t(0);
-    for (size_t d = 0; d < nd; ++d) {
-      if (done[d]) continue;
-      uint64_t cost = 0;
-      for (uint32_t sb : p->groups[d].needs)
-        if (!have[sb]) cost += p->src_bytes[sb];
-      if (cost < best_cost) {
-        best_cost = cost;
-        best = d;
-      }
-    }
-    done[best] = 1;
-    for (uint32_t sb : p->groups[best].needs) have[sb] = 1;
-    p->order.push_back(uint32_t(best));
-  }
-  if (!flat.empty()) {
-    BCP_CUDA(cudaMalloc(&p->d_host_tiles, flat.size() * sizeof(bcp_tile)));
-    BCP_CUDA(cudaMemcpy(p->d_host_tiles, flat.data(), flat.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
-  }
-  p->stage_src.assign(ns, nullptr);
-  p->stage_dst.assign(nd, nullptr);
-  for (size_t i = 0; i < ns; ++i) BCP_CUDA(cudaMalloc(&p->stage_src[i], p->src_bytes[i] ? p->src_bytes[i] : 16));
-  for (size_t i = 0; i < nd; ++i) BCP_CUDA(cudaMalloc(&p->stage_dst[i], p->dst_bytes[i] ? p->dst_bytes[i] : 16));
-  p->ev_src.assign(ns, nullptr);
-  p->ev_dst.assign(nd ? nd : 1, nullptr);
-  for (cudaEvent_t& e : p->ev_src) BCP_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-  for (cudaEvent_t& e : p->ev_dst) BCP_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-  BCP_CUDA(cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking));
-  BCP_CUDA(cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking));  // set last: marks the path as ready
-  return BCP_OK;
-}
-
 // address -> (address rounded down to 16 bytes, remainder)
 void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vector<uint8_t>* res,
                       std::vector<const void*>* bases) {
@@ -551,214 +440,6 @@ int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out) {
   return BCP_OK;
 }
 
-namespace {
-const char kMagic[8] = {'B', 'C', 'P', 'P', 'L', 'A', 'N', '1'};
-struct ImageHeader {
-  char magic[8];
-  uint32_t version, tile_size;
-  Options opt;
-  bcp_plan_stats_t stats;
-  uint64_t n_src_bufs, n_dst_bufs, n_tma, n_big, n_tiles, n_rects, n_gaps, n_cvt;
-};
-uint64_t fnv1a(const unsigned char* p, size_t n) {
-  uint64_t h = 1469598103934665603ull;
-  for (size_t i = 0; i < n; ++i) h = (h ^ p[i]) * 1099511628211ull;
-  return h;
-}
-// A unit is safe to execute if it stays inside its buffers and its flags match its geometry.
-bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db, const std::vector<Rect>& rects,
-             const Options& opt) {
-  if (t.rows == 0 || t.row_bytes == 0 || t.dst_buf >= db.size()) return false;
-  if (const uint32_t kind = (t.flags & BCP_TILE_CVT_MASK) >> BCP_TILE_CVT_SHIFT) {
-    // converting unit: element-aligned on both sides, source rows hold the same number of elements
-    if (kind > BCP_CONVERT_BF16_TO_F32 || (t.flags & ~(BCP_TILE_GRAN_MASK | BCP_TILE_CVT_MASK)) || t.src_buf >= sb.size()) return false;
-    const uint64_t s_isz = kind == BCP_CONVERT_F32_TO_BF16 ? 4 : 2, d_isz = 6 - s_isz;
-    const uint64_t s_row = uint64_t(t.row_bytes) / d_isz * s_isz;
-    if (t.row_bytes % d_isz || t.dst_off % d_isz || t.dst_pitch % d_isz || t.src_off % s_isz || t.src_pitch % s_isz) return false;
-    if (t.rows > 1 && (t.dst_pitch < t.row_bytes || t.src_pitch < s_row)) return false;
-    const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes, span_s = uint64_t(t.rows - 1) * t.src_pitch + s_row;
-    if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
-    if (t.src_off > sb[t.src_buf] || span_s > sb[t.src_buf] - t.src_off) return false;
-    return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
-  }
-  const bool zero = t.flags & BCP_TILE_ZERO;
-  const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes;
-  if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
-  if (t.rows > 1 && t.dst_pitch < t.row_bytes) return false;
-  uint64_t bits = t.dst_off | t.row_bytes | t.dst_pitch;
-  if (!zero) {
-    if (t.src_buf >= sb.size()) return false;
-    const uint64_t span_s = uint64_t(t.rows - 1) * t.src_pitch + t.row_bytes;
-    if (t.src_off > sb[t.src_buf] || span_s > sb[t.src_buf] - t.src_off) return false;
-    bits |= t.src_off | t.src_pitch;
-  }
-  uint32_t g = 0;
-  while (g < 4 && !((bits >> g) & 1)) ++g;
-  if ((t.flags & BCP_TILE_GRAN_MASK) > g) return false;  // a wider access than the offsets allow would fault
-  if (t.flags & BCP_TILE_TMA2D) {  // must be a whole number of boxes of the rectangle it names
-    if (!(t.flags & BCP_TILE_TMA) || zero || g < 4 || t.reserved[0] == 0 || t.reserved[0] > rects.size()) return false;
-    const Rect& r = rects[t.reserved[0] - 1];
-    const uint64_t row0 = t.reserved[1];
-    if (t.reserved[2] != r.box_rows || r.box_rows == 0 || row0 % r.box_rows || row0 + t.rows > r.rows) return false;
-    if (t.rows % r.box_rows && row0 + t.rows != r.rows) return false;
-    if (t.src_buf != r.src_buf || t.dst_buf != r.dst_buf || t.row_bytes != r.row_bytes || t.src_pitch != r.src_pitch ||
-        t.dst_pitch != r.dst_pitch || t.src_off != r.src_off + row0 * r.src_pitch || t.dst_off != r.dst_off + row0 * r.dst_pitch)
-      return false;
-    if (uint64_t(r.box_rows) * r.row_bytes > opt.tma_stage_bytes) return false;
-    return uint64_t(t.rows) * t.row_bytes <= std::max<uint64_t>(opt.tile_bytes, uint64_t(r.box_rows) * r.row_bytes);
-  }
-  if (t.flags & BCP_TILE_TMA) {
-    if (zero || t.row_bytes < 16) return false;
-    if (g < 4) {  // shifted run or rectangle: the aligned superset of the last row stays inside the source buffer
-      if (((t.src_off + uint64_t(t.rows - 1) * t.src_pitch + t.row_bytes + 15) & ~uint64_t(15)) > sb[t.src_buf]) return false;
-    }
-  }
-  return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
-}
-// A rectangle's two views must stay inside their buffers and satisfy the tensor-map rules.
-bool rect_ok(const Rect& r, const std::vector<uint64_t>& sb, const std::vector<uint64_t>& db) {
-  if (r.src_buf >= sb.size() || r.dst_buf >= db.size() || r.rows == 0 || r.rows >= (uint64_t(1) << 31)) return false;
-  if (r.row_bytes < 16 || r.row_bytes > 2048 || r.box_rows == 0 || r.box_rows > 256) return false;
-  if ((r.src_off | r.dst_off | r.row_bytes | r.src_pitch | r.dst_pitch) & 15) return false;
-  if (r.src_pitch < r.row_bytes || r.dst_pitch < r.row_bytes || r.src_pitch >= (uint64_t(1) << 40) || r.dst_pitch >= (uint64_t(1) << 40))
-    return false;
-  const uint64_t ss = (r.rows - 1) * r.src_pitch + r.row_bytes, ds = (r.rows - 1) * r.dst_pitch + r.row_bytes;
-  return r.src_off <= sb[r.src_buf] && ss <= sb[r.src_buf] - r.src_off && r.dst_off <= db[r.dst_buf] && ds <= db[r.dst_buf] - r.dst_off;
-}
-}  // namespace
-
-int bcp_plan_serialize(const bcp_plan_t* plan, void* out, size_t cap, size_t* n) {
-  if (!plan || !n) return fail(BCP_ERR_INVALID, "bcp_plan_serialize: NULL argument");
-  const size_t need = sizeof(ImageHeader) + (plan->src_bytes.size() + plan->dst_bytes.size()) * sizeof(uint64_t) +
-                      plan->tiles.size() * sizeof(bcp_tile) + plan->rects.size() * sizeof(Rect) + plan->gaps.size() * sizeof(Gap) +
-                      sizeof(uint64_t);
-  *n = need;
-  if (!out || cap < need) return fail(BCP_ERR_CAPACITY, "bcp_plan_serialize: image needs %zu bytes, room for %zu", need, out ? cap : size_t(0));
-  ImageHeader h;
-  memset(static_cast<void*>(&h), 0, sizeof h);  // padding bytes too: images are compared and checksummed
-  memcpy(h.magic, kMagic, 8);
-  h.version = uint32_t(bcp_version());
-  h.tile_size = sizeof(bcp_tile);
-  h.opt = plan->opt;
-  h.stats = plan->stats;
-  h.n_src_bufs = plan->src_bytes.size();
-  h.n_dst_bufs = plan->dst_bytes.size();
-  h.n_tma = plan->n_tma;
-  h.n_big = plan->n_big;
-  h.n_cvt = plan->n_cvt;
-  h.n_tiles = plan->tiles.size();
-  h.n_rects = plan->rects.size();
-  h.n_gaps = plan->gaps.size();
-  unsigned char* p = static_cast<unsigned char*>(out);
-  memcpy(p, &h, sizeof h);
-  p += sizeof h;
-  if (h.n_src_bufs) memcpy(p, plan->src_bytes.data(), h.n_src_bufs * sizeof(uint64_t));
-  p += h.n_src_bufs * sizeof(uint64_t);
-  if (h.n_dst_bufs) memcpy(p, plan->dst_bytes.data(), h.n_dst_bufs * sizeof(uint64_t));
-  p += h.n_dst_bufs * sizeof(uint64_t);
-  if (h.n_tiles) memcpy(p, plan->tiles.data(), h.n_tiles * sizeof(bcp_tile));
-  p += h.n_tiles * sizeof(bcp_tile);
-  if (h.n_rects) memcpy(p, plan->rects.data(), h.n_rects * sizeof(Rect));
-  p += h.n_rects * sizeof(Rect);
-  if (h.n_gaps) memcpy(p, plan->gaps.data(), h.n_gaps * sizeof(Gap));
-  p += h.n_gaps * sizeof(Gap);
-  const uint64_t sum = fnv1a(static_cast<unsigned char*>(out), size_t(p - static_cast<unsigned char*>(out)));
-  memcpy(p, &sum, sizeof sum);
-  return BCP_OK;
-}
-
-int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
-  if (!image || !out_plan) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: NULL argument");
-  if (n < sizeof(ImageHeader) + sizeof(uint64_t)) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image too short");
-  ImageHeader h;
-  memcpy(&h, image, sizeof h);
-  if (memcmp(h.magic, kMagic, 8) != 0) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: not a plan image");
-  if (h.version != uint32_t(bcp_version()) || h.tile_size != sizeof(bcp_tile))
-    return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image of library version %u, this is %d", h.version, bcp_version());
-  const uint64_t lim = uint64_t(1) << 32;
-  if (h.n_src_bufs >= lim || h.n_dst_bufs >= lim || h.n_tiles >= lim || h.n_rects >= lim || h.n_gaps >= lim || h.n_tma > h.n_tiles ||
-      h.n_big > h.n_tiles - h.n_tma || h.n_cvt > h.n_tiles - h.n_tma - h.n_big)
-    return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: implausible counts");
-  const uint64_t need = sizeof(ImageHeader) + (h.n_src_bufs + h.n_dst_bufs) * sizeof(uint64_t) + h.n_tiles * sizeof(bcp_tile) +
-                        h.n_rects * sizeof(Rect) + h.n_gaps * sizeof(Gap) + sizeof(uint64_t);
-  if (need != n) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: image is %zu bytes, its header implies %llu", n, (unsigned long long)need);
-  const unsigned char* base = static_cast<const unsigned char*>(image);
-  uint64_t sum;
-  memcpy(&sum, base + n - sizeof sum, sizeof sum);
-  if (sum != fnv1a(base, n - sizeof sum)) return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: checksum mismatch");
-  {  // the options were validated when the plan was made; re-check what the launch code relies on
-    const Options& o = h.opt;
-    if ((o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024) || o.ctas_per_sm < 1 || o.ctas_per_sm > 16 ||
-        o.tile_bytes < 4096 || o.tile_bytes > (64u << 20) || (o.unroll != 4 && o.unroll != 8) || (o.worker != 1 && o.worker != 2) || o.tma_stages < 2 || o.tma_stages > 8 ||
-        o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536 ||
-        uint64_t(o.tma_stage_bytes) * o.tma_stages > 200 * 1024 || o.tma_ctas_per_sm < 1 || o.tma_ctas_per_sm > 16 || o.cache_hints < 1 ||
-        o.cache_hints > 4)
-      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: options out of range");
-  }
-  bcp_plan_t* p = new (std::nothrow) bcp_plan_t;
-  if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
-  try {
-    const unsigned char* q = base + sizeof h;
-    p->opt = h.opt;
-    p->stats = h.stats;
-    p->src_bytes.resize(h.n_src_bufs);
-    p->dst_bytes.resize(h.n_dst_bufs);
-    p->tiles.resize(h.n_tiles);
-    if (h.n_src_bufs) memcpy(p->src_bytes.data(), q, h.n_src_bufs * sizeof(uint64_t));
-    q += h.n_src_bufs * sizeof(uint64_t);
-    if (h.n_dst_bufs) memcpy(p->dst_bytes.data(), q, h.n_dst_bufs * sizeof(uint64_t));
-    q += h.n_dst_bufs * sizeof(uint64_t);
-    if (h.n_tiles) memcpy(p->tiles.data(), q, h.n_tiles * sizeof(bcp_tile));
-    q += h.n_tiles * sizeof(bcp_tile);
-    p->rects.resize(h.n_rects);
-    if (h.n_rects) memcpy(p->rects.data(), q, h.n_rects * sizeof(Rect));
-    q += h.n_rects * sizeof(Rect);
-    p->gaps.resize(h.n_gaps);
-    if (h.n_gaps) memcpy(p->gaps.data(), q, h.n_gaps * sizeof(Gap));
-    p->n_tma = h.n_tma;
-    p->n_big = h.n_big;
-    p->n_cvt = h.n_cvt;
-  } catch (const std::bad_alloc&) {
-    delete p;
-    return fail(BCP_ERR_NOMEM, "out of host memory");
-  }
-  for (const Gap& g : p->gaps) {  // gaps are zeroed in host memory: they must stay inside their buffer
-    if (g.buf >= p->dst_bytes.size() || g.off > p->dst_bytes[g.buf] || g.len > p->dst_bytes[g.buf] - g.off) {
-      delete p;
-      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: a gap lies outside its target buffer");
-    }
-  }
-  for (size_t i = 0; i < p->rects.size(); ++i) {
-    if (!rect_ok(p->rects[i], p->src_bytes, p->dst_bytes)) {
-      delete p;
-      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: rectangle %zu is inconsistent with the recorded buffers", i);
-    }
-  }
-  {  // replica groups must be exactly what the planner would mark: a follower is never staged itself
-    std::vector<bcp_tile> again(p->tiles.begin(), p->tiles.begin() + p->n_tma);
-    for (bcp_tile& t : again) t.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));
-    if (p->opt.fanout == 1 && p->opt.order == 1) mark_followers(again.data(), again.size());
-    bool ok = true;
-    for (size_t i = 0; ok && i < p->tiles.size(); ++i)
-      ok = i < p->n_tma ? again[i].flags == p->tiles[i].flags : !(p->tiles[i].flags & (BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT)));
-    if (!ok) {
-      delete p;
-      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: replica groups of the work list are inconsistent");
-    }
-  }
-  for (size_t i = 0; i < p->tiles.size(); ++i) {
-    const bcp_tile& t = p->tiles[i];
-    const bool in_tma = i < p->n_tma, in_cvt = i >= p->tiles.size() - p->n_cvt, in_small = i >= p->n_tma + p->n_big && !in_cvt;
-    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->rects, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
-        bool(t.flags & BCP_TILE_SMALL) != in_small || bool(t.flags & BCP_TILE_CVT_MASK) != in_cvt) {
-      delete p;
-      return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: work unit %zu is inconsistent with the recorded buffers", i);
-    }
-  }
-  *out_plan = p;
-  return BCP_OK;
-}
-
 int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n) {
   if (!plan || !n || (cap && !out)) return fail(BCP_ERR_INVALID, "bcp_plan_tiles: NULL argument");
   *n = plan->tiles.size();
@@ -770,91 +451,6 @@ int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n)
 int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n_src_bufs, void* const* dst_bufs,
                 size_t n_dst_bufs, void* stream) {
   return execute(plan, src_blobs, n_src_bufs, dst_bufs, n_dst_bufs, static_cast<cudaStream_t>(stream));
-}
-
-int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src_bufs, void* const* dst_host,
-                     size_t n_dst_bufs, void* stream_) {
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
-  if (n_src_bufs != plan->src_bytes.size() || n_dst_bufs != plan->dst_bytes.size())
-    return fail(BCP_ERR_INVALID, "buffer counts differ from the planned ones");
-  if ((n_src_bufs && !src_host) || (n_dst_bufs && !dst_host)) return fail(BCP_ERR_INVALID, "pointer array is NULL");
-  for (size_t i = 0; i < n_src_bufs; ++i)
-    if (plan->src_bytes[i] && !src_host[i]) return fail(BCP_ERR_INVALID, "source buffer %zu is NULL", i);
-  for (size_t i = 0; i < n_dst_bufs; ++i)
-    if (plan->dst_bytes[i] && !dst_host[i]) return fail(BCP_ERR_INVALID, "target buffer %zu is NULL", i);
-  if (int rc = bind_device(plan)) return rc;
-  bcp_plan_t* p = plan;
-  // Pinned (or registered) host memory is addressable from the device: then the kernels read the
-  // sources and write the targets in place, over PCIe in both directions at once, and no staging
-  // copy exists at all.  Anything else goes through device staging buffers.
-  {
-    std::vector<const void*> dsrc(n_src_bufs, nullptr);
-    std::vector<void*> ddst(n_dst_bufs, nullptr);
-    bool mapped = true;
-    auto device_view = [&](const void* host, void** out) {
-      cudaPointerAttributes a;
-      if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-      }
-      if (a.type != cudaMemoryTypeHost || !a.devicePointer || (reinterpret_cast<uintptr_t>(a.devicePointer) & 15)) return false;
-      *out = a.devicePointer;
-      return true;
-    };
-    for (size_t i = 0; mapped && i < n_src_bufs; ++i)
-      if (p->src_bytes[i]) mapped = device_view(src_host[i], const_cast<void**>(&dsrc[i]));
-    for (size_t i = 0; mapped && i < n_dst_bufs; ++i)
-      if (p->dst_bytes[i]) mapped = device_view(dst_host[i], &ddst[i]);
-    if (mapped) {
-      // over PCIe every read costs: stage each source piece once and write all its replicas from it
-      if (!p->d_fan_tiles && p->n_tma && p->opt.order == 1 && p->opt.fanout != 1) {
-        std::vector<bcp_tile> fan(p->tiles.begin(), p->tiles.end());
-        mark_followers(fan.data(), p->n_tma);
-        BCP_CUDA(cudaMalloc(&p->d_fan_tiles, fan.size() * sizeof(bcp_tile)));
-        BCP_CUDA(cudaMemcpy(p->d_fan_tiles, fan.data(), fan.size() * sizeof(bcp_tile), cudaMemcpyHostToDevice));
-      }
-      for (const Gap& g : p->gaps) memset(static_cast<char*>(dst_host[g.buf]) + g.off, 0, g.len);
-      if (int rc = execute(p, dsrc.data(), n_src_bufs, ddst.data(), n_dst_bufs, stream, p->d_fan_tiles)) return rc;
-      BCP_CUDA(cudaStreamSynchronize(stream));
-      return BCP_OK;
-    }
-  }
-  if (int rc = prepare_host_path(plan)) return rc;
-  // device-side pointer table: the staging buffers
-  for (size_t i = 0; i < n_src_bufs; ++i) p->h_ptrs[i] = p->stage_src[i];
-  for (size_t i = 0; i < n_dst_bufs; ++i) p->h_ptrs[n_src_bufs + i] = p->stage_dst[i];
-  if (int rc = upload_tables(p, stream)) return rc;
-  p->table_current = false;  // the tables now name the staging buffers, not a caller's
-  // The upload stream starts after whatever the caller queued on `stream` before this call.
-  BCP_CUDA(cudaEventRecord(p->ev_dst[0], stream));
-  BCP_CUDA(cudaStreamWaitEvent(p->s_h2d, p->ev_dst[0], 0));
-  std::vector<char> uploaded(n_src_bufs, 0);
-  // Target buffers one after the other: upload the sources it still misses, run its units,
-  // download it.  Uploads, kernels and downloads sit on three streams, so the download of one
-  // target buffer overlaps the uploads for the next (PCIe is full duplex).
-  for (uint32_t d : p->order) {
-    const bcp_plan_s::Group& g = p->groups[d];
-    for (uint32_t sb : g.needs) {
-      if (uploaded[sb]) continue;
-      uploaded[sb] = 1;
-      BCP_CUDA(cudaMemcpyAsync(p->stage_src[sb], src_host[sb], p->src_bytes[sb], cudaMemcpyHostToDevice, p->s_h2d));
-      BCP_CUDA(cudaEventRecord(p->ev_src[sb], p->s_h2d));
-    }
-    if (!p->dst_bytes[d]) continue;
-    for (uint32_t sb : g.needs) BCP_CUDA(cudaStreamWaitEvent(stream, p->ev_src[sb], 0));
-    BCP_CUDA(cudaMemsetAsync(p->stage_dst[d], 0, p->dst_bytes[d], stream));
-    if (int rc = launch_units(p, p->d_host_tiles + g.first, g.n_tma, g.n_big, g.n_small, g.n_cvt, stream)) return rc;
-    BCP_CUDA(cudaEventRecord(p->ev_dst[d], stream));
-    BCP_CUDA(cudaStreamWaitEvent(p->s_d2h, p->ev_dst[d], 0));
-    BCP_CUDA(cudaMemcpyAsync(dst_host[d], p->stage_dst[d], p->dst_bytes[d], cudaMemcpyDeviceToHost, p->s_d2h));
-  }
-  p->last_stream = stream;
-  p->ran = true;
-  BCP_CUDA(cudaStreamSynchronize(p->s_h2d));
-  BCP_CUDA(cudaStreamSynchronize(stream));
-  BCP_CUDA(cudaStreamSynchronize(p->s_d2h));
-  return BCP_OK;
 }
 
 int bcp_plan_device_status(bcp_plan_t* plan, void* stream) {
