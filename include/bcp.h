@@ -17,8 +17,8 @@
  *     matching segments are copied into it (Sec. 3.3, Step 2 and Step 5).
  *
  * A "storage file" is a device buffer here (a blob); all source ranks and all target
- * ranks are separate buffers on ONE GPU.  No numeric conversion happens anywhere:
- * the engine moves raw bytes.
+ * ranks are separate buffers on ONE GPU.  The engine moves raw bytes unchanged, unless
+ * bcp_plan_opts.convert asks for a binary32 <-> bfloat16 conversion of some tensors.
  *
  * Conventions
  *   - Every function returns an int: BCP_OK (0) or a negative bcp_status.  A failing
@@ -474,7 +474,9 @@ BCP_API int bcp_stager_release(bcp_stager_t* stager, uint32_t slot);
  *     (the unit size grows up to 64 MiB to make a blob fit); beyond that the call returns
  *     BCP_ERR_CAPACITY and launches nothing: use bcp_pack.
  *   - the first call on each device looks up the device address of the fixed array, with
- *     that device current; make that first call before any stream capture begins.
+ *     that device current; make that first call before any stream capture begins.  A call
+ *     whose stream is being captured is refused with BCP_ERR_INVALID: its uploads come from a
+ *     host array that every call rewrites.
  *   - all calls share the one array per device.  Each call rewrites what it uses and clears the
  *     control words, so calls that run one after the other on the GPU (same stream, or
  *     otherwise ordered) are safe; two calls whose kernels may overlap on the GPU (different

@@ -59,14 +59,24 @@ int scratch_address(unsigned char** out) {
   return BCP_OK;
 }
 
+// The work list is produced in two passes over the same cutting rule: a counting pass (store ==
+// false) that only sizes the two groups, then a writing pass that puts CTA-wide units at
+// tiles[0, n_big) and warp units at tiles[small_base, small_base + n_small), each in emission
+// order.  No unit is ever moved inside the fixed array.
 struct UnitWriter {
-  uint32_t n_big = 0, n_small = 0;  // CTA-wide units fill tiles[] from the front, warp units from the back
+  uint32_t n_big = 0, n_small = 0;
+  uint32_t small_base = 0;  // writing pass: where the warp units start (= the counted n_big)
+  bool store = false;
   bool overflow = false;
 
   void emit(uint64_t src_off, uint64_t dst_off, uint64_t bytes, uint32_t src_buf, bool zero, uint32_t small_bytes) {
     if (bytes == 0) return;
     if (n_big + n_small >= kMaxUnits) {
       overflow = true;
+      return;
+    }
+    if (!store) {
+      if (bytes < small_bytes) ++n_small; else ++n_big;
       return;
     }
     bcp_tile t;
@@ -83,7 +93,7 @@ struct UnitWriter {
     t.flags = g | (zero ? BCP_TILE_ZERO : 0u);
     if (bytes < small_bytes) {
       t.flags |= BCP_TILE_SMALL;
-      g_host.tiles[kMaxUnits - 1 - n_small++] = t;
+      g_host.tiles[small_base + n_small++] = t;
     } else {
       g_host.tiles[n_big++] = t;
     }
@@ -129,6 +139,16 @@ extern "C" int bcp_pack_static(const void* const* tensors, const bcp_pack_meta* 
     if (metas[i].byte_length && !tensors[i]) return fail(BCP_ERR_INVALID, "bcp_pack_static: tensor %zu is NULL", i);
     pos = metas[i].byte_offset + metas[i].byte_length;
   }
+  // The uploads below read the shared host mirror when they execute.  Recorded by a stream
+  // capture they would read it again at every replay, after later calls have rewritten it, while
+  // the kernel node keeps this call's unit counts: refused rather than silently wrong.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(BCP_ERR_CUDA, "bcp_pack_static: cudaStreamIsCapturing failed");
+  }
+  if (capturing != cudaStreamCaptureStatusNone)
+    return fail(BCP_ERR_INVALID, "bcp_pack_static: the stream is being captured; its uploads come from a host array that every call rewrites");
   std::lock_guard<std::mutex> lock(g_mu);
   unsigned char* dev = nullptr;
   if (int rc = scratch_address(&dev)) return rc;
@@ -142,28 +162,32 @@ extern "C" int bcp_pack_static(const void* const* tensors, const bcp_pack_meta* 
 
   // work list; the unit size doubles until the list fits
   const uint32_t small_bytes = 4096;
-  UnitWriter w;
-  uint64_t tile_bytes = 65536;
-  for (;; tile_bytes *= 2) {
-    w = UnitWriter();
-    pos = 0;
+  auto cut = [&](UnitWriter& w, uint64_t tile_bytes) {
+    uint64_t at = 0;
     for (size_t i = 0; i < n; ++i) {
-      w.run(0, blob_res + pos, metas[i].byte_offset - pos, 0, true, tile_bytes, small_bytes);  // padding -> zeros
+      w.run(0, blob_res + at, metas[i].byte_offset - at, 0, true, tile_bytes, small_bytes);  // padding -> zeros
       const uint64_t res = reinterpret_cast<uintptr_t>(tensors[i]) & 15;
       w.run(res, blob_res + metas[i].byte_offset, metas[i].byte_length, uint32_t(i), false, tile_bytes, small_bytes);
-      pos = metas[i].byte_offset + metas[i].byte_length;
+      at = metas[i].byte_offset + metas[i].byte_length;
     }
-    w.run(0, blob_res + pos, blob_bytes - pos, 0, true, tile_bytes, small_bytes);
-    if (!w.overflow) break;
+    w.run(0, blob_res + at, blob_bytes - at, 0, true, tile_bytes, small_bytes);
+  };
+  UnitWriter counted;
+  uint64_t tile_bytes = 65536;
+  for (;; tile_bytes *= 2) {
+    counted = UnitWriter();
+    cut(counted, tile_bytes);
+    if (!counted.overflow) break;
     if (tile_bytes >= (64u << 20))
       return fail(BCP_ERR_CAPACITY, "bcp_pack_static: more than %u work units even at 64 MiB per unit (use bcp_pack)", kMaxUnits);
   }
-  if (w.n_big + w.n_small == 0) return BCP_OK;
-  // warp units were written from the back: move them behind the CTA-wide units, in order
-  for (uint32_t i = 0; i < w.n_small; ++i) {
-    const bcp_tile t = g_host.tiles[kMaxUnits - 1 - i];
-    g_host.tiles[w.n_big + i] = t;
-  }
+  if (counted.n_big + counted.n_small == 0) return BCP_OK;
+  UnitWriter w;
+  w.store = true;
+  w.small_base = counted.n_big;
+  cut(w, tile_bytes);
+  if (w.overflow || w.n_big != counted.n_big || w.n_small != counted.n_small)
+    return fail(BCP_ERR_INVALID, "bcp_pack_static: the two passes over the layout disagree (arguments changed during the call?)");
   memset(&g_host.ctrl, 0, sizeof g_host.ctrl);
 
 #define BCP_S_CUDA(call)                                                                             \
@@ -172,8 +196,9 @@ extern "C" int bcp_pack_static(const void* const* tensors, const bcp_pack_meta* 
     if (e_ != cudaSuccess) return fail(BCP_ERR_CUDA, "bcp_pack_static: %s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
   // The control words must start at zero for every launch; the pointer table and the work
-  // list are overwritten as far as this call uses them.  Pageable sources are staged by
-  // the runtime before the call returns, so g_host may be reused right after.
+  // list are overwritten as far as this call uses them.  Outside a capture (checked above)
+  // pageable sources are staged by the runtime before the call returns, so g_host may be
+  // reused right after.
   BCP_S_CUDA(cudaMemcpyAsync(&d->ctrl, &g_host.ctrl, sizeof(Control), cudaMemcpyHostToDevice, stream));
   BCP_S_CUDA(cudaMemcpyAsync(d->ptrs, g_host.ptrs, (n + 1) * sizeof(void*), cudaMemcpyHostToDevice, stream));
   BCP_S_CUDA(cudaMemcpyAsync(d->tiles, g_host.tiles, size_t(w.n_big + w.n_small) * sizeof(bcp_tile), cudaMemcpyHostToDevice, stream));

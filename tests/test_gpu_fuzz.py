@@ -83,3 +83,60 @@ def test_random_converting_problems_and_options(cuda_device, stream_seed):
         for b, m in zip(backs, case.dst.buf_bytes):
             assert bool((b[:4096] == 0xA5).all()) and bool((b[4096 + m:] == 0xA5).all()), (case.name, opts)
         plan.destroy()
+
+
+@pytest.mark.parametrize("stream_seed", [21, 22])
+def test_random_pack_layouts(cuda_device, stream_seed):
+    """Random save-blob layouts through bcp_pack, bcp_pack_static and bcp_unpack against the
+    oracle: many tensors under 4 KiB at odd addresses, a few large ones, alignments 16..4096,
+    tensor counts up to the fixed-scratch limit (cases beyond its work-unit limit must be
+    refused, never wrong)."""
+    from paper_2407_20143_b200 import api
+
+    rng = np.random.default_rng(stream_seed)
+    for it in range(12):
+        n = int(rng.choice([1, 7, 300, 2000, 4096]))
+        kind = it % 3
+        if kind == 0:
+            sizes = rng.integers(0, 400, size=n)
+        elif kind == 1:
+            sizes = rng.integers(1, 5000, size=n)
+        else:
+            sizes = np.where(rng.random(n) < 0.02, rng.integers(60_000, 3_000_000, size=n), rng.integers(1, 300, size=n))
+        sizes = [int(x) for x in sizes]
+        align = int(rng.choice([16, 64, 256, 4096]))
+        starts, pos = [], 0
+        for s in sizes:
+            pos = (pos + 15) // 16 * 16 + int(rng.integers(0, 16)) * int(rng.integers(0, 2))
+            starts.append(pos)
+            pos += s
+        host = rng.integers(0, 256, size=pos + 16, dtype=np.uint8)
+        back = torch.from_numpy(host).to(cuda_device)
+        tensors = [back[a:a + s] for a, s in zip(starts, sizes)]
+        ref, table = orc.pack([host[a:a + s] for a, s in zip(starts, sizes)], align)
+        offs, total = bcp.bcp_pack_layout(sizes, align)
+        assert total == ref.size and [int(o) for o, _ in table] == [int(o) for o in offs]
+        metas = list(zip(offs, sizes))
+        blob = torch.full((total,), 0xA5, dtype=torch.uint8, device=cuda_device)
+        bcp.bcp_pack(tensors, metas, blob)
+        torch.cuda.synchronize()
+        assert np.array_equal(blob.cpu().numpy(), ref), ("pack", it, n, align)
+        blob2 = torch.full((total,), 0x5A, dtype=torch.uint8, device=cuda_device)
+        try:
+            bcp.bcp_pack_static(tensors, metas, blob2)
+            torch.cuda.synchronize()
+            assert np.array_equal(blob2.cpu().numpy(), ref), ("static pack", it, n, align)
+        except bcp.BcpError as e:
+            assert e.code == api.ERR_CAPACITY, e
+            torch.cuda.synchronize()
+            assert bool((blob2 == 0x5A).all()), "a refused call must not write"
+        out_back = torch.full((pos + 16,), 0x33, dtype=torch.uint8, device=cuda_device)
+        outs = [out_back[a:a + s] for a, s in zip(starts, sizes)]
+        bcp.bcp_unpack(blob, metas, outs)
+        torch.cuda.synchronize()
+        got = out_back.cpu().numpy()
+        expect = np.full(pos + 16, 0x33, dtype=np.uint8)
+        for a, s in zip(starts, sizes):
+            expect[a:a + s] = host[a:a + s]
+        assert np.array_equal(got, expect), ("unpack", it, n, align)
+    bcp.bcp_pack_cache_clear()
