@@ -38,10 +38,16 @@ if ROOT not in sys.path:
 METRIC = "reshard GB/s (bytes read+written, device-timed)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes moved per algorithmic byte by the dominant kernel, from ncu captures summarised
-# under profiles/ (bcp_tma_kernel_*.md, bcp_convert_kernel_*.md): (dram__bytes_read.sum + dram__bytes_write.sum) / B_min.
-NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {("cfg2", "bcp_tma_kernel"): 0.9994, ("cfg3", "bcp_tma_kernel"): 0.9990,
-                                       ("cfg4", "bcp_tma_kernel"): 0.9998, ("evalmerge", "bcp_convert_kernel"): 0.9994}
+# DRAM bytes moved per algorithmic byte by the dominant kernel: (dram__bytes_read.sum + dram__bytes_write.sum) / B_min
+# of one launch under ncu.  A recorded measurement, not a live one: each entry names the summary under profiles/ it
+# was read from, the commit whose kernels were captured and the size of the captured case; the line repeats them in
+# roofline.traffic_note so that a stale ratio is visible.
+NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
+    ("cfg2", "bcp_tma_kernel"): (0.9994, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369", "full size"),
+    ("cfg3", "bcp_tma_kernel"): (0.9990, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369", "full size"),
+    ("cfg4", "bcp_tma_kernel"): (0.9998, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "0874854", "full size"),
+    ("evalmerge", "bcp_convert_kernel"): (0.9994, "profiles/bcp_convert_kernel_evalmerge-L2_ncu_full.md", "0874854", "full size"),
+}
 
 
 def parse_args():
@@ -56,9 +62,12 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
-    ap.add_argument("--pack", action="store_true", help="also time bcp_pack of one target rank (reported as extra keys)")
-    ap.add_argument("--stage", action="store_true",
-                    help="also time asynchronous save staging of every target rank through the pinned ping-pong pool")
+    ap.add_argument("--no-pack", action="store_true", help="skip the pack / unpack timing of one target rank (extra key `pack`)")
+    ap.add_argument("--no-stage", action="store_true",
+                    help="skip the asynchronous save staging of every target rank through the pinned ping-pong pool (extra key `stage`)")
+    ap.add_argument("--no-also", action="store_true", help="with the default workload: skip the device-timed run of cfg3 (extra key `also`)")
+    ap.add_argument("--pack", action="store_true", help=argparse.SUPPRESS)   # on by default now; accepted for old command lines
+    ap.add_argument("--stage", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--cpu-sample-gb", type=float, default=4.0,
                     help="bytes read+written by one pass of the CPU oracle over its sample of the workload")
     ap.add_argument("--cpu-passes", type=int, default=40, help="timed passes of the oracle over its sample (about 10 s)")
@@ -263,43 +272,48 @@ def run_reference(a):
 
 
 # ----------------------------------------------------------------------------------- main arm
-def main():
-    a = parse_args()
-    if a.impl == "reference":
-        run_reference(a)
-        return
+POISON = 0xA5
+
+
+def device_run(a, case, opts, dev, local_rank, ws):
+    """Plan, fill, warm up, time exactly a.steps executions of the plan on resident buffers, verify.
+
+    The targets are overwritten with a poison byte after the last-but-one timed step, outside both
+    event brackets, so the check that follows proves that a TIMED step wrote every target byte (and
+    left every byte no entry names alone).  Returns (figures, plan, src, dst, stream)."""
     import torch
 
     import paper_2407_20143_b200 as bcp
     from paper_2407_20143_b200 import dist as D
     from workloads import fills
 
-    rank, local_rank, ws = D.world()
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    D.init("nccl")
-    case = make_case(a)
     keys = case.key_ids
-    opts = plan_opts(a)
     t0 = time.perf_counter()
     plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts, **case.plan_opts)
     plan_ms = (time.perf_counter() - t0) * 1e3
     st = plan.stats()
     b_min = st["bytes_src_unique"] + st["bytes_copied"]
-    # what the unit list loads + stores (replica reads counted every time); a converting plan reads
-    # the saved type and writes the wanted one, and none of its sources is read twice
-    b_moved = b_min if case.convert else 2 * st["bytes_copied"]
     free, _ = torch.cuda.mem_get_info()
     need = sum(case.src.buf_bytes) + sum(case.dst.buf_bytes)
-    assert free > need + (2 << 30), f"{case.name} needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free"
+    assert free > need + (6 << 30), f"{case.name} needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free"
     src = fills.fill_state(case.src, keys, case.fill, case.seed, dev)
     dst = [torch.zeros(n, dtype=torch.uint8, device=dev) for n in case.dst.buf_bytes]
     stream = torch.cuda.current_stream()
 
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(a.steps)]
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    evs = [(ev(), ev()) for _ in range(a.steps)]
     # inputs far larger than the 126 MB L2 need no flush; small workloads get one before every step
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if b_min < (1 << 30) else None
+
+    def step(e0, e1):
+        if flush is not None:
+            flush.zero_()  # evict the previous step's lines: this workload would fit in L2
+        e0.record(stream)
+        bcp.bcp_reshard(plan, src, dst, stream)
+        e1.record(stream)
+
     with ClockSampler(local_rank) as clocks:
         clocks.wait_first_sample()
         torch.cuda.synchronize()
@@ -312,35 +326,67 @@ def main():
         torch.cuda.synchronize()
         D.barrier()
         torch.cuda.synchronize()
-        t_begin = torch.cuda.Event(enable_timing=True)
-        t_end = torch.cuda.Event(enable_timing=True)
+        head0, head1, last0, last1 = ev(), ev(), ev(), ev()
         clocks.mark_begin()
-        t_begin.record(stream)
-        for e0, e1 in evs:
-            if flush is not None:
-                flush.zero_()  # evict the previous step's lines: this workload would fit in L2
-            e0.record(stream)
-            bcp.bcp_reshard(plan, src, dst, stream)
-            e1.record(stream)
-        t_end.record(stream)
+        head0.record(stream)
+        for e0, e1 in evs[:-1]:
+            step(e0, e1)
+        head1.record(stream)
+        if not a.no_verify:  # between the two timed brackets
+            for d in dst:
+                d.fill_(POISON)
+        last0.record(stream)
+        step(*evs[-1])
+        last1.record(stream)
         torch.cuda.synchronize()
         clocks.mark_end()
     D.barrier()
-    total_ms = t_begin.elapsed_time(t_end)
+    total_ms = head0.elapsed_time(head1) + last0.elapsed_time(last1)
     launch_ms = sorted(e0.elapsed_time(e1) for e0, e1 in evs)
     # with flushes between the steps only the steps themselves count
     ms_step = D.max_over_ranks((sum(launch_ms) if flush is not None else total_ms) / a.steps, dev)
     bcp.bcp_plan_device_status(plan)
-    value = b_min * ws / (ms_step * 1e-3) / 1e9
 
-    verified = None
-    if not a.no_verify:  # spot check: a sample of target entries against the generative fill
+    verified, checked = None, 0
+    if not a.no_verify:  # whole target buffers against the generative fill; unnamed bytes must still be poison
         verified = True
-        for m in case.dst.metas[:: max(1, len(case.dst.metas) // 48)]:
-            hi = min(m.numel, 1 << 22)
-            want = fills.entry_bytes(m, keys[m.fqn], case.fill, case.seed, dev, 0, hi)
-            got = dst[m.buf_index][m.byte_offset:m.byte_offset + hi * m.itemsize]
-            verified = verified and bool(torch.equal(got, want))
+        for r in range(len(dst)):
+            want = torch.full_like(dst[r], POISON)
+            for m in case.dst.metas:
+                if m.buf_index == r:
+                    fills.write_entry(want, m, keys[m.fqn], case.fill, case.seed)
+            verified = verified and bool(torch.equal(dst[r], want))
+            checked += dst[r].numel()
+            del want
+    fig = {"st": st, "b_min": b_min, "plan_ms": plan_ms, "first_call_ms": first_call_ms, "ms_step": ms_step,
+           "launch_ms": launch_ms, "verified": verified, "verified_bytes": checked, "clocks": clocks.summary(),
+           "flushed": flush is not None}
+    del flush
+    return fig, plan, src, dst, stream
+
+
+def main():
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+        return
+    import torch
+
+    from paper_2407_20143_b200 import dist as D
+
+    rank, local_rank, ws = D.world()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    D.init("nccl")
+    case = make_case(a)
+    opts = plan_opts(a)
+    fig, plan, src, dst, stream = device_run(a, case, opts, dev, local_rank, ws)
+    st, b_min, ms_step, launch_ms = fig["st"], fig["b_min"], fig["ms_step"], fig["launch_ms"]
+    # what the unit list loads + stores (replica reads counted every time); a converting plan reads
+    # the saved type and writes the wanted one, and none of its sources is read twice
+    b_moved = b_min if case.convert else 2 * st["bytes_copied"]
+    value = b_min * ws / (ms_step * 1e-3) / 1e9
 
     # kernels enqueued by one bcp_reshard: the TMA staging kernel (if any unit qualifies) and the
     # register kernel (if any unit is left for it)
@@ -361,36 +407,42 @@ def main():
                    "bytes_per_step": b_min, "bytes_counted": "unique source bytes read + target bytes written",
                    "src_ranks": len(case.src.buf_bytes), "dst_ranks": len(case.dst.buf_bytes),
                    "work_units": st["n_tiles"] + st["n_small_tiles"] + st["n_cvt_tiles"],
-                   "l2": "inputs_exceed_l2" if flush is None else "flushed_before_every_step_512MiB", "fill": case.fill,
-                   "multi_gpu": "replicas only", "plan_opts": opts, "plan_ms": plan_ms, "first_call_ms": first_call_ms},
+                   "l2": "flushed_before_every_step_512MiB" if fig["flushed"] else "inputs_exceed_l2", "fill": case.fill,
+                   "multi_gpu": "replicas only", "plan_opts": opts, "plan_ms": fig["plan_ms"],
+                   "first_call_ms": fig["first_call_ms"]},
         "gbps_b_moved": b_moved * ws / (ms_step * 1e-3) / 1e9,
         "pct_of_8tbs_nominal": value / ws / 8000.0 * 100.0,
         "launch_ms": {"median": launch_ms[len(launch_ms) // 2], "best": launch_ms[0], "mean": avg_launch_ms},
         "gpu_launches": a.steps * kernels_per_step,
         "kernels_per_step": kernels_per_step,
-        "verified": verified,
-        "clocks": clocks.summary(),
+        "verified": fig["verified"],
+        "verified_how": f"targets poisoned before the last timed step; after it all {len(dst)} target buffers "
+                        f"({fig['verified_bytes']} bytes) equal the generative fill, unnamed bytes still poison",
+        "clocks": fig["clocks"],
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": f"of {peak_kind}", "traffic": None, "kernel": dominant,
                      "algorithmic_bytes_per_launch": b_min,
                      "duration_note": "CUDA events around one bcp_reshard (all its kernels; the dominant kernel's "
                                       "share of device time is in profiles/)"},
     }
-    ratio = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get((a.workload, dominant))
-    if ratio is not None:
+    rec = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get((a.workload, dominant))
+    if rec is not None:
+        ratio, where, commit, size = rec
         out["roofline"]["traffic"] = ratio * b_min
-        out["roofline"]["traffic_note"] = "ncu dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch " \
-                                          "(profiles/" + ("bcp_convert_kernel_evalmerge-L2_ncu_full.md" if case.convert else
-                                                          "bcp_tma_kernel_full_size_dram_bytes.md") + ")"
-        if a.layers:
-            out["roofline"]["traffic_note"] += ", scaled by algorithmic bytes to this shallower model"
+        out["roofline"]["traffic_note"] = (f"recorded, not live: ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch = "
+                                           f"{ratio} x algorithmic bytes, captured at {size} on the kernels of commit {commit} "
+                                           f"({where}), scaled by algorithmic bytes to this launch")
 
-    if a.pack and rank == 0:
+    # pack / unpack of one target rank and asynchronous save staging of every target rank: steps a6 / a7 of
+    # the path and the save pipeline's staging, timed separately from the headline (extra keys)
+    if not a.no_pack and rank == 0:
         out["pack"] = time_pack(case, dst, dev, stream, a.steps)
-    if a.stage and rank == 0:
-        out["stage"] = time_stage(case, dst, dev, stream)
+    if not a.no_stage and rank == 0:
+        try:
+            out["stage"] = time_stage(case, dst, dev, stream)
+        except Exception as e:  # e.g. the host refuses that much pinned memory
+            out["stage"] = {"skipped": str(e)[:200]}
 
-    # free the device-timed buffers' plan before the host-path run allocates its own staging
     if not a.no_e2e:
         out["e2e"] = run_e2e(a, case, plan, src, dst, dev, ws, b_min)
     else:
@@ -415,6 +467,26 @@ def main():
         except Exception as e:  # the single-core figure above is the reported baseline
             out["cpu_baseline_all_cores"] = {"value": None, "error": str(e)[:200]}
     plan.destroy()
+    del src, dst, plan
+    torch.cuda.empty_cache()
+
+    # the other half of the throughput target: the 8B merge (cfg3), device-timed the same way, no host leg
+    if a.workload == "cfg2" and not a.layers and not a.no_also:
+        from workloads.configs import CONFIGS
+
+        other = CONFIGS["cfg3"]()
+        f3, p3, s3, d3, _ = device_run(a, other, opts, dev, local_rank, ws)
+        mean3 = sum(f3["launch_ms"]) / len(f3["launch_ms"])
+        gbs3 = f3["b_min"] * ws / (f3["ms_step"] * 1e-3) / 1e9
+        out["also"] = {"cfg3": {"workload": other.name, "ms_per_step": f3["ms_step"], "value": gbs3, "unit": UNIT,
+                                "bytes_per_step": f3["b_min"], "steps": a.steps,
+                                "frac": f3["b_min"] / (mean3 * 1e-3) / 1e9 / peak, "peak_source": f"of {peak_kind}",
+                                "pct_of_8tbs_nominal": gbs3 / ws / 8000.0 * 100.0, "verified": f3["verified"],
+                                "verified_bytes": f3["verified_bytes"], "clocks": f3["clocks"],
+                                "gpu_launches": a.steps * (int(f3["st"]["n_tma_tiles"] > 0) +
+                                                           int(f3["st"]["n_tiles"] - f3["st"]["n_tma_tiles"] + f3["st"]["n_small_tiles"] > 0))}}
+        p3.destroy()
+        del s3, d3
     if rank == 0:
         print(json.dumps(out))
     D.shutdown()
@@ -460,10 +532,11 @@ def time_pack(case, dst, dev, stream, steps):
     torch.cuda.synchronize()
     ms_un = u0.elapsed_time(u1) / steps
     ok = all(bool(torch.equal(outs[o - outs.data_ptr():o - outs.data_ptr() + n],
-                              dst[r][m.byte_offset:m.byte_offset + n])) for o, n, m in list(zip(optrs, sizes, ms))[:64])
+                              dst[r][m.byte_offset:m.byte_offset + n])) for o, n, m in zip(optrs, sizes, ms))
     del blob, outs
     return {"tensors": len(ms), "blob_bytes": total, "ms_per_pack": ms_step, "gbps": nbytes / (ms_step * 1e-3) / 1e9,
             "ms_per_unpack": ms_un, "unpack_gbps": 2 * sum(sizes) / (ms_un * 1e-3) / 1e9, "round_trip_ok": ok,
+            "steps": steps, "rank": r,
             "bytes_counted": "pack: tensor bytes read + blob bytes written (padding included); unpack: 2 x tensor bytes"}
 
 
