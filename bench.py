@@ -65,6 +65,12 @@ def parse_args():
     ap.add_argument("--no-pack", action="store_true", help="skip the pack / unpack timing of one target rank (extra key `pack`)")
     ap.add_argument("--no-stage", action="store_true",
                     help="skip the asynchronous save staging of every target rank through the pinned ping-pong pool (extra key `stage`)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="time the cross-rank path instead: blobs and target buffers dealt to the N ranks, a step = pack -> "
+                         "all-to-all -> reshard (per-stage times, bytes crossed); without the flag --gpus N runs replicas")
+    ap.add_argument("--exchange-emulate", type=int, default=2,
+                    help="after the headline run, emulate this many ranks of the cross-rank path on the one GPU and report "
+                         "per-stage device times (extra key `exchange_emulated`); 0 or 1 skips it")
     ap.add_argument("--no-also", action="store_true", help="with the default workload: skip the device-timed run of cfg3 (extra key `also`)")
     ap.add_argument("--pack", action="store_true", help=argparse.SUPPRESS)   # on by default now; accepted for old command lines
     ap.add_argument("--stage", action="store_true", help=argparse.SUPPRESS)
@@ -348,16 +354,8 @@ def device_run(a, case, opts, dev, local_rank, ws):
     bcp.bcp_plan_device_status(plan)
 
     verified, checked = None, 0
-    if not a.no_verify:  # whole target buffers against the generative fill; unnamed bytes must still be poison
-        verified = True
-        for r in range(len(dst)):
-            want = torch.full_like(dst[r], POISON)
-            for m in case.dst.metas:
-                if m.buf_index == r:
-                    fills.write_entry(want, m, keys[m.fqn], case.fill, case.seed)
-            verified = verified and bool(torch.equal(dst[r], want))
-            checked += dst[r].numel()
-            del want
+    if not a.no_verify:
+        verified, checked = verify_targets(case, dst, range(len(dst)))
     fig = {"st": st, "b_min": b_min, "plan_ms": plan_ms, "first_call_ms": first_call_ms, "ms_step": ms_step,
            "launch_ms": launch_ms, "verified": verified, "verified_bytes": checked, "clocks": clocks.summary(),
            "flushed": flush is not None}
@@ -365,10 +363,196 @@ def device_run(a, case, opts, dev, local_rank, ws):
     return fig, plan, src, dst, stream
 
 
+def verify_targets(case, bufs, indices):
+    """Whole target buffers against the generative fill; bytes no entry names must still be poison.
+    bufs[i] is the buffer of target rank indices[i].  Returns (all equal, bytes compared)."""
+    import torch
+
+    from workloads import fills
+
+    by_buf = {}
+    for m in case.dst.metas:
+        by_buf.setdefault(m.buf_index, []).append(m)
+    ok, checked = True, 0
+    for buf, r in zip(bufs, indices):
+        want = torch.full_like(buf, POISON)
+        for m in by_buf.get(r, []):
+            fills.write_entry(want, m, case.key_ids[m.fqn], case.fill, case.seed)
+        ok = ok and bool(torch.equal(buf, want))
+        checked += buf.numel()
+        del want
+    return ok, checked
+
+
+def block_owner(n_bufs: int, world: int):
+    """Buffers to ranks in contiguous blocks (rank r holds buffers [r*n/world, (r+1)*n/world))."""
+    return [(b * world) // n_bufs for b in range(n_bufs)]
+
+
+def exchange_emulated(a, case, src, dst, dev, world):
+    """The cross-rank exchange with `world` ranks emulated one after the other on this one GPU:
+    saved blobs and target buffers are dealt to the ranks in contiguous blocks; every rank's pack
+    runs first (so that its peers' segments exist), then every rank's step, with the collective
+    replaced by device copies out of the peers' send buffers.  Device time of every stage, bytes
+    that would cross the links, and the usual whole-buffer check.  No kernel waits for another."""
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+    from paper_2407_20143_b200 import multi
+
+    opts = dict(plan_opts(a), **case.plan_opts)
+    t0 = time.perf_counter()
+    src_owner, dst_owner = block_owner(len(src), world), block_owner(len(dst), world)
+    args = (case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    needs = [multi.needed_entries(*args, dst_owner, r, **opts) for r in range(world)]
+    xs = [multi.build_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, r,
+                               world, needs, **opts) for r in range(world)]
+    plan_s = time.perf_counter() - t0
+    stream = torch.cuda.current_stream()
+    for x in xs:
+        x.bind(dev)
+    per_rank = []
+    for rep in range(3):  # two warm-up rounds (work lists uploaded, pack layouts cached), then the recorded one
+        if rep == 2 and not a.no_verify:
+            for d in dst:
+                d.fill_(POISON)
+        for x in xs:
+            multi.pack_sends(x, case.src.metas, [src[b] for b in x.local_src], x.send_buf, stream)
+        torch.cuda.synchronize()
+        for r, x in enumerate(xs):
+            def swap(recv, send, recv_splits, send_splits, r=r):
+                at = 0
+                for s_ in range(world):
+                    off = sum(xs[s_].send_bytes[:r])
+                    recv[at:at + recv_splits[s_]].copy_(xs[s_].send_buf[off:off + recv_splits[s_]])
+                    at += recv_splits[s_]
+
+            multi.run_exchange(x, case.src.metas, [src[b] for b in x.local_src], [dst[b] for b in x.local_dst], stream, all_to_all=swap)
+            torch.cuda.synchronize()
+            if rep == 2:
+                ms = x.stage_ms()
+                pl, pr = x.plan_local, x.plan_remote
+                per_rank.append({"rank": r, "blobs": len(x.local_src), "targets": len(x.local_dst),
+                                 "sent_bytes": sum(x.send_bytes), "received_bytes": sum(x.recv_bytes),
+                                 "local_bytes_written": pl.stats()["bytes_copied"] if pl else 0,
+                                 "remote_bytes_written": pr.stats()["bytes_copied"] if pr else 0,
+                                 "ms": {k: round(v, 4) for k, v in ms.items()}})
+    for x in xs:
+        for p in (x.plan_local, x.plan_remote):
+            if p is not None:
+                bcp.bcp_plan_device_status(p)
+    ok, checked = (None, 0) if a.no_verify else verify_targets(case, dst, range(len(dst)))
+    for x in xs:
+        x.destroy()
+    link = 770.0  # GB/s per direction per GPU: this pool's measured peer copy (context for the bytes, not a measurement here)
+    return {"world": world, "emulated_on_one_gpu": True, "plan_s_all_ranks": plan_s, "per_rank": per_rank, "verified": ok,
+            "verified_bytes": checked,
+            "all_to_all_note": "device copies out of the emulated peers' send buffers stand in for the collective; its "
+                               "time here says nothing about NVLink",
+            "all_to_all_ms_at_770GBs": max(max(p["sent_bytes"], p["received_bytes"]) for p in per_rank) / link / 1e6,
+            "stages": "pack (main stream) -> all-to-all (main) -> reshard_remote (main); reshard_local on a side stream "
+                      "behind the pack, beside the transfer; step = begin of pack to both streams done"}
+
+
+def run_exchange_bench(a):
+    """bench.py --exchange: saved blobs and target buffers of the workload are dealt to the ranks in
+    contiguous blocks; a step is pack -> all-to-all -> reshard with the plans reused.  With one rank
+    nothing crosses and the step is the rank's plain reshard."""
+    import torch
+
+    import paper_2407_20143_b200 as bcp
+    from paper_2407_20143_b200 import dist as D
+    from paper_2407_20143_b200 import multi
+    from workloads import fills
+
+    rank, local_rank, ws = D.world()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    D.init("nccl")
+    case = make_case(a)
+    opts = dict(plan_opts(a), **case.plan_opts)
+    src_owner, dst_owner = block_owner(len(case.src.buf_bytes), ws), block_owner(len(case.dst.buf_bytes), ws)
+    t0 = time.perf_counter()
+    x = multi.plan_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, **opts)
+    plan_ms = (time.perf_counter() - t0) * 1e3
+    by_buf = {}
+    for m in case.src.metas:
+        by_buf.setdefault(m.buf_index, []).append(m)
+    blobs = []
+    for b in x.local_src:
+        t = torch.zeros(case.src.buf_bytes[b], dtype=torch.uint8, device=dev)
+        for m in by_buf.get(b, []):
+            fills.write_entry(t, m, case.key_ids[m.fqn], case.fill, case.seed)
+        blobs.append(t)
+    dst = [torch.zeros(n, dtype=torch.uint8, device=dev) for n in x.dst_buf_bytes]
+    stream = torch.cuda.current_stream()
+    x.bind(dev)
+    plans = [p for p in (x.plan_local, x.plan_remote) if p is not None]
+    b_local = sum(p.stats()["bytes_src_unique"] + p.stats()["bytes_copied"] for p in plans)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    with ClockSampler(local_rank) as clocks:
+        clocks.wait_first_sample()
+        for _ in range(max(a.warmup, 3)):
+            multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+        torch.cuda.synchronize()
+        D.barrier()
+        torch.cuda.synchronize()
+        head0, head1, last0, last1 = ev(), ev(), ev(), ev()
+        clocks.mark_begin()
+        head0.record(stream)
+        for _ in range(a.steps - 1):
+            multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+        head1.record(stream)
+        if not a.no_verify:
+            for d in dst:
+                d.fill_(POISON)
+        last0.record(stream)
+        multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+        last1.record(stream)
+        torch.cuda.synchronize()
+        clocks.mark_end()
+    D.barrier()
+    ms_step = D.max_over_ranks((head0.elapsed_time(head1) + last0.elapsed_time(last1)) / a.steps, dev)
+    stages = {k: D.max_over_ranks(v, dev) for k, v in x.stage_ms().items()}  # of the last timed step
+    for p in plans:
+        bcp.bcp_plan_device_status(p)
+    ok, checked = (None, 0) if a.no_verify else verify_targets(case, dst, x.local_dst)
+    ok_all = None if ok is None else D.max_over_ranks(0.0 if ok else 1.0, dev) == 0.0
+    total_bytes = D.sum_over_ranks(b_local, dev)
+    sent = D.max_over_ranks(float(sum(x.send_bytes)), dev)
+    recv = D.max_over_ranks(float(sum(x.recv_bytes)), dev)
+    value = total_bytes / (ms_step * 1e-3) / 1e9
+    n_kernels = sum(int(p.stats()["n_tma_tiles"] > 0) + int(p.stats()["n_tiles"] - p.stats()["n_tma_tiles"] + p.stats()["n_small_tiles"] > 0)
+                    + int(p.stats()["n_cvt_tiles"] > 0) for p in plans) + (2 if sum(x.send_bytes) else 0)
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": a.steps, "warmup": max(a.warmup, 3),
+           "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "u8",
+           "data": "synthetic",
+           "config": {"workload": case.name, "mode": "exchange", "bytes_per_step": total_bytes,
+                      "bytes_counted": "per rank: distinct source bytes its plans read (own blobs and received segments) + "
+                                       "target bytes written; summed over ranks",
+                      "partition": "saved blobs and target buffers in contiguous blocks over the ranks",
+                      "l2": "inputs_exceed_l2", "fill": case.fill, "plan_ms": plan_ms, "plan_opts": plan_opts(a)},
+           "exchange": {"world": ws, "stage_ms_max_over_ranks": stages, "sent_bytes_max_rank": sent, "received_bytes_max_rank": recv,
+                        "collective": "torch.distributed.all_to_all_single (NCCL)" if ws > 1 else "none (one rank: nothing crosses)"},
+           "gpu_launches": a.steps * n_kernels, "verified": ok_all, "verified_bytes": checked, "clocks": clocks.summary(),
+           "e2e": None, "roofline": None, "cpu_baseline": None}
+    x.destroy()
+    if rank == 0:
+        print(json.dumps(out))
+    D.shutdown()
+
+
 def main():
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+        return
+    if a.exchange:
+        run_exchange_bench(a)
         return
     import torch
 
@@ -442,6 +626,10 @@ def main():
             out["stage"] = time_stage(case, dst, dev, stream)
         except Exception as e:  # e.g. the host refuses that much pinned memory
             out["stage"] = {"skipped": str(e)[:200]}
+
+    # the cross-rank exchange (pack -> all-to-all -> reshard in two plans), ranks emulated on this GPU
+    if a.exchange_emulate > 1 and rank == 0 and not case.convert:
+        out["exchange_emulated"] = exchange_emulated(a, case, src, dst, dev, a.exchange_emulate)
 
     if not a.no_e2e:
         out["e2e"] = run_e2e(a, case, plan, src, dst, dev, ws, b_min)

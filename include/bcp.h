@@ -160,6 +160,14 @@ typedef struct {
                                to a bf16 evaluation job (and back).                                       */
   uint32_t convert_src_tag; /* see convert */
   uint32_t convert_dst_tag;
+  uint32_t src_buf_first;   /* with src_buf_count != 0: matching, the disjointness check and the coverage check run */
+  uint32_t src_buf_count;   /* against every saved entry as usual, but the plan keeps only the pieces that are read
+                               from source buffers [src_buf_first, src_buf_first + src_buf_count); it writes the
+                               target bytes those pieces hold and no others.  Plans for disjoint ranges that
+                               together cover all source buffers write every target byte exactly once between
+                               them and may run concurrently (the exchange of Sec. 4.1 / 4.2 across GPUs: the
+                               pieces read from a rank's own blobs are copied while the segments of the other
+                               ranks are still on their way).  0: all source buffers                          */
 } bcp_plan_opts;
 
 /*
@@ -349,6 +357,7 @@ BCP_API int bcp_reshard(bcp_plan_t* plan, const void* const* src_blobs, size_t n
  *     buffer over three streams (`stream` for the kernels, two plan-owned streams for uploads
  *     and downloads), so that downloads of finished target buffers overlap the uploads still
  *     needed by later ones.
+ * Plans restricted to some source buffers (bcp_plan_opts.src_buf_count) are refused: BCP_ERR_INVALID.
  */
 BCP_API int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_blobs_host, size_t n_src_bufs,
                      void* const* dst_bufs_host, size_t n_dst_bufs, void* stream);

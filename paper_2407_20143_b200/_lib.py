@@ -50,6 +50,8 @@ class PlanOptsC(C.Structure):
         ("convert", C.c_uint32),
         ("convert_src_tag", C.c_uint32),
         ("convert_dst_tag", C.c_uint32),
+        ("src_buf_first", C.c_uint32),
+        ("src_buf_count", C.c_uint32),
     ]
 
 

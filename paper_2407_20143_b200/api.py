@@ -254,6 +254,19 @@ def bcp_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_byt
     _check(L.lib().bcp_pack(_ptrs(tensors), _pack_metas(metas), len(tensors), bp, nb, _stream(stream)))
 
 
+def marshal_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]]):
+    """The C arrays of a pack call, for callers that repeat one pack many times (see bcp_pack_marshalled)."""
+    return _ptrs(tensors), _pack_metas(metas), len(tensors)
+
+
+def bcp_pack_marshalled(args, blob, blob_bytes: Optional[int] = None, stream=None) -> None:
+    """bcp_pack with arrays prepared by marshal_pack (same call, no per-call marshalling)."""
+    ptrs, metas, n = args
+    nb = blob_bytes if blob_bytes is not None else blob.numel() * blob.element_size()
+    bp = blob if isinstance(blob, int) else blob.data_ptr()
+    _check(L.lib().bcp_pack(ptrs, metas, n, bp, nb, _stream(stream)))
+
+
 def bcp_pack_static(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_bytes: Optional[int] = None,
                     stream=None) -> None:
     """bcp_pack without any allocation: the work list lives in a fixed device array inside the

@@ -354,7 +354,7 @@ void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vec
 
 extern "C" {
 
-int bcp_version(void) { return 200; }  // 0.2.0: plan images carry converting units
+int bcp_version(void) { return 201; }  // 0.2.1: plan options (and so plan images) carry the source-buffer range
 
 const char* bcp_last_error(void) { return last_error().c_str(); }
 

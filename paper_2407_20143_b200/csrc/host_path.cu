@@ -83,6 +83,8 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
                      size_t n_dst_bufs, void* stream_) {
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
+  if (plan->opt.src_buf_count)  // it writes part of every target buffer; this call hands back whole buffers
+    return fail(BCP_ERR_INVALID, "bcp_reshard_host: the plan is restricted to some source buffers (src_buf_count)");
   if (n_src_bufs != plan->src_bytes.size() || n_dst_bufs != plan->dst_bytes.size())
     return fail(BCP_ERR_INVALID, "buffer counts differ from the planned ones");
   if ((n_src_bufs && !src_host) || (n_dst_bufs && !dst_host)) return fail(BCP_ERR_INVALID, "pointer array is NULL");

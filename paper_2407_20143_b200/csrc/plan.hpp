@@ -49,6 +49,7 @@ struct Options {
   uint32_t test_stall = 0;
   uint32_t fanout = 1;  // 1 on, 2 off
   uint32_t convert = 0, convert_src_tag = 0, convert_dst_tag = 0;
+  uint32_t src_buf_first = 0, src_buf_count = 0;  // count 0: pieces from every source buffer are executed
 };
 
 // A strided rectangle that is staged with 2-D tensor-map copies.  Its two descriptors (source

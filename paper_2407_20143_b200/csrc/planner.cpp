@@ -58,6 +58,8 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     o.convert = in->convert;
     o.convert_src_tag = in->convert_src_tag;
     o.convert_dst_tag = in->convert_dst_tag;
+    o.src_buf_first = in->src_buf_first;
+    o.src_buf_count = in->src_buf_count;
   }
   if (o.tile_bytes % 4096 || o.tile_bytes < 4096 || o.tile_bytes > (64u << 20))
     return fail(BCP_ERR_INVALID, "tile_bytes must be a multiple of 4096 in [4096, 64 MiB]");
@@ -86,6 +88,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
     return fail(BCP_ERR_INVALID, "convert needs two different dtype tags (convert_src_tag, convert_dst_tag)");
   if (!o.convert && (o.convert_src_tag || o.convert_dst_tag))
     return fail(BCP_ERR_INVALID, "convert_src_tag / convert_dst_tag are set but convert is 0");
+  if (!o.src_buf_count && o.src_buf_first) return fail(BCP_ERR_INVALID, "src_buf_first is set but src_buf_count is 0");
   if (o.tma_min_row_bytes < 16 || o.tma_min_row_bytes % 16 || o.tma_min_row_bytes > 65536)
     return fail(BCP_ERR_INVALID, "tma_min_row_bytes must be a multiple of 16 in [16, 65536]");
   *out = o;
@@ -469,6 +472,9 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       }
     }
   }
+  const uint32_t keep_first = opt.src_buf_first, keep_count = opt.src_buf_count;
+  if (keep_count && (keep_first > n_src_bufs || keep_count > n_src_bufs - keep_first))
+    return fail(BCP_ERR_INVALID, "source buffers [%u, %u + %u) are not among the %zu given", keep_first, keep_first, keep_count, n_src_bufs);
   struct Scratch {
     std::vector<SegKey> segs;    // matched segments of the family at hand
     std::vector<int64_t> reach;  // reach[i] = largest end (along dim 0) among the family's saved boxes 0..i
@@ -538,6 +544,9 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
         int64_t o[BCP_MAX_NDIM], l[BCP_MAX_NDIM];
         if (!intersect(s, d, nd, o, l)) continue;
         covered += volume(l, 0, nd);
+        // a plan restricted to some source buffers matches and checks coverage against all of
+        // them, and keeps the pieces that are read from the chosen ones
+        if (keep_count && (s.buf < keep_first || s.buf - keep_first >= keep_count)) continue;
         ++n_inter;
         lower(s, d, nd, f.itemsize, f.d_itemsize, f.cvt, o, l, items);
         SegKey key = {si, 0, 0, uint64_t(volume(l, 0, nd)) * f.itemsize};

@@ -12,7 +12,9 @@ their owners, so the same step becomes:
   3. every owner packs, per receiver, the needed entries of its blobs into one send buffer
      (`bcp_pack`, on the GPU), and one `all_to_all_single` moves the segments (NCCL over NVLink);
   4. every rank re-plans its targets against the entries as they now lie in its memory (its
-     own blobs plus one received segment per peer) and executes that plan (`bcp_reshard`).
+     own blobs plus one received segment per peer), as two plans: the pieces read from its own
+     blobs, which are copied on a side stream while the segments travel, and the pieces read
+     from received segments, copied once they have arrived (`bcp_reshard`, twice).
 
 Steps 1, 2 and 4's planning are metadata work; all bytes move in library kernels and in the
 collective.  Everything here is argument marshalling around the C ABI and `torch.distributed`.
@@ -30,7 +32,13 @@ SEGMENT_ALIGN = 256  # entries inside a send segment, and segments inside the bu
 
 @dataclass
 class Exchange:
-    """What one rank sends, receives and finally executes."""
+    """What one rank sends, receives and finally executes.
+
+    The rank's final work is split in two plans over the same buffer lists (sources = own blobs,
+    then one received segment per sender with recv_bytes > 0): `plan_local` holds the pieces read
+    from the rank's own blobs, `plan_remote` the pieces read from received segments.  Between them
+    they write every target byte exactly once, so the local one can run while the segments are
+    still travelling."""
 
     rank: int
     world: int
@@ -40,14 +48,54 @@ class Exchange:
     send_offsets: List[List[int]]        # per receiver: byte offset of every such entry inside the segment
     send_bytes: List[int]                # per receiver: segment size (multiple of SEGMENT_ALIGN; 0 for none / self)
     recv_bytes: List[int]                # per sender
-    plan: Optional[api.Plan] = None      # final plan: sources = own blobs, then one segment per sender with recv_bytes > 0
+    plan_local: Optional[api.Plan] = None
+    plan_remote: Optional[api.Plan] = None   # None when nothing is received
     src_buf_bytes: List[int] = field(default_factory=list)
     dst_buf_bytes: List[int] = field(default_factory=list)
+    # device side, created once by bind(): nothing is allocated per step
+    send_buf: object = None
+    recv_buf: object = None
+    side: object = None                  # stream of the local plan
+    events: Dict[str, object] = field(default_factory=dict)
+    pack_args: object = None             # marshalled arguments of the sender-side pack
+
+    def bind(self, device) -> None:
+        """Send / receive buffers, the side stream and the stage events, once per exchange."""
+        import torch
+
+        if self.send_buf is not None:
+            return
+        with torch.cuda.device(device):
+            self.send_buf = torch.empty(max(1, sum(self.send_bytes)), dtype=torch.uint8, device=device)
+            self.recv_buf = torch.empty(max(1, sum(self.recv_bytes)), dtype=torch.uint8, device=device)
+            self.side = torch.cuda.Stream(device=device)
+            for k in ("begin", "packed", "arrived", "remote_done", "local_begin", "local_done", "end"):
+                self.events[k] = torch.cuda.Event(enable_timing=True)
+
+    def sources(self, local_blobs: Sequence) -> List:
+        """Source list of both plans: own blobs, then the received segments (views of recv_buf)."""
+        srcs, at = list(local_blobs), 0
+        for s in range(self.world):
+            if self.recv_bytes[s]:
+                srcs.append(self.recv_buf[at:at + self.recv_bytes[s]])
+                at += self.recv_bytes[s]
+        return srcs
+
+    def stage_ms(self) -> Dict[str, float]:
+        """Device times of the last step's stages (call after synchronising)."""
+        e = self.events
+        out = {"pack": e["begin"].elapsed_time(e["packed"]), "all_to_all": e["packed"].elapsed_time(e["arrived"]),
+               "reshard_remote": e["arrived"].elapsed_time(e["remote_done"]),
+               "reshard_local": e["local_begin"].elapsed_time(e["local_done"]), "step": e["begin"].elapsed_time(e["end"])}
+        return out
 
     def destroy(self) -> None:
-        if self.plan is not None:
-            self.plan.destroy()
-            self.plan = None
+        for name in ("plan_local", "plan_remote"):
+            p = getattr(self, name)
+            if p is not None:
+                p.destroy()
+                setattr(self, name, None)
+        self.send_buf = self.recv_buf = None
 
 
 def _local_targets(dst_metas: Sequence, dst_buf_bytes: Sequence[int], dst_owner: Sequence[int], rank: int):
@@ -137,8 +185,16 @@ def build_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner:
             metas.append(k)
         sizes.append(total)
     local_dst, mine, mine_bytes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
-    plan = api.bcp_plan(metas, sizes, mine, mine_bytes, **opts)
-    return Exchange(rank, world, local_src, local_dst, send_entries, send_offsets, send_bytes, recv_bytes, plan, sizes, mine_bytes)
+    n_local = len(local_src)
+    if len(sizes) == n_local:   # nothing is received: one plan does everything
+        plan_local, plan_remote = api.bcp_plan(metas, sizes, mine, mine_bytes, **opts), None
+    elif n_local == 0:          # the rank owns no blob: everything it reads arrives
+        plan_local, plan_remote = None, api.bcp_plan(metas, sizes, mine, mine_bytes, **opts)
+    else:
+        plan_local = api.bcp_plan(metas, sizes, mine, mine_bytes, src_buf_first=0, src_buf_count=n_local, **opts)
+        plan_remote = api.bcp_plan(metas, sizes, mine, mine_bytes, src_buf_first=n_local, src_buf_count=len(sizes) - n_local, **opts)
+    return Exchange(rank, world, local_src, local_dst, send_entries, send_offsets, send_bytes, recv_bytes, plan_local, plan_remote,
+                    sizes, mine_bytes)
 
 
 def plan_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: Sequence[int], dst_metas: Sequence,
@@ -158,43 +214,65 @@ def plan_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: 
 
 def pack_sends(x: Exchange, src_metas: Sequence, local_blobs: Sequence, send_buf, stream=None) -> None:
     """Step 3, sender side: the needed entries of this rank's blobs, one segment per receiver,
-    into `send_buf` (device, sum(send_bytes) bytes) with one multi-tensor pack."""
-    local_id = {b: i for i, b in enumerate(x.local_src)}
-    ptrs, metas, base = [], [], 0
-    for q in range(x.world):
-        for i, o in zip(x.send_entries[q], x.send_offsets[q]):
-            m = src_metas[i]
-            ptrs.append(local_blobs[local_id[m.buf_index]].data_ptr() + m.byte_offset)
-            metas.append((base + o, m.byte_length))
-        base += x.send_bytes[q]
-    if base:
-        api.bcp_pack(ptrs, metas, send_buf, base, stream=stream)
+    into `send_buf` (device, sum(send_bytes) bytes) with one multi-tensor pack.  The marshalled
+    argument arrays are kept for as long as the blobs stay where they are."""
+    key = tuple(b.data_ptr() for b in local_blobs)
+    if x.pack_args is None or x.pack_args[0] != key:
+        local_id = {b: i for i, b in enumerate(x.local_src)}
+        ptrs, metas, base = [], [], 0
+        for q in range(x.world):
+            for i, o in zip(x.send_entries[q], x.send_offsets[q]):
+                m = src_metas[i]
+                ptrs.append(key[local_id[m.buf_index]] + m.byte_offset)
+                metas.append((base + o, m.byte_length))
+            base += x.send_bytes[q]
+        x.pack_args = (key, api.marshal_pack(ptrs, metas), base)
+    _, args, total = x.pack_args
+    if total:
+        api.bcp_pack_marshalled(args, send_buf, total, stream=stream)
 
 
 def run_exchange(x: Exchange, src_metas: Sequence, local_blobs: Sequence, dst_bufs: Sequence, stream=None,
-                 all_to_all: Optional[Callable] = None):
-    """Steps 3 and 4 on the current device.  `all_to_all(recv, send, recv_splits, send_splits)`
-    defaults to `torch.distributed.all_to_all_single`; returns the buffers that must stay alive
-    until the stream has run (send buffer, receive buffer)."""
+                 all_to_all: Optional[Callable] = None) -> None:
+    """Steps 3 and 4 on the current device, asynchronous on `stream` (default: the current one).
+
+    Main stream: pack the outgoing segments -> all-to-all -> copy the pieces that arrived.
+    Side stream: once the pack has left the SMs, copy the pieces whose sources are this rank's own
+    blobs; it runs while the segments travel (the paper overlaps the transfer between GPUs with the
+    rest of the load pipeline, Sec. 4.1 / 4.2).  The main stream then waits for the side stream, so
+    that work queued on `stream` afterwards sees complete targets.  The pack goes first on purpose:
+    the copy kernels are persistent and fill every SM, so whatever is launched behind one waits for it.
+    `all_to_all(recv, send, recv_splits, send_splits)` defaults to `torch.distributed.all_to_all_single`
+    on `stream`.  Buffers, side stream and events live in the Exchange (x.bind); x.stage_ms() gives the
+    device time of every stage after a synchronise."""
     import torch
 
     dev = local_blobs[0].device if local_blobs else dst_bufs[0].device
-    send = torch.empty(max(1, sum(x.send_bytes)), dtype=torch.uint8, device=dev)
-    recv = torch.empty(max(1, sum(x.recv_bytes)), dtype=torch.uint8, device=dev)
-    pack_sends(x, src_metas, local_blobs, send, stream)
-    if x.world > 1:
-        if all_to_all is None:
-            import torch.distributed as dist
+    x.bind(dev)
+    main = torch.cuda.current_stream(dev) if stream is None else stream
+    e = x.events
+    srcs = x.sources(local_blobs)
+    with torch.cuda.stream(main):
+        e["begin"].record(main)
+        pack_sends(x, src_metas, local_blobs, x.send_buf, main)
+        e["packed"].record(main)
+        if x.world > 1:
+            if all_to_all is None:
+                import torch.distributed as dist
 
-            s = torch.cuda.current_stream() if stream is None else stream
-            with torch.cuda.stream(s):
-                dist.all_to_all_single(recv[: sum(x.recv_bytes)], send[: sum(x.send_bytes)], list(x.recv_bytes), list(x.send_bytes))
-        else:
-            all_to_all(recv, send, list(x.recv_bytes), list(x.send_bytes))
-    srcs, at = list(local_blobs), 0
-    for s in range(x.world):
-        if x.recv_bytes[s]:
-            srcs.append(recv[at:at + x.recv_bytes[s]])
-            at += x.recv_bytes[s]
-    api.bcp_reshard(x.plan, srcs, dst_bufs, stream=stream)
-    return send, recv
+                dist.all_to_all_single(x.recv_buf[: sum(x.recv_bytes)], x.send_buf[: sum(x.send_bytes)], list(x.recv_bytes),
+                                       list(x.send_bytes))
+            else:
+                all_to_all(x.recv_buf, x.send_buf, list(x.recv_bytes), list(x.send_bytes))
+        e["arrived"].record(main)
+        # the local pieces, behind the pack and beside the transfer
+        x.side.wait_event(e["packed"])
+        e["local_begin"].record(x.side)
+        if x.plan_local is not None:
+            api.bcp_reshard(x.plan_local, srcs, dst_bufs, stream=x.side)
+        e["local_done"].record(x.side)
+        if x.plan_remote is not None:
+            api.bcp_reshard(x.plan_remote, srcs, dst_bufs, stream=main)
+        e["remote_done"].record(main)
+        main.wait_event(e["local_done"])
+        e["end"].record(main)

@@ -90,7 +90,22 @@ EXCHANGE_WORKER = textwrap.dedent("""
                 srcs.append(recv[at:at + x.recv_bytes[s]].numpy())
                 at += x.recv_bytes[s]
         assert [len(s) for s in srcs] == x.src_buf_bytes
-        got, _ = run_tiles(x.plan.tiles(), srcs, x.dst_buf_bytes)
+        # the rank's work comes as two plans over the same buffer lists: pieces read from its own blobs and
+        # pieces read from received segments; between them every target byte is written exactly once
+        n_local = len(x.local_src)
+        units = []
+        for plan, lo, hi in ((x.plan_local, 0, n_local), (x.plan_remote, n_local, len(srcs))):
+            assert plan is not None
+            ts = plan.tiles()
+            assert ts and all(lo <= t.src_buf < hi for t in ts), case.name
+            units += ts
+        got, count = run_tiles(units, srcs, x.dst_buf_bytes)
+        named = [np.zeros(n, dtype=bool) for n in x.dst_buf_bytes]
+        for m in case.dst.metas:
+            if dst_owner[m.buf_index] == rank:
+                named[x.local_dst.index(m.buf_index)][m.byte_offset:m.byte_offset + m.byte_length] = True
+        for c, nm in zip(count, named):
+            assert np.array_equal(c, nm.astype(c.dtype)), (case.name, rank)
         want = orc.reshard(case.src.metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, convert=case.convert)
         assert len(x.local_dst) > 0 and sum(x.recv_bytes) > 0 and sum(x.send_bytes) > 0, case.name
         for g, b in zip(got, x.local_dst):
@@ -142,9 +157,10 @@ def test_exchange_schedule_properties_without_a_process_group():
                 assert set(x.send_entries[q]) <= set(needs[q])
                 assert all(src_owner[case.src.metas[i].buf_index] == r for i in x.send_entries[q])
                 assert x.send_bytes[q] % multi.SEGMENT_ALIGN == 0
-            # the final plan writes exactly this rank's target bytes
+            # the two final plans together write exactly this rank's target bytes
             mine = sum(m.byte_length for m in case.dst.metas if dst_owner[m.buf_index] == r)
-            assert x.plan.stats()["bytes_copied"] == mine
+            assert sum(p.stats()["bytes_copied"] for p in (x.plan_local, x.plan_remote) if p is not None) == mine
+            assert (x.plan_remote is None) == (sum(x.recv_bytes) == 0)
         # every needed entry is either local or sent by its owner, once
         for q in range(world):
             got = sorted(i for x in xs for i in x.send_entries[q]) + [i for i in needs[q] if src_owner[case.src.metas[i].buf_index] == q]

@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+import paper_2407_20143_b200 as bcp
 from paper_2407_20143_b200 import multi
 from oracle import reshard_oracle as orc
 from workloads import fills
@@ -50,11 +51,20 @@ def test_emulated_ranks_exchange_and_reshard(cuda_device, case, world):
                 at += recv_splits[s]
 
         dst = [torch.full((n,), POISON, dtype=torch.uint8, device=cuda_device) for n in x.dst_buf_bytes]
-        keep = multi.run_exchange(x, case.src.metas, [blobs[b] for b in x.local_src], dst, all_to_all=swap)
-        torch.cuda.synchronize()
-        for d, b in zip(dst, x.local_dst):
-            assert np.array_equal(d.cpu().numpy(), want[b]), (case.name, world, r, b)
-        del keep
+        for rep in range(2):  # the second step reuses the exchange's buffers, stream and marshalled pack
+            if rep:
+                for d in dst:
+                    d.fill_(POISON)
+            multi.run_exchange(x, case.src.metas, [blobs[b] for b in x.local_src], dst, all_to_all=swap)
+            torch.cuda.synchronize()
+            for p in (x.plan_local, x.plan_remote):
+                if p is not None:
+                    bcp.bcp_plan_device_status(p)
+            for d, b in zip(dst, x.local_dst):
+                assert np.array_equal(d.cpu().numpy(), want[b]), (case.name, world, r, b, rep)
+        ms = x.stage_ms()
+        assert set(ms) == {"pack", "all_to_all", "reshard_remote", "reshard_local", "step"} and ms["step"] > 0
+        assert (x.plan_remote is None) == (world == 1 or sum(x.recv_bytes) == 0)
     # every target buffer has exactly one owner
     assert sorted(b for x in xs for b in x.local_dst) == list(range(nd))
     if world > 1:  # bytes that crossed ranks: at most what the targets read, and none for a rank's own blobs

@@ -37,7 +37,7 @@ def test_struct_sizes_match_header():
 
     assert C.sizeof(_lib.TileC) == 64
     assert C.sizeof(_lib.ShardMetaC) == 8 + 16 + 3 * 64 + 16 + 8 + 16
-    assert C.sizeof(_lib.PlanOptsC) == 80
+    assert C.sizeof(_lib.PlanOptsC) == 88
     assert C.sizeof(_lib.PlanStatsC) == 14 * 8
 
 
@@ -614,3 +614,42 @@ def test_planning_from_several_threads_at_once():
     for t in threads:
         t.join()
     assert not failures, failures[:3]
+
+
+# ---- plans restricted to some source buffers (the two-plan form of the cross-rank exchange) -------
+@pytest.mark.parametrize("path_mask", [1, 3])
+def test_source_ranges_partition_the_work_list(path_mask):
+    """Plans for disjoint source-buffer ranges that cover all buffers hold, between them, exactly
+    the units of the unrestricted plan, each reads only its own range, and coverage is still
+    checked against every saved entry."""
+    for case in [c for c in scenario_cases() if c.name in ("hybrid", "llama-tp8-to-tp2", "dp150-to-dp75")] + [random_case(5, n_tensors=4)]:
+        ns = len(case.src.buf_bytes)
+        args = (case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+        opts = dict(case.plan_opts, path_mask=path_mask, tile_bytes=8192)
+        whole = bcp.bcp_plan(*args, **opts)
+        key = lambda t: (t.src_buf, t.src_off, t.dst_buf, t.dst_off, t.rows, t.row_bytes, t.src_pitch, t.dst_pitch)  # noqa: E731
+        want = sorted(key(t) for t in whole.tiles())
+        for cuts in ([0, ns], [0, 1, ns], [0, ns // 2, ns], [0, ns // 3, ns - 1, ns]):
+            cuts = sorted(set(cuts))
+            got, copied, uniq = [], 0, 0
+            for lo, hi in zip(cuts[:-1], cuts[1:]):
+                part = bcp.bcp_plan(*args, src_buf_first=lo, src_buf_count=hi - lo, **opts)
+                ts = part.tiles()
+                assert all(lo <= t.src_buf < hi for t in ts)
+                got += [key(t) for t in ts]
+                copied += part.stats()["bytes_copied"]
+                uniq += part.stats()["bytes_src_unique"]
+                part.destroy()
+            assert sorted(got) == want, (case.name, cuts)
+            assert copied == whole.stats()["bytes_copied"] and uniq == whole.stats()["bytes_src_unique"]
+        whole.destroy()
+    # a restricted plan still refuses a target that the saved entries as a whole do not cover
+    case = [c for c in scenario_cases() if c.name == "hybrid"][0]
+    fewer = [m for m in case.src.metas if m.buf_index != 0]
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.bcp_plan(fewer, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, src_buf_first=1, src_buf_count=1)
+    assert e.value.code == api.ERR_UNCOVERED
+    for first, count in ((1, 0), (0, len(case.src.buf_bytes) + 1), (len(case.src.buf_bytes), 1)):
+        with pytest.raises(bcp.BcpError) as e:
+            bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, src_buf_first=first, src_buf_count=count)
+        assert e.value.code == api.ERR_INVALID
