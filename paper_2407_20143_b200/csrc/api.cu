@@ -1,6 +1,8 @@
 // C ABI of the resharding engine: plan objects, execution, pack / unpack.
 // (Plan images are in plan_image.cu, the host-buffer call in host_path.cu.)
 #include <chrono>
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 #include <new>
 
@@ -9,6 +11,13 @@
 using namespace bcp;
 
 namespace bcp {
+
+constexpr int kControls = 4;  // control blocks of a plan, one per kernel
+// Stage geometry of the staged converting kernel.  The warp converts out of shared memory itself,
+// so what counts is how many warps an SM has at work: six one-warp CTAs with two 16 KiB stages each
+// (192 KiB of shared memory per SM, like the copy) measured best on the full-size 8B merge
+// (7.02 ms; four CTAs with three stages 7.61 ms, two CTAs with three 32 KiB stages 11.6 ms).
+constexpr uint32_t kCvtStageBytes = 16384, kCvtStages = 2, kCvtCtasPerSm = 6;
 
 int bind_device_alloc(bcp_plan_t* p) {
   const size_t n_ptrs = p->src_bytes.size() + p->dst_bytes.size();
@@ -21,8 +30,8 @@ int bind_device_alloc(bcp_plan_t* p) {
     BCP_CUDA(cudaMalloc(&p->d_maps, p->rects.size() * 2 * sizeof(CUtensorMap)));
     p->h_maps.resize(p->rects.size() * 2);
   }
-  BCP_CUDA(cudaMalloc(&p->d_ctrl, 3 * sizeof(Control)));
-  BCP_CUDA(cudaMemset(p->d_ctrl, 0, 3 * sizeof(Control)));
+  BCP_CUDA(cudaMalloc(&p->d_ctrl, kControls * sizeof(Control)));
+  BCP_CUDA(cudaMemset(p->d_ctrl, 0, kControls * sizeof(Control)));
   if (p->opt.worker == 2) {
     BCP_CUDA(warp_kernel_max_grid(p->opt.ctas_per_sm, &p->grid));
   } else {
@@ -30,7 +39,21 @@ int bind_device_alloc(bcp_plan_t* p) {
   }
   if (p->n_tma)
     BCP_CUDA(tma_kernel_max_grid(p->opt.tma_stage_bytes, p->opt.tma_stages, p->opt.tma_ctas_per_sm, &p->tma_grid));
-  if (p->n_cvt) BCP_CUDA(convert_kernel_max_grid(&p->cvt_grid));
+  if (p->n_cvt) {
+    BCP_CUDA(convert_kernel_max_grid(&p->cvt_grid));
+    p->n_cvt_staged = 0;
+    for (size_t i = p->tiles.size() - p->n_cvt; i < p->tiles.size(); ++i) p->n_cvt_staged += (p->tiles[i].flags & BCP_TILE_TMA) != 0;
+    if (p->n_cvt_staged) {
+      p->cvt_stage_bytes = kCvtStageBytes, p->cvt_stages = kCvtStages;
+      uint32_t per_sm = kCvtCtasPerSm;
+      if (const char* g = getenv("BCP_CVT_GEOMETRY")) {  // tuning override: "stage_bytes,stages,ctas_per_sm"
+        unsigned a = 0, b = 0, c = 0;
+        if (sscanf(g, "%u,%u,%u", &a, &b, &c) == 3 && a >= 1024 && a % 128 == 0 && b >= 2 && b <= 8 && c >= 1 && c <= 16)
+          p->cvt_stage_bytes = a, p->cvt_stages = b, per_sm = c;
+      }
+      BCP_CUDA(convert_staged_max_grid(p->cvt_stage_bytes, p->cvt_stages, per_sm, &p->cvt_staged_grid));
+    }
+  }
   p->h_ptrs.resize(n_ptrs);
   return BCP_OK;
 }
@@ -152,7 +175,22 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
   a.cache_hints = p->opt.cache_hints;
   a.unroll = p->opt.unroll;
   if (units) BCP_CUDA(launch_copy(a, stream));
-  if (n_cvt) {
+  // converting units: both kernels walk the same list; the staged one takes the units marked
+  // BCP_TILE_TMA, the register one the rest (a kernel that would find nothing is not launched)
+  if (n_cvt && p->n_cvt_staged) {
+    ConvertStagedLaunchArgs c;
+    c.tiles = tiles + n_tma + n_big + n_small;
+    c.n_units = uint32_t(n_cvt);
+    c.src = a.src;
+    c.dst = a.dst;
+    c.ctrl = p->d_ctrl + 3;
+    c.stage_bytes = p->cvt_stage_bytes;
+    c.n_stages = p->cvt_stages;
+    c.grid = p->cvt_staged_grid;
+    c.wait_ns = uint64_t(p->opt.tma_wait_ms) * 1000000ull;
+    BCP_CUDA(launch_convert_staged(c, stream));
+  }
+  if (n_cvt && p->n_cvt_staged < p->n_cvt) {
     ConvertLaunchArgs c;
     c.tiles = tiles + n_tma + n_big + n_small;
     c.n_units = uint32_t(n_cvt);
@@ -457,12 +495,14 @@ int bcp_plan_device_status(bcp_plan_t* plan, void* stream) {
   if (!plan) return fail(BCP_ERR_INVALID, "plan is NULL");
   if (plan->device < 0) return BCP_OK;
   BCP_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-  Control c[2];
+  Control c[kControls];
   BCP_CUDA(cudaMemcpy(c, plan->d_ctrl, sizeof c, cudaMemcpyDeviceToHost));
-  const uint32_t status = c[0].status ? c[0].status : c[1].status;
+  uint32_t status = 0;
+  for (const Control& k : c)
+    if (!status) status = k.status;
   if (status) {
     BCP_CUDA(cudaMemset(plan->d_ctrl, 0, sizeof c));  // counters of an aborted launch are stale: start clean
-    return fail(BCP_ERR_DEVICE_TIMEOUT, "a bounded wait of the TMA staging kernel gave up (device status %d); "
+    return fail(BCP_ERR_DEVICE_TIMEOUT, "a bounded wait of a staging kernel gave up (device status %d); "
                 "the targets of that execution are incomplete", int(status));
   }
   return BCP_OK;

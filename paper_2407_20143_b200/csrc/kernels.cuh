@@ -57,6 +57,24 @@ struct ConvertLaunchArgs {
   uint32_t grid;
 };
 
+struct ConvertStagedLaunchArgs {
+  const bcp_tile* tiles;  // device: the same n_units converting units; this kernel takes those marked BCP_TILE_TMA
+  uint32_t n_units;
+  const void* const* src;
+  void* const* dst;
+  Control* ctrl;          // device, separate from the other kernels'
+  uint32_t stage_bytes;   // shared-memory stage, multiple of 128
+  uint32_t n_stages;      // 2..8
+  uint32_t grid;
+  uint64_t wait_ns;       // how long a CTA waits for one stage before it gives up (global timer)
+};
+
+// Persistent grid of the staged converting kernel (one warp per CTA) for a stage geometry.
+cudaError_t convert_staged_max_grid(uint32_t stage_bytes, uint32_t n_stages, uint32_t ctas_per_sm, uint32_t* grid);
+
+// Enqueue the staged converting kernel on `stream`.
+cudaError_t launch_convert_staged(const ConvertStagedLaunchArgs& a, cudaStream_t stream);
+
 // Persistent grid of the converting kernel (256-thread CTAs, every warp a worker).
 cudaError_t convert_kernel_max_grid(uint32_t* grid);
 

@@ -27,7 +27,8 @@ bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vect
   if (t.rows == 0 || t.row_bytes == 0 || t.dst_buf >= db.size()) return false;
   if (const uint32_t kind = (t.flags & BCP_TILE_CVT_MASK) >> BCP_TILE_CVT_SHIFT) {
     // converting unit: element-aligned on both sides, source rows hold the same number of elements
-    if (kind > BCP_CONVERT_BF16_TO_F32 || (t.flags & ~(BCP_TILE_GRAN_MASK | BCP_TILE_CVT_MASK)) || t.src_buf >= sb.size()) return false;
+    if (kind > BCP_CONVERT_BF16_TO_F32 || (t.flags & ~(BCP_TILE_GRAN_MASK | BCP_TILE_CVT_MASK | BCP_TILE_TMA)) || t.src_buf >= sb.size())
+      return false;
     const uint64_t s_isz = kind == BCP_CONVERT_F32_TO_BF16 ? 4 : 2, d_isz = 6 - s_isz;
     const uint64_t s_row = uint64_t(t.row_bytes) / d_isz * s_isz;
     if (t.row_bytes % d_isz || t.dst_off % d_isz || t.dst_pitch % d_isz || t.src_off % s_isz || t.src_pitch % s_isz) return false;
@@ -35,6 +36,8 @@ bool tile_ok(const bcp_tile& t, const std::vector<uint64_t>& sb, const std::vect
     const uint64_t span_d = uint64_t(t.rows - 1) * t.dst_pitch + t.row_bytes, span_s = uint64_t(t.rows - 1) * t.src_pitch + s_row;
     if (t.dst_off > db[t.dst_buf] || span_d > db[t.dst_buf] - t.dst_off) return false;
     if (t.src_off > sb[t.src_buf] || span_s > sb[t.src_buf] - t.src_off) return false;
+    // staged conversion fetches the 16-byte aligned superset of every source row
+    if ((t.flags & BCP_TILE_TMA) && (s_row < 16 || ((t.src_off + span_s + 15) & ~uint64_t(15)) > sb[t.src_buf])) return false;
     return uint64_t(t.rows) * t.row_bytes <= opt.tile_bytes;
   }
   const bool zero = t.flags & BCP_TILE_ZERO;
@@ -207,7 +210,7 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   for (size_t i = 0; i < p->tiles.size(); ++i) {
     const bcp_tile& t = p->tiles[i];
     const bool in_tma = i < p->n_tma, in_cvt = i >= p->tiles.size() - p->n_cvt, in_small = i >= p->n_tma + p->n_big && !in_cvt;
-    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->rects, p->opt) || bool(t.flags & BCP_TILE_TMA) != in_tma ||
+    if (!tile_ok(t, p->src_bytes, p->dst_bytes, p->rects, p->opt) || (!in_cvt && bool(t.flags & BCP_TILE_TMA) != in_tma) ||
         bool(t.flags & BCP_TILE_SMALL) != in_small || bool(t.flags & BCP_TILE_CVT_MASK) != in_cvt) {
       delete p;
       return fail(BCP_ERR_INVALID, "bcp_plan_deserialize: work unit %zu is inconsistent with the recorded buffers", i);

@@ -26,8 +26,10 @@ struct bcp_plan_s {
   bcp_tile* d_tiles = nullptr;
   bcp_tile* d_fan_tiles = nullptr;  // the same list with replica groups marked (in-place host path)
   void** d_ptrs = nullptr;  // source table followed by target table
-  bcp::Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel, [2] converting kernel
-  uint32_t grid = 0, tma_grid = 0, cvt_grid = 0;
+  bcp::Control* d_ctrl = nullptr;  // [0] register kernel, [1] TMA kernel, [2] converting kernel, [3] staged converting kernel
+  uint32_t grid = 0, tma_grid = 0, cvt_grid = 0, cvt_staged_grid = 0;
+  uint32_t cvt_stage_bytes = 0, cvt_stages = 0;  // stage geometry of the staged converting kernel
+  size_t n_cvt_staged = 0;  // converting units marked for the staged kernel (counted when the plan is bound)
   cudaStream_t last_stream = nullptr;
   cudaEvent_t ev_switch = nullptr;  // orders an execution after the previous one when the stream changes
   bool ran = false;

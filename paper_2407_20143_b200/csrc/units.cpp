@@ -28,9 +28,11 @@ struct Tally {
   uint64_t tma_busy = 0;    // ... in shifted runs and rectangles with rows under 2 KiB (the warp issues a lot)
   uint64_t tma_boxed = 0;   // ... in tensor-map boxes
   uint64_t cvt_bytes = 0;   // target bytes written by converting units
+  uint64_t cvt_staged = 0;  // source + target bytes of converting units that qualify for the staged kernel
   void add(const Tally& o) {
     bytes_copied += o.bytes_copied, bytes_misaligned += o.bytes_misaligned, n_strided += o.n_strided;
     tma_bytes += o.tma_bytes, tma_busy += o.tma_busy, tma_boxed += o.tma_boxed, cvt_bytes += o.cvt_bytes;
+    cvt_staged += o.cvt_staged;
   }
 };
 
@@ -40,6 +42,7 @@ struct Cutter {
   const Options& opt;
   const std::vector<uint64_t>* src_bytes;  // source buffer sizes (may be null: unknown)
   bool demote;                             // small job: TMA-eligible units go to the register kernel
+  bool demote_cvt;                         // small converting job: no unit is marked for the staged converting kernel
   bcp_tile* out[kClasses];
   Rect* rects_out;
   size_t pos[kClasses];
@@ -172,7 +175,9 @@ struct Cutter {
     return true;
   }
 
-  // Converting units: rows x row_bytes TARGET bytes each; no staging path, no warp path.
+  // Converting units: rows x row_bytes TARGET bytes each; no warp path.  A unit whose source rows
+  // are long enough, and whose 16-byte aligned supersets stay inside the source buffer, is marked
+  // BCP_TILE_TMA: the staged converting kernel takes it, the register one skips it.
   void emit_cvt(const Item& it, uint64_t src_off, uint64_t dst_off, uint64_t rows, uint64_t row_bytes) {
     bcp_tile t;
     memset(&t, 0, sizeof t);
@@ -192,6 +197,16 @@ struct Cutter {
     if (g < 4) st.bytes_misaligned += rows * row_bytes;
     st.bytes_copied += rows * row_bytes;
     st.cvt_bytes += rows * row_bytes;
+    const uint64_t src_row = it.cvt == BCP_CONVERT_F32_TO_BF16 ? row_bytes * 2 : row_bytes / 2;
+    bool staged = opt.path_mask != 1 && src_row >= opt.tma_min_row_bytes;
+    if (staged) {
+      const uint64_t end16 = (src_off + (rows - 1) * (rows > 1 ? it.src_pitch : 0) + src_row + 15) & ~uint64_t(15);
+      staged = src_bytes && it.src_buf < src_bytes->size() && end16 <= (*src_bytes)[it.src_buf];
+    }
+    if (staged) {
+      st.cvt_staged += rows * (row_bytes + src_row);
+      if (!demote_cvt) t.flags |= BCP_TILE_TMA;
+    }
     put(kCvt, t);
   }
 
@@ -323,7 +338,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   const size_t kBlock = 16;
   std::vector<Tally> tally((n_items + kBlock - 1) / kBlock);
   parallel_jobs(tally.size(), threads, [&](size_t j) {
-    Cutter c{opt, src_bytes, false, {nullptr, nullptr, nullptr, nullptr}, nullptr, {0, 0, 0, 0}, 0, Tally()};
+    Cutter c{opt, src_bytes, false, false, {nullptr, nullptr, nullptr, nullptr}, nullptr, {0, 0, 0, 0}, 0, Tally()};
     for (size_t i = j * kBlock; i < std::min(n_items, (j + 1) * kBlock); ++i) {
       const Count before = {{c.pos[0], c.pos[1], c.pos[2], c.pos[3]}, c.rect_pos};
       c.cut(merged[i]);
@@ -340,6 +355,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     for (size_t i = 0; i < n_items; ++i) cnt[i].n[kBig] += cnt[i].n[kTma], cnt[i].n[kTma] = 0, cnt[i].rects = 0;
     all.tma_bytes = all.tma_busy = all.tma_boxed = 0;
   }
+  const bool demote_cvt = opt.path_mask == 0 && all.cvt_staged < (128u << 20);
   Count run = {{0, 0, 0, 0}, 0};  // counts -> positions of each item's first unit inside its class
   for (size_t i = 0; i <= n_items; ++i) {
     const Count c = i < n_items ? cnt[i] : Count{{0, 0, 0, 0}, 0};
@@ -364,7 +380,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   }
   parallel_jobs(cuts.size() - 1, threads, [&](size_t j) {
     const Count& at = cnt[cuts[j]];
-    Cutter c{opt, src_bytes, demote, {cls[0], cls[1], cls[2], cls[3]}, rc.data(), {at.n[0], at.n[1], at.n[2], at.n[3]}, at.rects, Tally()};
+    Cutter c{opt, src_bytes, demote, demote_cvt, {cls[0], cls[1], cls[2], cls[3]}, rc.data(), {at.n[0], at.n[1], at.n[2], at.n[3]}, at.rects, Tally()};
     for (size_t i = cuts[j]; i < cuts[j + 1]; ++i) c.cut(merged[i]);
   });
   stats->bytes_copied = all.bytes_copied;

@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import paper_2407_20143_b200 as bcp
+from paper_2407_20143_b200 import api
 from oracle import reshard_oracle as orc
 from workloads import fills
 from workloads.configs import CONFIGS, STRESS, convert_cases, scenario_cases
@@ -543,14 +544,21 @@ def test_plans_run_from_several_threads_on_their_own_streams(cuda_device):
 
 
 # ---- element conversion (extension) --------------------------------------------------------------
+# kernel: the default keeps jobs this small on the register kernel; path_mask 3 sends every source row of
+# at least tma_min_row_bytes through the staged kernel (16: nearly all of them, 512: a mix of both kernels)
+CVT_PATHS = {"register": {}, "staged": {"path_mask": 3, "tma_min_row_bytes": 16}, "mixed": {"path_mask": 3, "tma_min_row_bytes": 512}}
+
+
+@pytest.mark.parametrize("path", list(CVT_PATHS))
 @pytest.mark.parametrize("fill", ["index", "uniform"])
 @pytest.mark.parametrize("case", convert_cases(), ids=lambda c: c.name)
-def test_converting_reshard(cuda_device, case, fill):
-    st = run_and_compare(case, cuda_device, fill, runs=2, tile_bytes=4096 if fill == "index" else 65536)
+def test_converting_reshard(cuda_device, case, fill, path):
+    st = run_and_compare(case, cuda_device, fill, runs=2, tile_bytes=4096 if fill == "index" else 65536, **CVT_PATHS[path])
     assert st["n_cvt_tiles"] > 0
 
 
-def test_converting_reshard_every_bit_pattern_and_alignment(cuda_device):
+@pytest.mark.parametrize("path", ["register", "staged"])
+def test_converting_reshard_every_bit_pattern_and_alignment(cuda_device, path):
     """All 2^32 binary32 patterns are too many; all 2^16 upper halves times the lower halves around
     the halfway point are not (every exponent, every tie, NaNs, infinities), and rows that start
     at every element phase exercise the leading / body / tail split of the kernel."""
@@ -569,7 +577,10 @@ def test_converting_reshard_every_bit_pattern_and_alignment(cuda_device):
         pos += m.byte_length + (2 if (b - a) % 2 else 6)  # odd gaps: targets start at odd element offsets too
     blob = torch.from_numpy(bits.view(np.uint8).copy()).to(cuda_device)
     want = orc.reshard(src_meta, [bits.view(np.uint8)], dst_meta, [pos], fill_byte=POISON, convert=(1, 2, 1))[0]
-    plan = bcp.bcp_plan(src_meta, [n * 4], dst_meta, [pos], convert=1, convert_src_tag=2, convert_dst_tag=1, tile_bytes=8192)
+    plan = bcp.bcp_plan(src_meta, [n * 4], dst_meta, [pos], convert=1, convert_src_tag=2, convert_dst_tag=1, tile_bytes=8192,
+                        **CVT_PATHS[path])
+    staged = sum(1 for t in plan.tiles() if t.flags & api.TILE_TMA)
+    assert (staged > 0) == (path == "staged")
     dst, backs = guarded([pos], cuda_device)
     bcp.bcp_reshard(plan, [blob], dst)
     torch.cuda.synchronize()
@@ -582,7 +593,7 @@ def test_converting_reshard_every_bit_pattern_and_alignment(cuda_device):
     dst_meta = [ShardMeta("h", 4, 2, (1 << 16,), (a,), (b - a,), 0, 4 * a + 4) for a, b in ((0, 3), (3, 40001), (40001, 1 << 16))]
     total = 4 * (1 << 16) + 4
     want = orc.reshard(src_meta, [h.view(np.uint8)], dst_meta, [total], fill_byte=POISON, convert=(2, 1, 2))[0]
-    plan = bcp.bcp_plan(src_meta, [h.nbytes], dst_meta, [total], convert=2, convert_src_tag=1, convert_dst_tag=2)
+    plan = bcp.bcp_plan(src_meta, [h.nbytes], dst_meta, [total], convert=2, convert_src_tag=1, convert_dst_tag=2, **CVT_PATHS[path])
     dst, backs = guarded([total], cuda_device)
     bcp.bcp_reshard(plan, [torch.from_numpy(h.view(np.uint8).copy()).to(cuda_device)], dst)
     torch.cuda.synchronize()

@@ -89,7 +89,7 @@ def run_tiles(tiles, src, dst_sizes, poison=0xA5):
         assert t.dst_off % g == 0 and t.row_bytes % g == 0 and t.dst_pitch % g == 0
         kind = (t.flags & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
         if kind:  # converting unit: row_bytes counts target bytes, the source row holds the same elements
-            assert not t.flags & (api.TILE_ZERO | api.TILE_SMALL | api.TILE_TMA | api.TILE_TMA2D | api.TILE_FOLLOW)
+            assert not t.flags & (api.TILE_ZERO | api.TILE_SMALL | api.TILE_TMA2D | api.TILE_FOLLOW)
             s_isz, d_isz = (4, 2) if kind == api.CONVERT_F32_TO_BF16 else (2, 4)
             assert t.row_bytes % d_isz == 0 and t.dst_off % d_isz == 0 and t.src_off % s_isz == 0
             n = t.row_bytes // d_isz
