@@ -46,7 +46,7 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     ("cfg2", "bcp_tma_kernel"): (0.9994, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369", "full size"),
     ("cfg3", "bcp_tma_kernel"): (0.9990, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369", "full size"),
     ("cfg4", "bcp_tma_kernel"): (0.9998, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "0874854", "full size"),
-    ("evalmerge", "bcp_convert_kernel"): (0.9961, "profiles/bcp_convert_staged_kernel_evalmerge-L2_ncu_full.md", "this file's commit", "2 layers (8.9 GB)"),
+    ("evalmerge", "bcp_convert_kernel"): (0.9961, "profiles/bcp_convert_staged_kernel_evalmerge-L2_ncu_full.md", "4f5ee6b", "2 layers (8.9 GB)"),
 }
 
 
