@@ -526,8 +526,7 @@ def run_exchange_bench(a):
     sent = D.max_over_ranks(float(sum(x.send_bytes)), dev)
     recv = D.max_over_ranks(float(sum(x.recv_bytes)), dev)
     value = total_bytes / (ms_step * 1e-3) / 1e9
-    n_kernels = sum(int(p.stats()["n_tma_tiles"] > 0) + int(p.stats()["n_tiles"] - p.stats()["n_tma_tiles"] + p.stats()["n_small_tiles"] > 0)
-                    + int(p.stats()["n_cvt_tiles"] > 0) for p in plans) + (2 if sum(x.send_bytes) else 0)
+    n_kernels = sum(p.stats()["n_kernels"] for p in plans) + (2 if sum(x.send_bytes) else 0)
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": a.steps, "warmup": max(a.warmup, 3),
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "u8",
            "data": "synthetic",
@@ -575,9 +574,7 @@ def main():
     # kernels enqueued by one bcp_reshard: the TMA staging kernel (if any unit qualifies) and the
     # register kernel (if any unit is left for it)
     n_tma = st["n_tma_tiles"]
-    n_reg = st["n_tiles"] - n_tma + st["n_small_tiles"]
-    n_cvt = st["n_cvt_tiles"]
-    kernels_per_step = int(n_tma > 0) + int(n_reg > 0) + int(n_cvt > 0)
+    kernels_per_step = st["n_kernels"]
     dominant = "bcp_convert_kernel" if case.convert else "bcp_tma_kernel" if n_tma > 0 else "bcp_copy_kernel"
     peak, peak_kind = measured_peak()
     avg_launch_ms = sum(launch_ms) / len(launch_ms)
@@ -671,8 +668,7 @@ def main():
                                 "frac": f3["b_min"] / (mean3 * 1e-3) / 1e9 / peak, "peak_source": f"of {peak_kind}",
                                 "pct_of_8tbs_nominal": gbs3 / ws / 8000.0 * 100.0, "verified": f3["verified"],
                                 "verified_bytes": f3["verified_bytes"], "clocks": f3["clocks"],
-                                "gpu_launches": a.steps * (int(f3["st"]["n_tma_tiles"] > 0) +
-                                                           int(f3["st"]["n_tiles"] - f3["st"]["n_tma_tiles"] + f3["st"]["n_small_tiles"] > 0))}}
+                                "gpu_launches": a.steps * f3["st"]["n_kernels"]}}
         p3.destroy()
         del s3, d3
     if rank == 0:

@@ -120,8 +120,10 @@ typedef struct {
                                 with 2-D tensor-map copies (cp.async.bulk.tensor.2d, one command per box of
                                 up to 256 rows) instead of one bulk copy per row; their descriptors are
                                 re-encoded on the host whenever a buffer address changes;
-                              0 default: 7 when at least 128 MiB of payload qualifies for TMA staging, else 1
-                                (small jobs are launch-bound and one kernel is cheaper than two)            */
+                              0 default: 7 when at least 4 MiB of payload qualifies for TMA staging, else 1
+                                (measured: from there on the staging kernel is the faster one; when all that
+                                is left for the register kernel are a few thousand units under small_bytes,
+                                the staging kernel's warps copy those too and one kernel is launched)        */
   uint32_t cache_hints;    /* 0 default (= 1); register path: 1 streaming loads and stores, 2 plain accesses;
                               TMA path: 3 evict-first L2 hint on stores, 4 on loads too, else no hint    */
   uint32_t tma_stage_bytes; /* TMA path: bytes per shared-memory stage, multiple of 128; default 32768, or
@@ -235,6 +237,9 @@ typedef struct {
   uint64_t bytes_misaligned; /* payload in units whose access granularity is < 16 B   */
   double plan_ms;            /* host time spent in bcp_plan                           */
   uint64_t n_cvt_tiles;      /* converting work units (bcp_plan_opts.convert)         */
+  uint64_t n_kernels;        /* kernels one bcp_reshard of this plan launches (1..4): the staging kernel (which
+                                also takes a short rest of unstaged units), the register kernel (a long rest),
+                                the staged and the register converting kernel                                 */
 } bcp_plan_stats_t;
 
 /* ByteMeta of one tensor inside a packed blob (Sec. 3.2): start offset and length. */

@@ -74,7 +74,7 @@ class PlanStatsC(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "n_src_entries", "n_dst_entries", "n_fqns", "n_intersections", "n_items", "n_tiles", "n_small_tiles",
         "n_strided_tiles", "n_tma_tiles", "bytes_copied", "bytes_src_unique", "bytes_misaligned")] + [
-        ("plan_ms", C.c_double), ("n_cvt_tiles", C.c_uint64)]
+        ("plan_ms", C.c_double), ("n_cvt_tiles", C.c_uint64), ("n_kernels", C.c_uint64)]
 
 
 class ExportEntryC(C.Structure):

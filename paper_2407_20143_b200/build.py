@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libbcp.so")
 SOURCES = ["planner.cpp", "units.cpp", "api.cu", "plan_image.cu", "host_path.cu", "kernels.cu", "tma_kernel.cu", "convert_kernel.cu", "static_pack.cu", "stager.cu", "export.cu"]
-HEADERS = ["plan.hpp", "kernels.cuh", "host_threads.hpp", "plan_object.hpp", "tma_ptx.cuh"]
+HEADERS = ["plan.hpp", "kernels.cuh", "host_threads.hpp", "plan_object.hpp", "tma_ptx.cuh", "copy_loops.cuh"]
 
 
 def nvcc_path() -> str:

@@ -12,6 +12,10 @@ using namespace bcp;
 
 namespace bcp {
 
+// Only warp units (under 4 KiB each) ride along: one warp copies such a unit in a round trip or two,
+// while a CTA-wide unit of 64 KiB would keep a single warp busy for tens of microseconds.
+constexpr size_t kFoldMaxSmall = 8192;
+inline bool folds(size_t n_tma, size_t n_big, size_t n_small) { return n_tma && n_big == 0 && n_small > 0 && n_small <= kFoldMaxSmall; }
 constexpr int kControls = 4;  // control blocks of a plan, one per kernel
 // Stage geometry of the staged converting kernel.  The warp converts out of shared memory itself,
 // so what counts is how many warps an SM has at work: six one-warp CTAs with two 16 KiB stages each
@@ -139,10 +143,14 @@ int upload_tables(bcp_plan_t* p, cudaStream_t stream) {
 int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_big, size_t n_small, size_t n_cvt,
                  cudaStream_t stream) {
   const size_t ns = p->src_bytes.size();
+  // A rest of nothing but a few thousand warp units rides along in the staging kernel (one launch
+  // instead of two); anything more is better served by the register kernel's many warps.
+  const bool fold = folds(n_tma, n_big, n_small);
   if (n_tma) {
     TmaLaunchArgs t;
     t.tiles = tiles;
     t.n_tiles = uint32_t(n_tma);
+    t.n_tail = fold ? uint32_t(n_big + n_small) : 0u;
     t.src = reinterpret_cast<const void* const*>(p->d_ptrs);
     t.dst = reinterpret_cast<void* const*>(p->d_ptrs + ns);
     t.ctrl = p->d_ctrl + 1;
@@ -174,7 +182,7 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
   a.grid = uint32_t(ctas < p->grid ? ctas : p->grid);
   a.cache_hints = p->opt.cache_hints;
   a.unroll = p->opt.unroll;
-  if (units) BCP_CUDA(launch_copy(a, stream));
+  if (units && !fold) BCP_CUDA(launch_copy(a, stream));
   // converting units: both kernels walk the same list; the staged one takes the units marked
   // BCP_TILE_TMA, the register one the rest (a kernel that would find nothing is not launched)
   if (n_cvt && p->n_cvt_staged) {
@@ -475,6 +483,11 @@ int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_by
 int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out) {
   if (!plan || !out) return fail(BCP_ERR_INVALID, "bcp_plan_stats: NULL argument");
   *out = plan->stats;
+  size_t staged = 0;
+  for (size_t i = plan->tiles.size() - plan->n_cvt; i < plan->tiles.size(); ++i) staged += (plan->tiles[i].flags & BCP_TILE_TMA) != 0;
+  const size_t rest = plan->n_big + plan->n_small();
+  out->n_kernels = (plan->n_tma > 0) + (rest > 0 && !folds(plan->n_tma, plan->n_big, plan->n_small())) + (staged > 0) +
+                   (staged < plan->n_cvt);
   return BCP_OK;
 }
 

@@ -36,6 +36,7 @@ struct LaunchArgs {
 struct TmaLaunchArgs {
   const bcp_tile* tiles;  // device: n_tiles units, all eligible for bulk copies
   uint32_t n_tiles;
+  uint32_t n_tail;        // units right behind them in the list that the warps copy through registers
   const void* const* src;
   void* const* dst;
   Control* ctrl;          // device, separate from the register kernel's

@@ -25,7 +25,13 @@
 // (source view, target view; 8-byte elements, no swizzle) live in global memory, are encoded
 // by the host for the buffer addresses of the call, and are read through the tensormap proxy
 // after an acquire fence.
+//
+// The few units of a plan that cannot be staged (pieces under 4 KiB, short unaligned rows, zero
+// fills) may ride along as a tail of the ticket range: whoever draws such a ticket copies the
+// unit with the warp's own loads and stores while its staged chunks are in flight, which saves a
+// second kernel launch behind this one.
 #include "kernels.cuh"
+#include "copy_loops.cuh"
 #include "tma_ptx.cuh"
 
 namespace bcp {
@@ -172,7 +178,7 @@ __device__ __forceinline__ void warp_store_out(const unsigned char* smem, char* 
   for (; i < ne; i += 32) __stcs(dv + i, sv[i]);
 }
 
-__global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles,
+__global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_tiles, uint32_t n_tail,
                                                      const void* const* __restrict__ src, void* const* __restrict__ dst,
                                                      Control* ctrl, uint32_t stage_bytes, uint32_t n_stages,
                                                      uint64_t wait_ns, uint32_t hints, const unsigned char* maps,
@@ -204,11 +210,17 @@ __global__ void __launch_bounds__(32) bcp_tma_kernel(const bcp_tile* __restrict_
     while (!cur.live) {
       if (drained) return false;
       const uint32_t ticket = __shfl_sync(0xffffffffu, pending, 0);
-      if (ticket >= n_tiles) {
+      if (ticket >= n_tiles + n_tail) {
         drained = true;
         return false;
       }
       const bcp_tile* t = tiles + ticket;
+      if (ticket >= n_tiles) {  // a unit of the tail: copied through registers, here and now
+        if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
+        const bcp_tile u = load_tile(t);
+        copy_tile<2, 1, 32>(u, src, dst, lane);
+        continue;
+      }
       const uint4 e = __ldg(reinterpret_cast<const uint4*>(t) + 3);  // flags, reserved[0..2]
       if (e.x & BCP_TILE_FOLLOW) {  // written by the CTA that stages the head of its group
         if (lane == 0) pending = atomicAdd(&ctrl->ticket, 1u);
@@ -465,7 +477,7 @@ cudaError_t launch_tma(const TmaLaunchArgs& a, cudaStream_t stream) {
   if (a.n_tiles == 0) return cudaSuccess;
   if (a.n_stages < 2 || a.n_stages > kMaxStages || a.stage_bytes % 128 || a.stage_bytes == 0) return cudaErrorInvalidValue;
   const size_t smem = size_t(a.stage_bytes) * a.n_stages;
-  bcp_tma_kernel<<<a.grid, 32, smem, stream>>>(a.tiles, a.n_tiles, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages,
+  bcp_tma_kernel<<<a.grid, 32, smem, stream>>>(a.tiles, a.n_tiles, a.n_tail, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages,
                                                a.wait_ns, a.cache_hints, static_cast<const unsigned char*>(a.maps),
                                                a.test_stall);
   return cudaGetLastError();

@@ -349,8 +349,11 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   });
   Tally all;
   for (const Tally& t : tally) all.add(t);
-  // small jobs are launch-bound: keep them in one kernel
-  const bool demote = opt.path_mask == 0 && all.tma_bytes < (128u << 20);
+  // Tiny jobs stay in the register kernel.  From 4 MiB of stageable payload on the staging kernel is
+  // the faster one (measured with L2 flushed, runs of 1 MiB..1 GiB: 10-12 us against 12 us up to 4 MiB,
+  // 14 / 16 us at 16 MiB, 31 / 33 us at 64 MiB, 90 / 94 us at 256 MiB; rectangles with 2 KiB rows: 14 / 21 us
+  // at 16 MiB, 32 / 49 us at 64 MiB), and the warp units of such a job ride along in the same launch.
+  const bool demote = opt.path_mask == 0 && all.tma_bytes < (4u << 20);
   if (demote) {
     for (size_t i = 0; i < n_items; ++i) cnt[i].n[kBig] += cnt[i].n[kTma], cnt[i].n[kTma] = 0, cnt[i].rects = 0;
     all.tma_bytes = all.tma_busy = all.tma_boxed = 0;

@@ -38,7 +38,7 @@ def test_struct_sizes_match_header():
     assert C.sizeof(_lib.TileC) == 64
     assert C.sizeof(_lib.ShardMetaC) == 8 + 16 + 3 * 64 + 16 + 8 + 16
     assert C.sizeof(_lib.PlanOptsC) == 88
-    assert C.sizeof(_lib.PlanStatsC) == 14 * 8
+    assert C.sizeof(_lib.PlanStatsC) == 15 * 8
 
 
 # ---- decomposition (Sec. 3.2) ----------------------------------------------------------------------
