@@ -109,6 +109,19 @@ def check_family(entries: Sequence) -> Tuple[Tuple[int, ...], int]:
     return tuple(int(g) for g in e0.global_shape), int(e0.itemsize)
 
 
+def _held(global_shape: Sequence[int], e) -> np.ndarray:
+    """Which elements of the global tensor the entry holds (boolean array of the global shape)."""
+    m = np.zeros(tuple(global_shape), dtype=bool)
+    b = _box(e)
+    if e.kind == FLAT_SLICE:
+        flat = m[b].ravel()
+        flat[int(e.flat_begin):int(e.flat_end)] = True
+        m[b] = flat.reshape(m[b].shape)
+    else:
+        m[b] = True
+    return m
+
+
 def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payloads: Sequence[np.ndarray],
              first_wins: bool = False):
     """Full global tensor from saved shards, plus how many shards supplied each element.
@@ -116,11 +129,19 @@ def assemble(global_shape: Sequence[int], itemsize: int, entries: Sequence, payl
     Sec. 3.2: shard i covers the box offsets_i + lengths_i of the global shape; an irregular
     shard covers elements [flat_begin, flat_end) of the flattened local box.
     first_wins: replicated shards are allowed and the earliest entry supplies the value
-    (entries are assigned last to first, so the first one overwrites the rest).
+    (entries are assigned last to first, so the first one overwrites the rest).  Replicas are
+    whole shards stored more than once: two entries that share an element must hold exactly the
+    same elements; entries that overlap only partly are an error, with or without first_wins.
     """
     T = np.zeros(tuple(global_shape), dtype=_UINT[itemsize])
     cover = np.zeros(tuple(global_shape), dtype=np.uint8)
     pairs = list(zip(entries, payloads))
+    if first_wins:
+        held = [_held(global_shape, e) for e in entries]
+        for i in range(len(held)):
+            for j in range(i):
+                if (held[i] & held[j]).any() and not np.array_equal(held[i], held[j]):
+                    raise OracleError(f"{entries[i].fqn}: two saved shards overlap only partly")
     for e, data in (reversed(pairs) if first_wins else pairs):
         b = _box(e)
         if e.kind == FLAT_SLICE:

@@ -49,10 +49,11 @@ def _lin(c: Sequence[int], lengths: Sequence[int]) -> int:
     return i
 
 
-def brute_force_reshard(src_metas, src_blobs, dst_metas, dst_buf_bytes, fill_byte=0):
+def brute_force_reshard(src_metas, src_blobs, dst_metas, dst_buf_bytes, fill_byte=0, first_wins=False):
     """Element-by-element definition, written independently of the oracle: for every element
     of every wanted entry find the one saved entry that holds its global coordinate and copy
-    its bytes.  Pure Python loops: tiny inputs only."""
+    its bytes (first_wins: several may hold it, the first in input order supplies the bytes).
+    Pure Python loops: tiny inputs only."""
     out = [np.full(int(n), fill_byte, dtype=np.uint8) for n in dst_buf_bytes]
     for d in dst_metas:
         base = d.flat_begin if d.kind == 1 else 0
@@ -72,7 +73,7 @@ def brute_force_reshard(src_metas, src_blobs, dst_metas, dst_buf_bytes, fill_byt
                         continue
                     pos -= s.flat_begin
                 hits.append((s, pos))
-            assert len(hits) == 1, (d.fqn, g, len(hits))
+            assert len(hits) == 1 or (first_wins and len(hits) > 1), (d.fqn, g, len(hits))
             s, pos = hits[0]
             sb = s.byte_offset + pos * s.itemsize
             db = d.byte_offset + i * d.itemsize

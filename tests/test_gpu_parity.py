@@ -457,10 +457,20 @@ def _pack_full_rank(case, dst, device):
         assert torch.equal(blob[o:o + m.byte_length], dst[r][m.byte_offset:m.byte_offset + m.byte_length])
         end = o + m.byte_length
     assert not bool(blob[end:].any())
-    # oracle on the first 64 tensors
+    # oracle on the first 64 tensors as one blob ...
     k = 64
     want, _ = orc.pack([dst[r][m.byte_offset:m.byte_offset + m.byte_length].cpu().numpy() for m in ms[:k]], 256)
     assert np.array_equal(blob[:offs[k]].cpu().numpy()[:want.size], want)
+    # ... and on a spread sample (first, last, largest, 64 evenly spaced), one tensor at a time: the blob from the
+    # tensor's offset in the oracle's table to the next offset is the oracle's pack of that tensor alone
+    table, table_total = orc.pack_layout(sizes, 256)
+    ends = list(table[1:]) + [table_total]
+    largest = max(range(len(ms)), key=lambda i: sizes[i])
+    for i in sorted({0, len(ms) - 1, largest, *range(0, len(ms), max(1, len(ms) // 64))}):
+        m = ms[i]
+        want, _ = orc.pack([dst[r][m.byte_offset:m.byte_offset + m.byte_length].cpu().numpy()], 256)
+        assert want.size == ends[i] - table[i]
+        assert np.array_equal(blob[table[i]:ends[i]].cpu().numpy(), want), f"packed tensor {i} differs from the oracle"
     out = torch.full((ms[0].byte_length + ms[1].byte_length,), POISON, dtype=torch.uint8, device=device)
     bcp.bcp_unpack(blob, list(zip(offs[:2], sizes[:2])), [out.data_ptr(), out.data_ptr() + sizes[0]], blob_bytes=total)
     torch.cuda.synchronize()

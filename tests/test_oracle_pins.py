@@ -310,3 +310,56 @@ def test_conversion_commutes_with_resharding():
             else:
                 want = torch.from_numpy(raw.view(np.int16).copy()).view(torch.bfloat16).to(torch.float32).numpy().view(np.uint8)
             assert np.array_equal(got[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length], want), (case.name, m.fqn)
+
+
+# ---- replicated saved shards: the first entry in input order wins --------------------------------
+def _with_replicas(case, rng):
+    """Every saved entry of `case`, plus copies of about half of them in a new blob holding OTHER
+    bytes, inserted at random places of the entry list (so that who comes first varies)."""
+    import copy
+
+    metas = list(case.src.metas)
+    extra, pos = [], 0
+    for m in case.src.metas:
+        if m.byte_length and rng.random() < 0.5:
+            k = copy.copy(m)
+            k.buf_index, k.byte_offset = len(case.src.buf_bytes), pos
+            pos += m.byte_length + int(rng.integers(0, 3)) * m.itemsize
+            extra.append(k)
+    for k in extra:
+        metas.insert(int(rng.integers(0, len(metas) + 1)), k)
+    return metas, list(case.src.buf_bytes) + [max(pos, 1)], len(extra)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_first_replica_wins_against_brute_force(seed):
+    """Random tiny problems whose saved side stores some shards twice with different bytes: the
+    oracle's first-wins rule (assign last to first) against the element-by-element mapper that
+    takes the first saved entry, in input order, holding each wanted element."""
+    rng = np.random.default_rng(1000 + seed)
+    case = random_case(seed, n_tensors=3, max_dim=5, dst_replicas=1 + seed % 2)
+    metas, sizes, n_extra = _with_replicas(case, rng)
+    blobs = [rng.integers(0, 256, size=n, dtype=np.uint8) for n in sizes]
+    want = brute_force_reshard(metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, first_wins=True)
+    got = orc.reshard(metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, allow_replicas=True)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    if n_extra:  # without the permission the same input is an error
+        with pytest.raises(orc.OracleError):
+            orc.reshard(metas, blobs, case.dst.metas, case.dst.buf_bytes)
+
+
+def test_partly_overlapping_saved_shards_are_an_error_even_with_replicas_allowed():
+    from workloads.meta import ShardMeta
+
+    whole = ShardMeta("x", 1, 3, (4, 4), (0, 0), (4, 4), 0, 0)
+    a = ShardMeta("x", 1, 3, (4, 4), (0, 0), (3, 4), 0, 0)
+    b = ShardMeta("x", 1, 3, (4, 4), (2, 0), (2, 4), 0, 16)   # shares row 2 with a
+    blob = np.arange(32, dtype=np.uint8)
+    for allow in (False, True):
+        with pytest.raises(orc.OracleError):
+            orc.reshard([a, b], [blob], [whole], [16], allow_replicas=allow)
+    # a flat slice and a box that share some but not all of their elements
+    f = ShardMeta("x", 1, 3, (4, 4), (0, 0), (4, 4), 0, 0, kind=1, flat_begin=2, flat_end=10)
+    with pytest.raises(orc.OracleError):
+        orc.reshard([f, a], [blob], [ShardMeta("x", 1, 3, (4, 4), (0, 2), (1, 2), 0, 0)], [2], allow_replicas=True)

@@ -653,3 +653,55 @@ def test_source_ranges_partition_the_work_list(path_mask):
         with pytest.raises(bcp.BcpError) as e:
             bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, src_buf_first=first, src_buf_count=count)
         assert e.value.code == api.ERR_INVALID
+
+
+# ---- replicated saved shards, random layouts ---------------------------------------------------------
+@pytest.mark.parametrize("seed", range(12))
+def test_random_replicated_sources_first_in_input_order_is_read(seed):
+    """Some saved shards are stored twice with different bytes, at random places of the input:
+    the work list (numpy simulator) must read the first one, as the oracle does."""
+    import copy
+
+    rng = np.random.default_rng(2000 + seed)
+    case = random_case(seed, n_tensors=4, dst_replicas=1 + seed % 2)
+    metas, pos = list(case.src.metas), 0
+    extra = []
+    for m in case.src.metas:
+        if m.byte_length and rng.random() < 0.5:
+            k = copy.copy(m)
+            k.buf_index, k.byte_offset = len(case.src.buf_bytes), pos
+            pos += m.byte_length + int(rng.integers(0, 3)) * m.itemsize
+            extra.append(k)
+    for k in extra:
+        metas.insert(int(rng.integers(0, len(metas) + 1)), k)
+    sizes = list(case.src.buf_bytes) + [max(pos, 1)]
+    blobs = [rng.integers(0, 256, size=n, dtype=np.uint8) for n in sizes]
+    plan = bcp.bcp_plan(metas, sizes, case.dst.metas, case.dst.buf_bytes, allow_replicas=1, tile_bytes=4096)
+    got, _ = run_tiles(plan.tiles(), blobs, case.dst.buf_bytes)
+    want = orc.reshard(metas, blobs, case.dst.metas, case.dst.buf_bytes, fill_byte=0xA5, allow_replicas=True)
+    assert all(np.array_equal(g, w) for g, w in zip(got, want))
+    plan.destroy()
+    if extra:
+        assert _plan_err(metas, sizes, case.dst.metas, case.dst.buf_bytes) == api.ERR_OVERLAP
+
+
+def test_replicas_must_be_whole_shards():
+    """One rank saved a tensor whole, another saved the same tensor as two flat slices: the element
+    sets overlap only partly entry by entry, which is an error with and without allow_replicas
+    (library and oracle alike): replicas are shards stored more than once, box for box."""
+    whole = ShardMeta("x", 4, 2, (6, 4), (0, 0), (6, 4), 0, 0)
+    lo = ShardMeta("x", 4, 2, (6, 4), (0, 0), (6, 4), 1, 0, kind=FLAT_SLICE, flat_begin=0, flat_end=10)
+    hi = ShardMeta("x", 4, 2, (6, 4), (0, 0), (6, 4), 1, 40, kind=FLAT_SLICE, flat_begin=10, flat_end=24)
+    want = [ShardMeta("x", 4, 2, (6, 4), (0, 0), (6, 4), 0, 0)]
+    blobs = [np.arange(96, dtype=np.uint8), np.arange(96, dtype=np.uint8)[::-1].copy()]
+    for allow in (0, 1):
+        assert _plan_err([whole, lo, hi], [96, 96], want, [96], allow_replicas=allow) == api.ERR_OVERLAP
+        with pytest.raises(orc.OracleError):
+            orc.reshard([whole, lo, hi], blobs, want, [96], allow_replicas=bool(allow))
+    # the same flat slices stored twice are replicas
+    lo2, hi2 = ShardMeta(**{**lo.__dict__, "buf_index": 0}), ShardMeta(**{**hi.__dict__, "buf_index": 0})
+    plan = bcp.bcp_plan([lo, hi, lo2, hi2], [96, 96], want, [96], allow_replicas=1)
+    got, _ = run_tiles(plan.tiles(), blobs, [96])
+    assert np.array_equal(got[0], orc.reshard([lo, hi, lo2, hi2], blobs, want, [96], allow_replicas=True)[0])
+    assert np.array_equal(got[0], blobs[1])
+    plan.destroy()
