@@ -71,3 +71,30 @@ def test_emulated_ranks_exchange_and_reshard(cuda_device, case, world):
         assert all(x.send_bytes[x.rank] == 0 for x in xs) and sum(sum(x.send_bytes) for x in xs) > 0
     for x in xs:
         x.destroy()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_zero_copy_variant_reads_peer_blobs_in_place(cuda_device, world):
+    """Without any exchange: every emulated rank plans only its own target buffers against the
+    global saved metadata and hands bcp_reshard the addresses of ALL saved blobs (on several GPUs
+    the other ranks' blobs would be peer-mapped; here they simply live on the same device).  The
+    kernels fetch their tiles straight from wherever a blob lies, so the ranks' plans together
+    write every target buffer and nothing is packed or received."""
+    case = [c for c in scenario_cases() if c.name == "hybrid"][0]
+    nd = len(case.dst.buf_bytes)
+    dst_owner = [(b * world) // nd for b in range(nd)]
+    blobs = fills.fill_state(case.src, case.key_ids, "index", case.seed, cuda_device, poison=0x5A)
+    want = orc.reshard(case.src.metas, [b.cpu().numpy() for b in blobs], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON)
+    written = 0
+    for r in range(world):
+        mine, metas, sizes = multi._local_targets(case.dst.metas, case.dst.buf_bytes, dst_owner, r)
+        plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, metas, sizes, path_mask=7, tma_min_row_bytes=16)
+        dst = [torch.full((n,), POISON, dtype=torch.uint8, device=cuda_device) for n in sizes]
+        bcp.bcp_reshard(plan, blobs, dst)
+        torch.cuda.synchronize()
+        bcp.bcp_plan_device_status(plan)
+        for d, b in zip(dst, mine):
+            assert np.array_equal(d.cpu().numpy(), want[b]), (world, r, b)
+        written += plan.stats()["bytes_copied"]
+        plan.destroy()
+    assert written == case.dst.total_bytes
