@@ -640,13 +640,21 @@ def main():
             t = src[m.buf_index][m.byte_offset:m.byte_offset + m.byte_length]
             return t.cpu().numpy().view(orc._UINT[m.itemsize])
 
-        sec, sb, db, n = time_oracle(case, fetch, a.cpu_sample_gb * 1e9 / 2, steps=a.cpu_passes, warmup=1)
+        # bounded: one pass to see what a pass costs (a converting oracle rounds in float64 and is far slower
+        # than a copying one), then as many passes as fit in about 15 s, at most --cpu-passes
+        sample_bytes = a.cpu_sample_gb * 1e9 / 2
+        probe, sb, db, n = time_oracle(case, fetch, sample_bytes, steps=1, warmup=0)
+        if probe > 15.0:  # shrink the sample as well
+            sample_bytes *= 15.0 / probe
+            probe, sb, db, n = time_oracle(case, fetch, sample_bytes, steps=1, warmup=0)
+        passes = int(max(1, min(a.cpu_passes, 15.0 / max(probe, 1e-3))))
+        sec, sb, db, n = time_oracle(case, fetch, sample_bytes, steps=passes, warmup=0)
         out["cpu_baseline"] = {"value": (sb + db) / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                                "sample": f"{n} FQNs of {case.name}, {sb + db} bytes read+written per pass, "
-                                         f"mean of {a.cpu_passes} passes, {sec:.2f} s each",
+                                         f"mean of {passes} passes after one untimed pass, {sec:.2f} s each",
                                "host_cores_available": os.cpu_count()}
         try:
-            sec2, sb2, db2, n2, cores = time_oracle_all_cores(case, fetch, a.cpu_sample_gb * 1e9 / 2)
+            sec2, sb2, db2, n2, cores = time_oracle_all_cores(case, fetch, sample_bytes, passes=3 if sec < 2 else 1)
             out["cpu_baseline_all_cores"] = {"value": (sb2 + db2) / sec2 / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
                                              "sample": f"same {n2} FQNs, one FQN per task over a fork pool, {sec2:.2f} s per pass"}
         except Exception as e:  # the single-core figure above is the reported baseline
@@ -743,7 +751,7 @@ def time_stage(case, dst, dev, stream):
         st.wait(k)
         st.release(k)
     torch.cuda.synchronize()
-    evs, pending, blocked = [], [], []
+    evs, pending = [], []
     t0 = time.perf_counter()
     for ptrs, metas, total in jobs:
         if len(pending) == 2:
@@ -763,8 +771,14 @@ def time_stage(case, dst, dev, stream):
     blocked = [e0.elapsed_time(e1) for e0, e1 in evs]
     nbytes = sum(t for _, _, t in jobs)
     st.destroy()
+    # The producer's stream is held for the pack alone when a slot is free (the first two saves here: the
+    # blocking part of a save, what the paper calls T_Block).  Saves issued back to back, faster than PCIe
+    # drains the pool, also wait for a slot's download: that is the pool's throughput, not the stall.
+    free = blocked[:2]
     return {"ranks": len(jobs), "blob_bytes_total": nbytes, "wall_s": wall, "host_gbps": nbytes / wall / 1e9,
-            "blocking_ms_per_save": sum(blocked) / len(blocked), "slots": 2}
+            "blocking_ms_per_save": sum(free) / len(free), "blocking_ms_back_to_back": sum(blocked) / len(blocked), "slots": 2,
+            "blocking_note": "blocking_ms_per_save: device time of a save that finds a free slot (the pack); "
+                             "back_to_back: mean over all saves issued without pause, waits for a slot included"}
 
 
 def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
