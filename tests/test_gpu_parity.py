@@ -554,9 +554,9 @@ def test_plans_run_from_several_threads_on_their_own_streams(cuda_device):
 
 
 # ---- element conversion (extension) --------------------------------------------------------------
-# kernel: the default keeps jobs this small on the register kernel; path_mask 3 sends every source row of
+# kernel: path_mask 1 keeps every converting unit on the register kernel; path_mask 3 sends every source row of
 # at least tma_min_row_bytes through the staged kernel (16: nearly all of them, 512: a mix of both kernels)
-CVT_PATHS = {"register": {}, "staged": {"path_mask": 3, "tma_min_row_bytes": 16}, "mixed": {"path_mask": 3, "tma_min_row_bytes": 512}}
+CVT_PATHS = {"register": {"path_mask": 1}, "staged": {"path_mask": 3, "tma_min_row_bytes": 16}, "mixed": {"path_mask": 3, "tma_min_row_bytes": 512}}
 
 
 @pytest.mark.parametrize("path", list(CVT_PATHS))
