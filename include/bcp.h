@@ -330,6 +330,17 @@ BCP_API int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_p
 BCP_API int bcp_plan_tiles(const bcp_plan_t* plan, bcp_tile* out, size_t cap, size_t* n);
 
 /*
+ * Which saved entries the plan reads: ascending indices into the `src` array that was given to
+ * bcp_plan, one per saved entry that holds at least one element some wanted entry of the plan
+ * asks for (the "matching segments" of Sec. 3.3 Step 2, reported per saved shard).  This is what a
+ * rank has to obtain before it can run the plan: the cross-GPU exchange (Sec. 4.1, "Eliminating
+ * redundant loading"; Sec. 4.2, load pipeline) sends exactly these entries.  Writes min(cap, count)
+ * indices to out (may be NULL when cap == 0) and the full count to *n.  Only plans built by
+ * bcp_plan record this (BCP_ERR_INVALID for deserialized images).
+ */
+BCP_API int bcp_plan_used_sources(const bcp_plan_t* plan, uint32_t* out, size_t cap, size_t* n);
+
+/*
  * Execute a plan (Sec. 3.3, Step 5: copy every matched segment into its target shard).
  * src_blobs[n_src_bufs] and dst_bufs[n_dst_bufs] are HOST arrays of DEVICE pointers to
  * buffers at least as large as planned, each 16-byte aligned (BCP_ERR_INVALID otherwise),

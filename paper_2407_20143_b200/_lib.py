@@ -101,6 +101,7 @@ _PROTOS = {
     "bcp_plan_serialize": (C.c_int, [_VP, _VP, C.c_size_t, C.POINTER(C.c_size_t)]),
     "bcp_plan_deserialize": (C.c_int, [_VP, C.c_size_t, C.POINTER(_VP)]),
     "bcp_plan_tiles": (C.c_int, [_VP, C.POINTER(TileC), C.c_size_t, C.POINTER(C.c_size_t)]),
+    "bcp_plan_used_sources": (C.c_int, [_VP, C.POINTER(C.c_uint32), C.c_size_t, C.POINTER(C.c_size_t)]),
     "bcp_reshard": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),
     "bcp_reshard_host": (C.c_int, [_VP, C.POINTER(_VP), C.c_size_t, C.POINTER(_VP), C.c_size_t, _VP]),
     "bcp_plan_device_status": (C.c_int, [_VP, _VP]),

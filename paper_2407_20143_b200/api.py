@@ -115,6 +115,14 @@ class Plan:
         _check(L.lib().bcp_plan_stats(self.handle, C.byref(st)))
         return {n: getattr(st, n) for n, _ in L.PlanStatsC._fields_}
 
+    def used_sources(self) -> List[int]:
+        """Indices (into the saved metas given to bcp_plan) of the entries the plan reads, ascending."""
+        n = C.c_size_t()
+        _check(L.lib().bcp_plan_used_sources(self.handle, None, 0, C.byref(n)))
+        arr = (C.c_uint32 * max(1, n.value))()
+        _check(L.lib().bcp_plan_used_sources(self.handle, arr, n.value, C.byref(n)))
+        return list(arr[: n.value])
+
     def tiles(self) -> List[L.TileC]:
         n = C.c_size_t()
         _check(L.lib().bcp_plan_tiles(self.handle, None, 0, C.byref(n)))

@@ -462,12 +462,15 @@ int bcp_plan(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_by
     std::vector<Gap> gaps;
     bcp_plan_stats_t st;
     memset(&st, 0, sizeof st);
-    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt, &items, &gaps, &st))
+    std::vector<uint32_t> used;
+    if (int rc = match_and_lower(src, n_src, src_buf_bytes, n_src_bufs, dst, n_dst, dst_buf_bytes, n_dst_bufs, opt, &items, &gaps, &st, &used))
       return rc;
     bcp_plan_t* p = finish_plan(items, opt, st, std::vector<uint64_t>(src_buf_bytes, src_buf_bytes + n_src_bufs),
                               std::vector<uint64_t>(dst_buf_bytes, dst_buf_bytes + n_dst_bufs));
     if (!p) return fail(BCP_ERR_NOMEM, "out of host memory");
     p->gaps = std::move(gaps);
+    p->used_src = std::move(used);
+    p->has_used_src = true;
     if (p->tiles.size() > 0xFFFF0000ull) {
       delete p;
       return fail(BCP_ERR_INVALID, "work list too long for one launch");
@@ -488,6 +491,15 @@ int bcp_plan_stats(const bcp_plan_t* plan, bcp_plan_stats_t* out) {
   const size_t rest = plan->n_big + plan->n_small();
   out->n_kernels = (plan->n_tma > 0) + (rest > 0 && !folds(plan->n_tma, plan->n_big, plan->n_small())) + (staged > 0) +
                    (staged < plan->n_cvt);
+  return BCP_OK;
+}
+
+int bcp_plan_used_sources(const bcp_plan_t* plan, uint32_t* out, size_t cap, size_t* n) {
+  if (!plan || !n || (cap && !out)) return fail(BCP_ERR_INVALID, "bcp_plan_used_sources: NULL argument");
+  if (!plan->has_used_src) return fail(BCP_ERR_INVALID, "bcp_plan_used_sources: this plan was not built by bcp_plan (images and pack layouts do not record it)");
+  *n = plan->used_src.size();
+  const size_t k = cap < plan->used_src.size() ? cap : plan->used_src.size();
+  if (k) memcpy(out, plan->used_src.data(), k * sizeof(uint32_t));
   return BCP_OK;
 }
 

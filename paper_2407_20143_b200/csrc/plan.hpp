@@ -75,10 +75,11 @@ struct RelBox {
 void decompose(const int64_t* lengths, uint32_t ndim, int64_t a, int64_t b, std::vector<RelBox>* out);
 
 // Matching (Sec. 3.3 Step 2) + lowering: metas -> items.  Fills the entry / intersection
-// counters of `stats`.
+// counters of `stats` and, if asked, the ascending indices of the saved entries the items read.
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats);
+                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats,
+                    std::vector<uint32_t>* used_src);
 
 // Coalesce adjacent items, cut them into work units, classify and order them.
 // tiles = [TMA units..., other CTA-wide units..., warp units..., converting units...].

@@ -19,6 +19,8 @@ struct bcp_plan_s {
   std::vector<uint64_t> src_bytes, dst_bytes;
   std::vector<bcp::Rect> rects;  // rectangles staged through tensor maps (two descriptors each)
   std::vector<bcp::Gap> gaps;    // target bytes no entry names (zeroed by the host-buffer call)
+  std::vector<uint32_t> used_src;  // bcp_plan only: indices of the saved entries the work list reads
+  bool has_used_src = false;
   std::vector<CUtensorMap> h_maps;
   CUtensorMap* d_maps = nullptr;
   // device side, created by the first execution

@@ -378,7 +378,8 @@ struct SegKey {
 
 int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src_buf_bytes, size_t n_src_bufs,
                     const bcp_shard_meta* dst, size_t n_dst, const uint64_t* dst_buf_bytes, size_t n_dst_bufs,
-                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats) {
+                    const Options& opt, std::vector<Item>* items, std::vector<Gap>* gaps, bcp_plan_stats_t* stats,
+                    std::vector<uint32_t>* used_src) {
   const bool allow_replicas = opt.allow_replicas != 0;
   if ((n_src && !src) || (n_dst && !dst) || (n_src_bufs && !src_buf_bytes) || (n_dst_bufs && !dst_buf_bytes))
     return fail(BCP_ERR_INVALID, "bcp_plan: NULL array with non-zero count");
@@ -475,6 +476,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
   const uint32_t keep_first = opt.src_buf_first, keep_count = opt.src_buf_count;
   if (keep_count && (keep_first > n_src_bufs || keep_count > n_src_bufs - keep_first))
     return fail(BCP_ERR_INVALID, "source buffers [%u, %u + %u) are not among the %zu given", keep_first, keep_first, keep_count, n_src_bufs);
+  std::vector<uint8_t> src_used(n_src ? n_src : 1, 0);  // saved entries that a kept piece reads
   struct Scratch {
     std::vector<SegKey> segs;    // matched segments of the family at hand
     std::vector<int64_t> reach;  // reach[i] = largest end (along dim 0) among the family's saved boxes 0..i
@@ -547,6 +549,7 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
         // a plan restricted to some source buffers matches and checks coverage against all of
         // them, and keeps the pieces that are read from the chosen ones
         if (keep_count && (s.buf < keep_first || s.buf - keep_first >= keep_count)) continue;
+        src_used[s.meta] = 1;  // (a saved entry belongs to one tensor, so no two threads write the same flag)
         ++n_inter;
         lower(s, d, nd, f.itemsize, f.d_itemsize, f.cvt, o, l, items);
         SegKey key = {si, 0, 0, uint64_t(volume(l, 0, nd)) * f.itemsize};
@@ -626,6 +629,11 @@ int match_and_lower(const bcp_shard_meta* src, size_t n_src, const uint64_t* src
       n_se += b.n_se;
       n_de += b.n_de;
     }
+  }
+  if (used_src) {
+    used_src->clear();
+    for (size_t i = 0; i < n_src; ++i)
+      if (src_used[i]) used_src->push_back(uint32_t(i));
   }
   stats->n_src_entries = n_se;
   stats->n_dst_entries = n_de;

@@ -113,38 +113,14 @@ def _local_targets(dst_metas: Sequence, dst_buf_bytes: Sequence[int], dst_owner:
 
 def needed_entries(src_metas: Sequence, src_buf_bytes: Sequence[int], dst_metas: Sequence, dst_buf_bytes: Sequence[int],
                    dst_owner: Sequence[int], rank: int, **opts) -> List[int]:
-    """Indices of the saved entries whose bytes this rank's targets read.  The planner does the
-    matching; this only maps the source ranges of its work units back to entries."""
+    """Indices of the saved entries whose bytes this rank's targets read: the planner does the
+    matching and reports them (bcp_plan_used_sources)."""
     _, mine, mine_bytes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
     probe = api.bcp_plan(src_metas, src_buf_bytes, mine, mine_bytes, **opts)
     try:
-        import numpy as np
-
-        tiles = probe.tiles_array()
-        tiles = tiles[(tiles["flags"] & api.TILE_ZERO) == 0]
-        kind = (tiles["flags"] & api.TILE_CVT_MASK) >> api.TILE_CVT_SHIFT
-        row = tiles["row_bytes"].astype(np.uint64)
-        row = np.where(kind == api.CONVERT_F32_TO_BF16, row * 2, np.where(kind == api.CONVERT_BF16_TO_F32, row // 2, row))
-        lo = tiles["src_off"]
-        hi = lo + (tiles["rows"].astype(np.uint64) - 1) * tiles["src_pitch"] + row  # a rectangle lies inside one entry
-        named = np.array([i for i, m in enumerate(src_metas) if m.byte_length], dtype=np.int64)
-        bufs = np.array([src_metas[i].buf_index for i in named], dtype=np.int64)
-        offs = np.array([src_metas[i].byte_offset for i in named], dtype=np.uint64)
-        used: List[int] = []
-        for b in np.unique(tiles["src_buf"]):
-            sel = named[bufs == b]
-            sel = sel[np.argsort(offs[bufs == b], kind="stable")]
-            starts = np.array([src_metas[i].byte_offset for i in sel], dtype=np.uint64)
-            of_buf = tiles["src_buf"] == b
-            first = np.searchsorted(starts, lo[of_buf], side="right") - 1   # entry that holds the unit's first byte
-            last = np.searchsorted(starts, hi[of_buf], side="left")          # a coalesced run may span adjacent entries
-            mark = np.zeros(len(sel) + 1, dtype=np.int64)
-            np.add.at(mark, first, 1)
-            np.add.at(mark, last, -1)
-            used.extend(int(i) for i in sel[np.cumsum(mark[:-1]) > 0])
+        return probe.used_sources()
     finally:
         probe.destroy()
-    return sorted(used)
 
 
 def build_exchange(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: Sequence[int], dst_metas: Sequence,

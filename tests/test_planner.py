@@ -705,3 +705,42 @@ def test_replicas_must_be_whole_shards():
     assert np.array_equal(got[0], orc.reshard([lo, hi, lo2, hi2], blobs, want, [96], allow_replicas=True)[0])
     assert np.array_equal(got[0], blobs[1])
     plan.destroy()
+
+
+# ---- which saved entries a plan reads ------------------------------------------------------------------
+def _element_mask(m):
+    mask = np.zeros(tuple(m.global_shape), dtype=bool)
+    box = tuple(slice(o, o + l) for o, l in zip(m.offsets, m.lengths))
+    if m.kind == FLAT_SLICE:
+        flat = mask[box].ravel()
+        flat[m.flat_begin:m.flat_end] = True
+        mask[box] = flat.reshape(mask[box].shape)
+    else:
+        mask[box] = True
+    return mask
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_used_sources_are_the_saved_entries_that_share_an_element_with_a_wanted_one(seed):
+    case = random_case(300 + seed, n_tensors=5, dst_replicas=1 + seed % 2)
+    wanted = {}
+    for d in case.dst.metas:
+        wanted[d.fqn] = wanted.get(d.fqn, False) | _element_mask(d)
+    expect = [i for i, s in enumerate(case.src.metas) if s.fqn in wanted and bool((_element_mask(s) & wanted[s.fqn]).any())]
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes)
+    assert plan.used_sources() == expect
+    plan.destroy()
+    # a plan for part of the targets reads fewer entries; a plan restricted to some source buffers only entries in them
+    half = [d for d in case.dst.metas if d.buf_index == 0]
+    if half:
+        sub = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, half, case.dst.buf_bytes)
+        assert set(sub.used_sources()) <= set(expect)
+        sub.destroy()
+    only0 = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, src_buf_first=0, src_buf_count=1)
+    assert only0.used_sources() == [i for i in expect if case.src.metas[i].buf_index == 0]
+    image = only0.serialize()
+    only0.destroy()
+    again = bcp.Plan.deserialize(image)
+    with pytest.raises(bcp.BcpError):
+        again.used_sources()
+    again.destroy()
