@@ -68,6 +68,9 @@ def parse_args():
     ap.add_argument("--exchange", action="store_true",
                     help="time the cross-rank path instead: blobs and target buffers dealt to the N ranks, a step = pack -> "
                          "all-to-all -> reshard (per-stage times, bytes crossed); without the flag --gpus N runs replicas")
+    ap.add_argument("--zero-copy", action="store_true",
+                    help="with --exchange: no pack and no collective; every rank maps its peers' blobs (bcp_ipc_*) and its "
+                         "copy kernels read them in place")
     ap.add_argument("--exchange-emulate", type=int, default=2,
                     help="after the headline run, emulate this many ranks of the cross-rank path on the one GPU and report "
                          "per-stage device times (extra key `exchange_emulated`); 0 or 1 skips it")
@@ -458,6 +461,7 @@ def run_exchange_bench(a):
     """bench.py --exchange: saved blobs and target buffers of the workload are dealt to the ranks in
     contiguous blocks; a step is pack -> all-to-all -> reshard with the plans reused.  With one rank
     nothing crosses and the step is the rank's plain reshard."""
+    import numpy as np
     import torch
 
     import paper_2407_20143_b200 as bcp
@@ -473,23 +477,36 @@ def run_exchange_bench(a):
     case = make_case(a)
     opts = dict(plan_opts(a), **case.plan_opts)
     src_owner, dst_owner = block_owner(len(case.src.buf_bytes), ws), block_owner(len(case.dst.buf_bytes), ws)
-    t0 = time.perf_counter()
-    x = multi.plan_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, **opts)
-    plan_ms = (time.perf_counter() - t0) * 1e3
+    local_src = [b for b, o in enumerate(src_owner) if o == rank]
     by_buf = {}
     for m in case.src.metas:
         by_buf.setdefault(m.buf_index, []).append(m)
     blobs = []
-    for b in x.local_src:
+    for b in local_src:
         t = torch.zeros(case.src.buf_bytes[b], dtype=torch.uint8, device=dev)
         for m in by_buf.get(b, []):
             fills.write_entry(t, m, case.key_ids[m.fqn], case.fill, case.seed)
         blobs.append(t)
-    dst = [torch.zeros(n, dtype=torch.uint8, device=dev) for n in x.dst_buf_bytes]
+    torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
-    x.bind(dev)
-    plans = [p for p in (x.plan_local, x.plan_remote) if p is not None]
+    t0 = time.perf_counter()
+    if a.zero_copy:
+        x = multi.plan_zero_copy(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, blobs, **opts)
+        plans = [x.plan]
+
+        def step():
+            x.run(dst, stream)
+    else:
+        x = multi.plan_exchange(case.src.metas, case.src.buf_bytes, src_owner, case.dst.metas, case.dst.buf_bytes, dst_owner, **opts)
+        x.bind(dev)
+        plans = [p for p in (x.plan_local, x.plan_remote) if p is not None]
+
+        def step():
+            multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+    plan_ms = (time.perf_counter() - t0) * 1e3
+    dst = [torch.zeros(n, dtype=torch.uint8, device=dev) for n in x.dst_buf_bytes]
     b_local = sum(p.stats()["bytes_src_unique"] + p.stats()["bytes_copied"] for p in plans)
+    D.barrier()  # every owner's blobs are complete before anybody reads them
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -497,7 +514,7 @@ def run_exchange_bench(a):
     with ClockSampler(local_rank) as clocks:
         clocks.wait_first_sample()
         for _ in range(max(a.warmup, 3)):
-            multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+            step()
         torch.cuda.synchronize()
         D.barrier()
         torch.cuda.synchronize()
@@ -505,41 +522,48 @@ def run_exchange_bench(a):
         clocks.mark_begin()
         head0.record(stream)
         for _ in range(a.steps - 1):
-            multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+            step()
         head1.record(stream)
         if not a.no_verify:
             for d in dst:
                 d.fill_(POISON)
         last0.record(stream)
-        multi.run_exchange(x, case.src.metas, blobs, dst, stream)
+        step()
         last1.record(stream)
         torch.cuda.synchronize()
         clocks.mark_end()
     D.barrier()
     ms_step = D.max_over_ranks((head0.elapsed_time(head1) + last0.elapsed_time(last1)) / a.steps, dev)
-    stages = {k: D.max_over_ranks(v, dev) for k, v in x.stage_ms().items()}  # of the last timed step
+    stages = None if a.zero_copy else {k: D.max_over_ranks(v, dev) for k, v in x.stage_ms().items()}  # of the last timed step
     for p in plans:
         bcp.bcp_plan_device_status(p)
     ok, checked = (None, 0) if a.no_verify else verify_targets(case, dst, x.local_dst)
     ok_all = None if ok is None else D.max_over_ranks(0.0 if ok else 1.0, dev) == 0.0
     total_bytes = D.sum_over_ranks(b_local, dev)
-    sent = D.max_over_ranks(float(sum(x.send_bytes)), dev)
-    recv = D.max_over_ranks(float(sum(x.recv_bytes)), dev)
+    if a.zero_copy:  # bytes its kernels read from peers' blobs, from the work list
+        u = x.plan.tiles_array()
+        far = np.array([src_owner[b] != rank for b in range(len(src_owner))])[u["src_buf"]] & ((u["flags"] & 0x88) == 0)  # not zero fills, not followers
+        sent, recv = 0.0, D.max_over_ranks(float((u["rows"].astype("int64") * u["row_bytes"])[far].sum()), dev)
+    else:
+        sent = D.max_over_ranks(float(sum(x.send_bytes)), dev)
+        recv = D.max_over_ranks(float(sum(x.recv_bytes)), dev)
     value = total_bytes / (ms_step * 1e-3) / 1e9
-    n_kernels = sum(p.stats()["n_kernels"] for p in plans) + (2 if sum(x.send_bytes) else 0)
+    n_kernels = sum(p.stats()["n_kernels"] for p in plans) + (0 if a.zero_copy else (2 if sum(x.send_bytes) else 0))
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": a.steps, "warmup": max(a.warmup, 3),
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "u8",
            "data": "synthetic",
-           "config": {"workload": case.name, "mode": "exchange", "bytes_per_step": total_bytes,
+           "config": {"workload": case.name, "mode": "zero-copy (peers' blobs read in place)" if a.zero_copy else "exchange", "bytes_per_step": total_bytes,
                       "bytes_counted": "per rank: distinct source bytes its plans read (own blobs and received segments) + "
                                        "target bytes written; summed over ranks",
                       "partition": "saved blobs and target buffers in contiguous blocks over the ranks",
                       "l2": "inputs_exceed_l2", "fill": case.fill, "plan_ms": plan_ms, "plan_opts": plan_opts(a)},
            "exchange": {"world": ws, "stage_ms_max_over_ranks": stages, "sent_bytes_max_rank": sent, "received_bytes_max_rank": recv,
-                        "collective": "torch.distributed.all_to_all_single (NCCL)" if ws > 1 else "none (one rank: nothing crosses)"},
+                        "collective": "none: peer loads inside the copy kernel" if a.zero_copy else
+                                      "torch.distributed.all_to_all_single (NCCL)" if ws > 1 else "none (one rank: nothing crosses)"},
            "gpu_launches": a.steps * n_kernels, "verified": ok_all, "verified_bytes": checked, "clocks": clocks.summary(),
            "e2e": None, "roofline": None, "cpu_baseline": None}
-    x.destroy()
+    D.barrier()  # nobody reads a peer's blob any more
+    x.close() if a.zero_copy else x.destroy()
     if rank == 0:
         print(json.dumps(out))
     D.shutdown()

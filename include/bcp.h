@@ -482,6 +482,41 @@ BCP_API int bcp_stager_load(bcp_stager_t* stager, uint32_t slot, uint64_t blob_b
 BCP_API int bcp_stager_release(bcp_stager_t* stager, uint32_t slot);
 
 /*
+ * Peer mapping of saved blobs, for cross-GPU resharding without an exchange step.  The paper's
+ * load pipeline moves the pieces a rank needs from its DP peers in an all-to-all (Sec. 4.1,
+ * "Eliminating redundant loading"; Sec. 4.2); with every GPU able to address its peers' memory the
+ * same pieces can be read where they lie: a rank plans its own targets against the global saved
+ * metadata (a plan may cover any subset of the wanted entries) and hands bcp_reshard the addresses
+ * of ALL saved blobs, its own and its peers' mapped ones.  The copy kernels then fetch every tile
+ * straight from its owner (plain bulk loads, one destination CTA each; over NVLink when the owner is
+ * another GPU) and the transfer overlaps the copy tile by tile; nothing is packed, sent or received.
+ *
+ *   bcp_ipc_export  fills *out for the device pointer dev_ptr (device current = the one that owns
+ *                   it): the CUDA IPC handle of the allocation that contains it, the pointer's offset
+ *                   inside that allocation and the bytes from there to the allocation's end.  The
+ *                   96 bytes are plain data: send them to the other processes by any means.
+ *   bcp_ipc_open    maps the allocation in the calling process (device current = the one that will
+ *                   read it; peer access is enabled on demand) and returns the address that
+ *                   corresponds to the exported pointer.  An allocation is mapped once per process and
+ *                   device however many pointers into it are opened.  A process cannot open its own
+ *                   handles: it uses its own pointers.
+ *   bcp_ipc_close   gives a pointer from bcp_ipc_open back; the allocation is unmapped with the last one.
+ * The owner keeps the memory allocated, and its contents in place, from the export until every
+ * reader has closed; ordering between the owner's writes and the readers' kernels is the caller's
+ * (a barrier between the processes).  Memory of a virtual-memory pool cannot be exported: BCP_ERR_CUDA.
+ */
+typedef struct {
+  unsigned char handle[64];
+  uint64_t offset;
+  uint64_t bytes_after;
+  int32_t device;     /* device index in the exporting process (informational) */
+  int32_t reserved[3];
+} bcp_ipc_handle;
+BCP_API int bcp_ipc_export(const void* dev_ptr, bcp_ipc_handle* out);
+BCP_API int bcp_ipc_open(const bcp_ipc_handle* handle, void** out_ptr);
+BCP_API int bcp_ipc_close(void* ptr);
+
+/*
  * bcp_pack for callers that cannot allocate.  (The paper has no counterpart: this entry point
  * exists for the way the library gets embedded, not for the method.)
  *

@@ -77,6 +77,11 @@ class PlanStatsC(C.Structure):
         ("plan_ms", C.c_double), ("n_cvt_tiles", C.c_uint64), ("n_kernels", C.c_uint64)]
 
 
+class IpcHandleC(C.Structure):
+    _fields_ = [("handle", C.c_ubyte * 64), ("offset", C.c_uint64), ("bytes_after", C.c_uint64), ("device", C.c_int32),
+                ("reserved", C.c_int32 * 3)]
+
+
 class ExportEntryC(C.Structure):
     _fields_ = [("name", C.c_char_p), ("dtype", C.c_char_p), ("ndim", C.c_uint32), ("reserved", C.c_uint32),
                 ("shape", C.c_int64 * BCP_MAX_NDIM)]
@@ -123,6 +128,9 @@ _PROTOS = {
     "bcp_stager_acquire": (C.c_int, [_VP, C.POINTER(C.c_uint32), C.POINTER(_VP)]),
     "bcp_stager_load": (C.c_int, [_VP, C.c_uint32, C.c_uint64, C.POINTER(PackMetaC), C.c_size_t, C.POINTER(_VP), _VP]),
     "bcp_stager_release": (C.c_int, [_VP, C.c_uint32]),
+    "bcp_ipc_export": (C.c_int, [_VP, C.POINTER(IpcHandleC)]),
+    "bcp_ipc_open": (C.c_int, [C.POINTER(IpcHandleC), C.POINTER(_VP)]),
+    "bcp_ipc_close": (C.c_int, [_VP]),
     "bcp_pack_static": (C.c_int, [C.POINTER(_VP), C.POINTER(PackMetaC), C.c_size_t, _VP, C.c_uint64, _VP]),
 }
 

@@ -262,6 +262,25 @@ def bcp_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]], blob, blob_byt
     _check(L.lib().bcp_pack(_ptrs(tensors), _pack_metas(metas), len(tensors), bp, nb, _stream(stream)))
 
 
+def bcp_ipc_export(tensor) -> bytes:
+    """Handle (96 plain bytes) under which another process can map the device memory `tensor` starts at."""
+    h = L.IpcHandleC()
+    _check(L.lib().bcp_ipc_export(tensor if isinstance(tensor, int) else tensor.data_ptr(), C.byref(h)))
+    return bytes(h)
+
+
+def bcp_ipc_open(handle: bytes) -> int:
+    """Address, in this process and on the current device, of memory another process exported."""
+    h = L.IpcHandleC.from_buffer_copy(handle)
+    p = C.c_void_p()
+    _check(L.lib().bcp_ipc_open(C.byref(h), C.byref(p)))
+    return p.value
+
+
+def bcp_ipc_close(ptr: int) -> None:
+    _check(L.lib().bcp_ipc_close(ptr))
+
+
 def marshal_pack(tensors: Sequence, metas: Sequence[Tuple[int, int]]):
     """The C arrays of a pack call, for callers that repeat one pack many times (see bcp_pack_marshalled)."""
     return _ptrs(tensors), _pack_metas(metas), len(tensors)

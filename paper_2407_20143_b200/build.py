@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libbcp.so")
-SOURCES = ["planner.cpp", "units.cpp", "api.cu", "plan_image.cu", "host_path.cu", "kernels.cu", "tma_kernel.cu", "convert_kernel.cu", "static_pack.cu", "stager.cu", "export.cu"]
+SOURCES = ["planner.cpp", "units.cpp", "api.cu", "plan_image.cu", "host_path.cu", "kernels.cu", "tma_kernel.cu", "convert_kernel.cu", "static_pack.cu", "stager.cu", "export.cu", "ipc.cu"]
 HEADERS = ["plan.hpp", "kernels.cuh", "host_threads.hpp", "plan_object.hpp", "tma_ptx.cuh", "copy_loops.cuh"]
 
 

@@ -252,3 +252,76 @@ def run_exchange(x: Exchange, src_metas: Sequence, local_blobs: Sequence, dst_bu
         e["remote_done"].record(main)
         main.wait_event(e["local_done"])
         e["end"].record(main)
+
+
+# ----------------------------------------------------------------------------- without an exchange
+@dataclass
+class ZeroCopy:
+    """Cross-GPU resharding with no exchange step: this rank's plan for its own target buffers against
+    the global saved metadata, and the addresses of ALL saved blobs (own pointers, peers' blobs mapped
+    through bcp_ipc_open).  bcp_reshard then reads every tile where it lies."""
+
+    rank: int
+    world: int
+    local_dst: List[int]
+    dst_buf_bytes: List[int]
+    plan: Optional[api.Plan]
+    src_ptrs: List[int]                  # one address per saved blob, in global order
+    opened: List[int] = field(default_factory=list)
+    keep: List[object] = field(default_factory=list)   # own blobs, kept alive while peers may read them
+
+    def run(self, dst_bufs: Sequence, stream=None) -> None:
+        """Asynchronous on `stream`.  The caller orders it against the owners' writes of their blobs
+        (a barrier between the processes before the first run and before anybody frees a blob)."""
+        api.bcp_reshard(self.plan, self.src_ptrs, dst_bufs, stream=stream)
+
+    def close(self) -> None:
+        for p in self.opened:
+            api.bcp_ipc_close(p)
+        self.opened = []
+        if self.plan is not None:
+            self.plan.destroy()
+            self.plan = None
+        self.keep = []
+
+
+def plan_zero_copy(src_metas: Sequence, src_buf_bytes: Sequence[int], src_owner: Sequence[int], dst_metas: Sequence,
+                   dst_buf_bytes: Sequence[int], dst_owner: Sequence[int], local_blobs: Sequence, **opts) -> ZeroCopy:
+    """Collective: every rank of the default process group calls this with the same metadata and its
+    own blobs (device tensors, in the order of its entries in src_owner).  Handles of all blobs are
+    gathered, every rank maps the blobs of the others, and plans its own targets against everything.
+    Only the blobs a rank's plan reads are mapped."""
+    import torch.distributed as dist
+
+    rank, world = (dist.get_rank(), dist.get_world_size()) if dist.is_initialized() else (0, 1)
+    mine = [b for b, o in enumerate(src_owner) if o == rank]
+    assert len(mine) == len(local_blobs), "one device tensor per saved blob this rank owns"
+    handles = {b: api.bcp_ipc_export(t) for b, t in zip(mine, local_blobs)} if world > 1 else {}
+    everybody: List = [None] * world
+    if world > 1:
+        dist.all_gather_object(everybody, handles)
+    local_dst, metas, sizes = _local_targets(dst_metas, dst_buf_bytes, dst_owner, rank)
+    plan = api.bcp_plan(src_metas, src_buf_bytes, metas, sizes, **opts)
+    wanted = {src_metas[i].buf_index for i in plan.used_sources()}
+    own = dict(zip(mine, local_blobs))
+    ptrs, opened = [], []
+    try:
+        for b in range(len(src_buf_bytes)):
+            if b in own:
+                ptrs.append(own[b].data_ptr())
+            elif b in wanted:
+                p = api.bcp_ipc_open(everybody[src_owner[b]][b])
+                opened.append(p)
+                ptrs.append(p)
+            elif mine:
+                ptrs.append(own[mine[0]].data_ptr())  # never read by this plan: any valid address will do
+            else:  # a rank without blobs of its own has no address to spare: map the blob after all
+                p = api.bcp_ipc_open(everybody[src_owner[b]][b])
+                opened.append(p)
+                ptrs.append(p)
+    except Exception:
+        for p in opened:
+            api.bcp_ipc_close(p)
+        plan.destroy()
+        raise
+    return ZeroCopy(rank, world, local_dst, sizes, plan, ptrs, opened, list(local_blobs))

@@ -98,3 +98,30 @@ def test_zero_copy_variant_reads_peer_blobs_in_place(cuda_device, world):
         written += plan.stats()["bytes_copied"]
         plan.destroy()
     assert written == case.dst.total_bytes
+
+
+def test_two_processes_zero_copy_and_exchange(cuda_device):
+    """Two rank processes on the one GPU (independent launches, host-side barriers): peers' blobs
+    mapped through bcp_ipc_* and read in place, then the pack -> all-to-all -> two-plan exchange with
+    a real collective carrying the segments; every rank's targets against the oracle."""
+    import os
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    worker = os.path.join(root, "tests", "two_process_worker.py")
+    port = 29700 + os.getpid() % 200
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK="0", WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, worker], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        try:
+            outs.append(p.communicate(timeout=240))
+        except subprocess.TimeoutExpired:
+            for q in procs:
+                q.kill()
+            raise
+    assert all(p.returncode == 0 for p in procs), [o[1][-1500:] for o in outs]
+    assert all("two-process ok" in o[0] for o in outs)
