@@ -795,6 +795,7 @@ def time_stage(case, dst, dev, stream):
     torch.cuda.synchronize()
     blocked = [e0.elapsed_time(e1) for e0, e1 in evs]
     nbytes = sum(t for _, _, t in jobs)
+    load = stage_load_leg(st, jobs, dev, stream)
     st.destroy()
     # The producer's stream is held for the pack alone when a slot is free (the first two saves here: the
     # blocking part of a save, what the paper calls T_Block).  Saves issued back to back, faster than PCIe
@@ -802,8 +803,71 @@ def time_stage(case, dst, dev, stream):
     free = blocked[:2]
     return {"ranks": len(jobs), "blob_bytes_total": nbytes, "wall_s": wall, "host_gbps": nbytes / wall / 1e9,
             "blocking_ms_per_save": sum(free) / len(free), "blocking_ms_back_to_back": sum(blocked) / len(blocked), "slots": 2,
+            "load": load,
             "blocking_note": "blocking_ms_per_save: device time of a save that finds a free slot (the pack); "
                              "back_to_back: mean over all saves issued without pause, waits for a slot included"}
+
+
+def stage_load_leg(st, jobs, dev, stream):
+    """The way back: blobs that sit in the pinned slots are uploaded on the side stream and unpacked into
+    tensors on `stream` (bcp_stager_load), as many at once as there are slots and device memory for the
+    unpacked copies; wall clock from the first load to the last release, and a byte-for-byte check."""
+    import torch
+
+    free, _ = torch.cuda.mem_get_info()
+    n = 0
+    for _, _, total in jobs[:2]:
+        if free > total + (4 << 30):
+            free -= total
+            n += 1
+    if n == 0:
+        return {"skipped": "no device memory for an unpacked copy"}
+    # put the blobs into the pinned slots (not timed), give the slots back and take them again the way a
+    # loader does: the pinned buffers keep their bytes, which stand for blobs just read from storage
+    saved = {}
+    for j, (ptrs, metas, total) in enumerate(jobs[:n]):
+        saved[st.save(ptrs, metas, total, stream=stream)] = j
+    for k in saved:
+        st.wait(k)
+    for k in saved:
+        st.release(k)
+    held = [st.acquire()[0] for _ in range(n)]
+    jobs = [jobs[saved[k]] for k in held]
+    outs, optrs = [], []
+    for ptrs, metas, total in jobs[:n]:
+        o = torch.empty(total, dtype=torch.uint8, device=dev)  # tensors laid out like the blob: any addresses would do
+        outs.append(o)
+        optrs.append([o.data_ptr() + off for off, _ in metas])
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k, (ptrs, metas, total), op in zip(held, jobs, optrs):
+        st.load(k, total, metas, op, stream=stream)
+    for k in held:
+        st.release(k)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    ok = True
+    for (ptrs, metas, total), o in zip(jobs, outs):
+        for p, (off, nb) in list(zip(ptrs, metas))[:: max(1, len(metas) // 256)]:
+            if nb:
+                a = o[off:off + nb]
+                b = _view_at(p, nb, dev)
+                ok = ok and bool(torch.equal(a, b))
+    nbytes = sum(t for _, _, t in jobs[:n])
+    return {"blobs": n, "bytes": nbytes, "wall_s": wall, "device_gbps": nbytes / wall / 1e9, "round_trip_ok": ok}
+
+
+def _view_at(address: int, nbytes: int, dev):
+    """uint8 tensor over device memory at a raw address (the rank's tensors are known to the bench by address)."""
+    import ctypes
+
+    import torch
+
+    class _Iface:  # the CUDA array interface is the one way to wrap a raw device address without a copy
+        def __init__(self, ptr, n):
+            self.__cuda_array_interface__ = {"shape": (n,), "typestr": "|u1", "data": (ptr, False), "version": 3}
+
+    return torch.as_tensor(_Iface(address, nbytes), device=dev)
 
 
 def run_e2e(a, case, plan, src, dst, dev, ws, b_min):
