@@ -148,9 +148,10 @@ typedef struct {
                                written to every member's target (fewer L2 reads; over PCIe, fewer reads
                                at all); 2: every unit is staged on its own (bcp_reshard_host still groups
                                when it works in place)                                                     */
-  uint32_t test_stall;      /* test hook, 0 in normal use: 1 makes the first CTA of the TMA kernel arm its
-                               first stage for more bytes than it loads, so that exactly one bounded wait
-                               runs out and the time-out path can be exercised without any fault          */
+  uint32_t test_stall;      /* test hook, 0 in normal use: 1 makes the first CTA of each staging kernel (copy and
+                               conversion) arm its first stage for more bytes than it loads, so that exactly
+                               one bounded wait per kernel runs out and the time-out path can be exercised
+                               without any fault                                                          */
   uint32_t convert;         /* 0 default: entries of one FQN must agree on itemsize and dtype_tag, bytes are
                                moved unchanged.  BCP_CONVERT_F32_TO_BF16 / BCP_CONVERT_BF16_TO_F32: an FQN
                                whose saved entries have dtype_tag convert_src_tag and whose wanted entries have

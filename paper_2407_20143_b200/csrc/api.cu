@@ -196,6 +196,7 @@ int launch_units(bcp_plan_t* p, const bcp_tile* tiles, size_t n_tma, size_t n_bi
     c.n_stages = p->cvt_stages;
     c.grid = p->cvt_staged_grid;
     c.wait_ns = uint64_t(p->opt.tma_wait_ms) * 1000000ull;
+    c.test_stall = p->opt.test_stall;
     BCP_CUDA(launch_convert_staged(c, stream));
   }
   if (n_cvt && p->n_cvt_staged < p->n_cvt) {

@@ -330,7 +330,7 @@ struct CvtChunk {  // what one stage holds: `rows` source rows of `ne` elements,
 __global__ void __launch_bounds__(32) bcp_convert_staged_kernel(const bcp_tile* __restrict__ tiles, uint32_t n_units,
                                                                 const void* const* __restrict__ src, void* const* __restrict__ dst,
                                                                 Control* ctrl, uint32_t stage_bytes, uint32_t n_stages,
-                                                                uint64_t wait_ns) {
+                                                                uint64_t wait_ns, uint32_t test_stall) {
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full[kMaxStages];
   __shared__ CvtChunk held[kMaxStages];
@@ -400,6 +400,7 @@ __global__ void __launch_bounds__(32) bcp_convert_staged_kernel(const bcp_tile* 
     return true;
   };
 
+  bool first_load = true;
   auto issue_load = [&](uint32_t stage, const CvtChunk& ch) {
     const uint32_t bar = smem_u32(&full[stage]);
     const uint32_t base = smem_u32(stage_mem) + stage * stage_bytes;
@@ -413,8 +414,10 @@ __global__ void __launch_bounds__(32) bcp_convert_staged_kernel(const bcp_tile* 
     for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
     if (lane == 0) {
       held[stage] = ch;
-      mbar_expect_tx(bar, mine);
+      // test hook: the very first stage of CTA 0 is armed for 16 bytes that never arrive
+      mbar_expect_tx(bar, mine + ((test_stall && blockIdx.x == 0 && first_load) ? 16u : 0u));
     }
+    first_load = false;
     __syncwarp();
     for (uint32_t r = lane; r < ch.rows; r += 32) {
       const char* a = ch.src + uint64_t(r) * ch.sp;
@@ -538,7 +541,8 @@ cudaError_t launch_convert_staged(const ConvertStagedLaunchArgs& a, cudaStream_t
   if (a.n_stages < 2 || a.n_stages > uint32_t(kMaxStages) || a.stage_bytes % 128 || a.stage_bytes < 1024) return cudaErrorInvalidValue;
   const size_t smem = size_t(a.stage_bytes) * a.n_stages;
   const uint32_t grid = a.n_units < a.grid ? a.n_units : a.grid;
-  bcp_convert_staged_kernel<<<grid, 32, smem, stream>>>(a.tiles, a.n_units, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages, a.wait_ns);
+  bcp_convert_staged_kernel<<<grid, 32, smem, stream>>>(a.tiles, a.n_units, a.src, a.dst, a.ctrl, a.stage_bytes, a.n_stages, a.wait_ns,
+                                                        a.test_stall);
   return cudaGetLastError();
 }
 

@@ -68,6 +68,7 @@ struct ConvertStagedLaunchArgs {
   uint32_t n_stages;      // 2..8
   uint32_t grid;
   uint64_t wait_ns;       // how long a CTA waits for one stage before it gives up (global timer)
+  uint32_t test_stall;    // test hook: CTA 0 over-arms its first stage so that one wait runs out
 };
 
 // Persistent grid of the staged converting kernel (one warp per CTA) for a stage geometry.

@@ -177,6 +177,34 @@ def test_bounded_wait_runs_out_and_is_reported(cuda_device):
     assert np.array_equal(dst2[0].cpu().numpy(), want[0]) and guards_intact(backs, case.dst.buf_bytes)
 
 
+def test_bounded_wait_of_the_staged_converting_kernel(cuda_device):
+    """The same for the staged converting kernel: one over-armed stage, a 20 ms wait that runs out, the status
+    word, and an exact converting plan on the same device right afterwards."""
+    case = convert_cases()[1]
+    host = fills.fill_state(case.src, case.key_ids, "uniform", case.seed, "cpu")
+    want = orc.reshard(case.src.metas, [h.numpy() for h in host], case.dst.metas, case.dst.buf_bytes, fill_byte=POISON, convert=case.convert)
+    src = [h.to(cuda_device) for h in host]
+    opts = dict(case.plan_opts, path_mask=3, tma_min_row_bytes=16)
+    stalled = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, test_stall=1, tma_wait_ms=20, **opts)
+    assert any(t.flags & api.TILE_TMA and t.flags & api.TILE_CVT_MASK for t in stalled.tiles())
+    dst, _ = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(stalled, src, dst)
+    with pytest.raises(bcp.BcpError) as e:
+        bcp.bcp_plan_device_status(stalled)
+    assert e.value.code == api.ERR_DEVICE_TIMEOUT
+    torch.cuda.synchronize()  # no sticky error: the kernel returned normally
+    assert any(not np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst, want)), "the stalled CTA's unit stays incomplete"
+    bcp.bcp_plan_device_status(stalled)
+    stalled.destroy()
+    plan = bcp.bcp_plan(case.src.metas, case.src.buf_bytes, case.dst.metas, case.dst.buf_bytes, **opts)
+    dst2, backs = guarded(case.dst.buf_bytes, cuda_device)
+    bcp.bcp_reshard(plan, src, dst2)
+    torch.cuda.synchronize()
+    bcp.bcp_plan_device_status(plan)
+    assert all(np.array_equal(d.cpu().numpy(), w) for d, w in zip(dst2, want)) and guards_intact(backs, case.dst.buf_bytes)
+    plan.destroy()
+
+
 def test_side_stream_and_plan_reuse(cuda_device):
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
