@@ -108,6 +108,7 @@ def test_two_processes_zero_copy_and_exchange(cuda_device):
     import subprocess
     import sys
 
+    torch.cuda.empty_cache()  # what this process has cached is not available to the two ranks
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     worker = os.path.join(root, "tests", "two_process_worker.py")
     port = 29700 + os.getpid() % 200
