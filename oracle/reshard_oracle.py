@@ -30,7 +30,8 @@ the even one on a tie), not from a bit trick.
 
 Pins (tests/test_oracle_pins.py): the paper's worked example of an irregular shard, the
 identity / round-trip / exact-cover invariants, textbook reductions to numpy concatenate
-and split, a brute-force per-element index map on tiny inputs, and the closed-form
+and split, a brute-force per-element index map on tiny inputs (also with replicated saved
+shards, where the first holder in input order supplies the bytes), and the closed-form
 index-pattern fill; for the conversions, hand-worked bit patterns (tests/golden/
 f32_to_bf16_examples.txt), torch's own cast on everything but NaN, and the half-ulp error
 bound.  No function here is "parity unpinned".
