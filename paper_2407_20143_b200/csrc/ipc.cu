@@ -24,6 +24,7 @@ struct Mapping {  // one opened allocation of another process
   unsigned char handle[64];
   int device;
   char* base;
+  uint64_t bytes;  // size of the mapped allocation
   unsigned refs;
 };
 std::mutex g_mu;
@@ -105,6 +106,7 @@ int bcp_ipc_open(const bcp_ipc_handle* h, void** out_ptr) {
   memcpy(m.handle, h->handle, 64);
   m.device = dev;
   m.base = static_cast<char*>(base);
+  m.bytes = h->offset + h->bytes_after;
   m.refs = 1;
   g_maps.push_back(m);
   *out_ptr = m.base + h->offset;
@@ -114,10 +116,9 @@ int bcp_ipc_open(const bcp_ipc_handle* h, void** out_ptr) {
 int bcp_ipc_close(void* ptr) {
   if (!ptr) return BCP_OK;
   std::lock_guard<std::mutex> lock(g_mu);
-  // the mapping with the highest base at or below ptr (mapped allocations do not overlap)
-  Mapping* best = nullptr;
+  Mapping* best = nullptr;  // the mapped allocation that contains ptr
   for (Mapping& m : g_maps)
-    if (m.base <= static_cast<char*>(ptr) && (!best || m.base > best->base)) best = &m;
+    if (m.base <= static_cast<char*>(ptr) && static_cast<char*>(ptr) - m.base < ptrdiff_t(m.bytes ? m.bytes : 1)) best = &m;
   if (!best) return fail(BCP_ERR_INVALID, "bcp_ipc_close: %p was not returned by bcp_ipc_open", ptr);
   if (--best->refs == 0) {
     int cur = 0;

@@ -51,6 +51,11 @@ def main():
         for d, b in zip(dst, zc.local_dst):
             assert np.array_equal(d.cpu().numpy(), want[b]), ("zero-copy", case.name, rank, b)
         dist.barrier()  # nobody reads any more: blobs may go
+        try:
+            bcp.api.bcp_ipc_close(blobs[0].data_ptr())  # an address that no bcp_ipc_open returned
+            raise AssertionError("closing a pointer that was never opened must fail")
+        except bcp.BcpError as e:
+            assert e.code == bcp.api.ERR_INVALID
         zc.close()
 
         # (2) the exchange: pack on the GPU, segments through a real collective, two plans
