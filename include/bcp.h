@@ -17,7 +17,8 @@
  *     matching segments are copied into it (Sec. 3.3, Step 2 and Step 5).
  *
  * A "storage file" is a device buffer here (a blob); all source ranks and all target
- * ranks are separate buffers on ONE GPU.  The engine moves raw bytes unchanged, unless
+ * ranks are separate buffers, normally on ONE GPU (source blobs may also be another GPU's
+ * memory mapped into this process: bcp_ipc_*).  The engine moves raw bytes unchanged, unless
  * bcp_plan_opts.convert asks for a binary32 <-> bfloat16 conversion of some tensors.
  *
  * Conventions
