@@ -401,7 +401,7 @@ void* split_addresses(const void* const* tensors, size_t n, void* blob, std::vec
 
 extern "C" {
 
-int bcp_version(void) { return 201; }  // 0.2.1: plan options (and so plan images) carry the source-buffer range
+int bcp_version(void) { return 202; }  // 0.2.2: plan options (and so plan images) carry the source-buffer range and the run unit size
 
 const char* bcp_last_error(void) { return last_error().c_str(); }
 

@@ -32,10 +32,11 @@ struct Item {
 
 struct Options {
   uint32_t tile_bytes = 65536;
+  uint32_t run_tile_bytes = 0;  // unit size of 16-byte aligned contiguous runs; 0: chosen from the work list (see build_tiles)
   uint32_t small_bytes = 4096;
   uint32_t block_threads = 512;
   uint32_t ctas_per_sm = 0;  // 0: chosen from the work list
-  uint32_t order = 1;
+  uint32_t order = 0;  // 0: chosen from the work list (see build_tiles)
   uint32_t path_mask = 0;  // 0: decided from the work list
   uint32_t cache_hints = 1;
   uint32_t tma_stage_bytes = 0;  // 0: chosen from the work list (see build_tiles)
