@@ -45,8 +45,10 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     ("cfg2", "bcp_tma_kernel"): (0.9994, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369",
                                  "full size; the 2-layer capture was redone when the kernel gained its tail units: 0.993 before and after"),
-    ("cfg3", "bcp_tma_kernel"): (0.9990, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369", "full size (staged path unchanged since)"),
-    ("cfg4", "bcp_tma_kernel"): (0.9998, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "0874854", "full size (staged path unchanged since)"),
+    ("cfg3", "bcp_tma_kernel"): (0.9915, "profiles/bcp_tma_kernel_cfg3-L2_ncu_full.md", "4497f17",
+                                 "2 layers (5.9 GB), units in target order; the full-size capture in source order read 0.9990"),
+    ("cfg4", "bcp_tma_kernel"): (0.9998, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "0874854",
+                                 "full size, in source order (the default is target order now; cfg3's 2-layer re-capture shows the traffic unchanged)"),
     ("evalmerge", "bcp_convert_kernel"): (0.9961, "profiles/bcp_convert_staged_kernel_evalmerge-L2_ncu_full.md", "4f5ee6b", "2 layers (8.9 GB)"),
 }
 
