@@ -23,8 +23,8 @@ def _draw(rng, it, scen):
         case = big_random_case(seed, itemsize=int(rng.choice([1, 2, 4, 8])), gap_mod=int(rng.choice([0, 1, 4, 7, 8])))
     else:
         case = scen[int(rng.integers(0, len(scen)))]
-    opts = dict(path_mask=int(rng.choice([0, 1, 3, 7])), tile_bytes=int(rng.choice([4096, 8192, 16384, 65536, 262144])),
-                fanout=int(rng.choice([1, 2])), order=int(rng.choice([1, 1, 2])),
+    opts = dict(path_mask=int(rng.choice([0, 1, 3, 7])), tile_bytes=int(rng.choice([0, 4096, 8192, 16384, 65536, 262144])),
+                fanout=int(rng.choice([1, 2])), order=int(rng.choice([0, 1, 2])),
                 tma_stage_bytes=int(rng.choice([1024, 2048, 4096, 16384, 32768])), tma_stages=int(rng.choice([2, 3, 4, 6])),
                 tma_ctas_per_sm=int(rng.choice([1, 2, 4])), tma_min_row_bytes=int(rng.choice([16, 64, 512, 2048])),
                 worker=int(rng.choice([1, 2])), unroll=int(rng.choice([4, 8])), block_threads=int(rng.choice([256, 512, 1024])),
@@ -63,7 +63,7 @@ def test_random_converting_problems_and_options(cuda_device, stream_seed):
     for it in range(30):
         seed = int(rng.integers(0, 1 << 30))
         case = random_convert_case(seed, narrow=bool(it % 2), big=it % 3 == 0, dst_replicas=int(rng.integers(1, 3)))
-        opts = dict(path_mask=int(rng.choice([0, 1, 3, 7])), tile_bytes=int(rng.choice([4096, 8192, 65536])), order=int(rng.choice([1, 2])),
+        opts = dict(path_mask=int(rng.choice([0, 1, 3, 7])), tile_bytes=int(rng.choice([4096, 8192, 65536])), order=int(rng.choice([0, 1, 2])),
                     tma_min_row_bytes=int(rng.choice([16, 512])), worker=int(rng.choice([1, 2])), small_bytes=int(rng.choice([64, 4096])))
         g = torch.Generator(device="cpu").manual_seed(seed)
         host = [torch.randint(0, 256, (n,), dtype=torch.uint8, generator=g) for n in case.src.buf_bytes]
