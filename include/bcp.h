@@ -110,10 +110,13 @@ typedef struct {
   uint32_t small_bytes;    /* work units with a payload below this go to the warp path; default 4096  */
   uint32_t block_threads;  /* threads per CTA of the register kernel: 256, 512 or 1024; default 512     */
   uint32_t ctas_per_sm;    /* register path: persistent CTAs per SM; default 2 (4 with worker 2)       */
-  uint32_t order;          /* 1 order work by source address (replica reads of one source region run back to
-                              back, are staged once and hit L2); 2 order by target address (the pieces of one
-                              stretch of a target are written at about the same time); 0 default: 1 when
-                              source bytes are wanted more than once (DP replicas), else 2               */
+  uint32_t order;          /* 1 units that read the same source bytes (replicas of a target shard) side by side,
+                              so that they are staged once and hit L2: the lists are in source-address order,
+                              and the staged units are then rearranged group by group into the order of each
+                              group's first target address; 2 order by target address (the pieces of one
+                              stretch of a target are written at about the same time; replicas are not
+                              grouped); 0 default: 1 when source bytes are wanted more than once (DP
+                              replicas), else 2                                                          */
   uint32_t path_mask;      /* which kernels execute the list.
                               1 every unit goes through registers (LDG/STG kernel);
                               3 runs of at least tma_min_row_bytes (any alignment) and rectangles with rows of
