@@ -115,8 +115,9 @@ typedef struct {
                               and the staged units are then rearranged group by group into the order of each
                               group's first target address; 2 order by target address (the pieces of one
                               stretch of a target are written at about the same time; replicas are not
-                              grouped); 0 default: 1 when source bytes are wanted more than once (DP
-                              replicas), else 2                                                          */
+                              grouped); 3 plain source-address order (replicas side by side, nothing
+                              rearranged); 0 default: 2 when every source byte is wanted once, else 1 if
+                              the plan has strided rectangles, else 3                                    */
   uint32_t path_mask;      /* which kernels execute the list.
                               1 every unit goes through registers (LDG/STG kernel);
                               3 runs of at least tma_min_row_bytes (any alignment) and rectangles with rows of

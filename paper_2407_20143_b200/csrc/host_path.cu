@@ -117,7 +117,7 @@ int bcp_reshard_host(bcp_plan_t* plan, const void* const* src_host, size_t n_src
       if (p->dst_bytes[i]) mapped = device_view(dst_host[i], &ddst[i]);
     if (mapped) {
       // over PCIe every read costs: stage each source piece once and write all its replicas from it
-      if (!p->d_fan_tiles && p->n_tma && p->opt.order == 1 && p->opt.fanout != 1) {
+      if (!p->d_fan_tiles && p->n_tma && p->opt.order != 2 && p->opt.fanout != 1) {
         std::vector<bcp_tile> fan(p->tiles.begin(), p->tiles.end());
         mark_followers(fan.data(), p->n_tma);
         BCP_CUDA(cudaMalloc(&p->d_fan_tiles, fan.size() * sizeof(bcp_tile)));

@@ -198,7 +198,7 @@ int bcp_plan_deserialize(const void* image, size_t n, bcp_plan_t** out_plan) {
   {  // replica groups must be exactly what the planner would mark: a follower is never staged itself
     std::vector<bcp_tile> again(p->tiles.begin(), p->tiles.begin() + p->n_tma);
     for (bcp_tile& t : again) t.flags &= ~(BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT));
-    if (p->opt.fanout == 1 && p->opt.order == 1) mark_followers(again.data(), again.size());
+    if (p->opt.fanout == 1 && p->opt.order != 2) mark_followers(again.data(), again.size());
     bool ok = true;
     for (size_t i = 0; ok && i < p->tiles.size(); ++i)
       ok = i < p->n_tma ? again[i].flags == p->tiles[i].flags : !(p->tiles[i].flags & (BCP_TILE_FOLLOW | (7u << BCP_TILE_FAN_SHIFT)));

@@ -67,7 +67,7 @@ int parse_options(const bcp_plan_opts* in, Options* out) {
   if (o.block_threads != 256 && o.block_threads != 512 && o.block_threads != 1024)
     return fail(BCP_ERR_INVALID, "block_threads must be 256, 512 or 1024");
   if (o.ctas_per_sm > 16) return fail(BCP_ERR_INVALID, "ctas_per_sm must be in [1, 16]");
-  if (o.order > 2) return fail(BCP_ERR_INVALID, "order must be 0, 1 or 2");
+  if (o.order > 3) return fail(BCP_ERR_INVALID, "order must be 0, 1, 2 or 3");
   if (o.path_mask != 0 && o.path_mask != 1 && o.path_mask != 3 && o.path_mask != 7)
     return fail(BCP_ERR_INVALID, "path_mask must be 0, 1, 3 or 7");
   if (o.tma_stage_bytes && (o.tma_stage_bytes % 128 || o.tma_stage_bytes < 1024 || o.tma_stage_bytes > 65536))

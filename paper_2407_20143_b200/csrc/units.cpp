@@ -346,8 +346,11 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   // come from several saved shards -- are then written at about the same time; measured: cfg3 1.2 %, cfg4 0.6 %,
   // the converting 8B merge 0.8 % faster than in source order; cfg5, where an eighth of the target bytes are
   // replicas, 5 % slower).  Under order 1 the staged units get both: replicas side by side, and these groups in
-  // the order of their first member's target address (cfg2 6.66 -> 6.59 ms).
-  if (!opt.order) opt.order = (uniq && written > uniq + uniq / 50) ? 1 : 2;
+  // the order of their first member's target address; that pays when the plan has rectangles, whose target rows
+  // are completed by pieces from several shards (cfg2 6.66 -> 6.59 ms), and costs a little when it has only runs
+  // (cfg5 17.00 -> 17.08 ms), which stay in plain source order (3).  Decided after the counting pass below.
+  const bool choose_order = !opt.order;
+  const bool reads_twice = uniq && written > uniq + uniq / 50;
 
   // Pass 1: how many units of each class (and rectangles) every item gives.  A rough unit count
   // decides whether helpers are worth starting.
@@ -372,6 +375,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   });
   Tally all;
   for (const Tally& t : tally) all.add(t);
+  if (choose_order) opt.order = !reads_twice ? 2 : all.n_strided ? 1 : 3;
   // Tiny jobs stay in the register kernel.  From 4 MiB of stageable payload on the staging kernel is
   // the faster one (measured with L2 flushed, runs of 1 MiB..1 GiB: 10-12 us against 12 us up to 4 MiB,
   // 14 / 16 us at 16 MiB, 31 / 33 us at 64 MiB, 90 / 94 us at 256 MiB; rectangles with 2 KiB rows: 14 / 21 us
@@ -440,7 +444,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
   // Order every class by source address (order 1: the reads of replicas meet in L2) or by target
   // address, through compact keys, and gather the units into the final list.
   std::unique_ptr<Key[]> keys(new Key[total ? total : 1]), spare(new Key[total ? total : 1]);
-  const bool by_src = opt.order == 1;
+  const bool by_src = opt.order != 2;
   const size_t kChunk = 65536;
   parallel_jobs((total + kChunk - 1) / kChunk, threads, [&](size_t j) {
     for (size_t i = j * kChunk; i < std::min(total, (j + 1) * kChunk); ++i) {
@@ -459,7 +463,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     bcp_tile* dst = tiles->data() + base;
     const bcp_tile* src = cls[k];
     std::unique_ptr<Key[]> again, again_spare;
-    if (k == kTma && by_src && n > 1) {
+    if (k == kTma && opt.order == 1 && n > 1) {
       // Second key of the staged class: units that read the same source bytes (neighbours in source order) form
       // a group; a group is keyed by the target address of its first member, a member by its place in the group.
       again.reset(new Key[n]);
@@ -481,7 +485,7 @@ void build_tiles(std::vector<Item>& items, Options& opt, const std::vector<uint6
     });
     base += n;
   }
-  if (opt.order == 1 && opt.fanout == 1) mark_followers(tiles->data(), run.n[kTma]);
+  if (opt.order != 2 && opt.fanout == 1) mark_followers(tiles->data(), run.n[kTma]);
   stats->n_tiles = run.n[kTma] + run.n[kBig];
   stats->n_small_tiles = run.n[kSmall];
   *n_tma = run.n[kTma];
