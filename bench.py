@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # roofline.traffic_note so that a stale ratio is visible.
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     ("cfg2", "bcp_tma_kernel"): (0.9994, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "07a4369",
-                                 "full size; the 2-layer capture was redone when the kernel gained its tail units: 0.993 before and after"),
+                                 "full size, in plain source order; the 2-layer capture was redone when the kernel gained its tail units: 0.993 before and after; the order of the replica groups changed since (same groups, same bytes)"),
     ("cfg3", "bcp_tma_kernel"): (0.9915, "profiles/bcp_tma_kernel_cfg3-L2_ncu_full.md", "4497f17",
                                  "2 layers (5.9 GB), units in target order; the full-size capture in source order read 0.9990"),
     ("cfg4", "bcp_tma_kernel"): (0.9998, "profiles/bcp_tma_kernel_full_size_dram_bytes.md", "0874854",
